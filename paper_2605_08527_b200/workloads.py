@@ -1,0 +1,323 @@
+"""Seeded synthetic inputs for the multi-tenant LoRA layer.
+
+This module only *draws numbers*: it contains no part of the layer's arithmetic
+(no products, no gradients), so that the CPU oracle and the CUDA path can both be fed
+from it without sharing any of the method's code.  Everything is a pure function of
+(seed, tensor id, element index): a 64-bit counter hash gives two uniforms per element,
+Box-Muller turns them into a normal deviate, and the value is rounded to bf16
+(round-to-nearest-even) because the layer's inputs are bf16 tensors.
+
+The five workloads mirror the shapes of the paper's multi-task RLVR runs (Experimental
+Setup: up to 32 concurrent tasks, 10 replicas, generation lengths up to 4096, decode
+batches of one token per sequence); the paper's datasets themselves are not used.
+
+Arrays are numpy: bf16 tensors are returned as ``uint16`` bit patterns (``*_bits``) and
+the same values widened exactly to ``float32``.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Dict, List, Optional
+
+import numpy as np
+
+BASE_SEED = 0x4D41524C  # "MARL"
+
+# tensor ids of the counter hash
+TID_W, TID_X, TID_DY, TID_A, TID_B, TID_TABLE, TID_RANKS, TID_PERTURB = 1, 2, 3, 4, 5, 6, 7, 8
+
+_M1 = np.uint64(0xBF58476D1CE4E5B9)
+_M2 = np.uint64(0x94D049BB133111EB)
+_GOLD = np.uint64(0x9E3779B97F4A7C15)
+
+
+def _mix64(z: np.ndarray) -> np.ndarray:
+    """SplitMix64 finaliser, vectorised over a uint64 array (wraps modulo 2**64)."""
+    z = (z ^ (z >> np.uint64(30))) * _M1
+    z = (z ^ (z >> np.uint64(27))) * _M2
+    return z ^ (z >> np.uint64(31))
+
+
+def _stream_key(seed: int, tensor_id: int, sub: int = 0) -> np.uint64:
+    k = (seed * 0x9E3779B97F4A7C15 + tensor_id * 0xD1B54A32D192ED03 + sub * 0x8CB92BA72F3D8DD7) & (2**64 - 1)
+    with np.errstate(over="ignore"):
+        return _mix64(np.array([k], dtype=np.uint64))[0]
+
+
+def hash_u64(seed: int, tensor_id: int, index: np.ndarray, sub: int = 0) -> np.ndarray:
+    """64 hashed bits per counter value ``index`` (any integer array)."""
+    key = _stream_key(seed, tensor_id, sub)
+    with np.errstate(over="ignore"):
+        return _mix64(index.astype(np.uint64) * _GOLD + key)
+
+
+def uniform01(seed: int, tensor_id: int, index: np.ndarray, sub: int = 0) -> np.ndarray:
+    """Uniform doubles in (0, 1): top 53 bits of the hash, offset by half an ulp."""
+    h = hash_u64(seed, tensor_id, index, sub)
+    return ((h >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+
+
+def f32_to_bf16_bits(v: np.ndarray) -> np.ndarray:
+    """Round float32 to bf16 (1-8-7), round-to-nearest-even; returns uint16 bit patterns."""
+    b = np.ascontiguousarray(v, dtype=np.float32).view(np.uint32)
+    bias = np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))
+    return ((b + bias) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def normal_bf16(seed: int, tensor_id: int, shape, sigma: float, sub: int = 0, chunk: int = 1 << 22):
+    """bf16-rounded N(0, sigma^2) tensor -> (bits uint16, values float32), element i of the
+    flattened tensor uses counters 2i and 2i+1."""
+    n = int(np.prod(shape))
+    bits = np.empty(n, dtype=np.uint16)
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        idx = np.arange(lo, hi, dtype=np.uint64)
+        u1 = uniform01(seed, tensor_id, idx * np.uint64(2), sub)
+        u2 = uniform01(seed, tensor_id, idx * np.uint64(2) + np.uint64(1), sub)
+        z = np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)
+        bits[lo:hi] = f32_to_bf16_bits((z * sigma).astype(np.float32))
+    bits = bits.reshape(shape)
+    return bits, bf16_bits_to_f32(bits)
+
+
+@dataclasses.dataclass
+class Adapter:
+    """One tenant's LoRA parameters: A is d_in x rank, B is rank x d_out, scale = alpha / rank."""
+    tenant_id: int
+    rank: int
+    alpha: float
+    A_bits: np.ndarray
+    B_bits: np.ndarray
+
+    @property
+    def scale(self) -> float:
+        return self.alpha / self.rank if self.rank > 0 else 0.0
+
+    @property
+    def A(self) -> np.ndarray:
+        return bf16_bits_to_f32(self.A_bits)
+
+    @property
+    def B(self) -> np.ndarray:
+        return bf16_bits_to_f32(self.B_bits)
+
+
+@dataclasses.dataclass
+class Projection:
+    """One adapted projection: a frozen base weight shared by all tenants plus one adapter per tenant."""
+    name: str
+    d_in: int
+    d_out: int
+    W_bits: np.ndarray
+    adapters: List[Adapter]
+    x_bits: np.ndarray                  # [T][d_in]
+    dy_bits: Optional[np.ndarray]       # [T_bwd][d_out] or None (forward-only workload)
+
+    @property
+    def W(self) -> np.ndarray:
+        return bf16_bits_to_f32(self.W_bits)
+
+    @property
+    def x(self) -> np.ndarray:
+        return bf16_bits_to_f32(self.x_bits)
+
+    @property
+    def dy(self) -> Optional[np.ndarray]:
+        return None if self.dy_bits is None else bf16_bits_to_f32(self.dy_bits)
+
+
+@dataclasses.dataclass
+class Workload:
+    """A mixed batch: the token-to-adapter segment table plus the projections it is run through.
+
+    seg_offsets[S+1] / seg_slot[S] describe contiguous token ranges; slot j means the j-th
+    adapter of every projection (slot -1 = base weight only).  ``T_bwd`` rows (a prefix of
+    the batch) take part in the backward pass; 0 means forward only.
+    """
+    name: str
+    T: int
+    T_bwd: int
+    seg_offsets: np.ndarray
+    seg_slot: np.ndarray
+    projections: List[Projection]
+    n_tenants: int
+    max_rank: int
+
+    def tok_slot(self) -> np.ndarray:
+        """Per-token slot by plain expansion of the table (input bookkeeping, not the method's index build)."""
+        out = np.empty(self.T, dtype=np.int32)
+        for s in range(len(self.seg_slot)):
+            out[self.seg_offsets[s]:self.seg_offsets[s + 1]] = self.seg_slot[s]
+        return out
+
+
+def _make_adapters(seed, n, ranks, alphas, d_in, d_out, proj_index) -> List[Adapter]:
+    out = []
+    for t in range(n):
+        r = int(ranks[t])
+        a_bits, _ = normal_bf16(seed, TID_A, (d_in, r), 0.02, sub=proj_index * 4096 + t)
+        b_bits, _ = normal_bf16(seed, TID_B, (r, d_out), 0.02, sub=proj_index * 4096 + t)
+        out.append(Adapter(tenant_id=1000 + t, rank=r, alpha=float(alphas[t]), A_bits=a_bits, B_bits=b_bits))
+    return out
+
+
+def _make_projection(seed, name, d_in, d_out, n, ranks, alphas, T, T_bwd, proj_index, x_group) -> Projection:
+    w_bits, _ = normal_bf16(seed, TID_W, (d_in, d_out), 0.02, sub=proj_index)
+    x_bits, _ = normal_bf16(seed, TID_X, (T, d_in), 1.0, sub=x_group)
+    dy_bits = None
+    if T_bwd > 0:
+        dy_bits, _ = normal_bf16(seed, TID_DY, (T_bwd, d_out), 1.0, sub=proj_index)
+    return Projection(name, d_in, d_out, w_bits, _make_adapters(seed, n, ranks, alphas, d_in, d_out, proj_index),
+                      x_bits, dy_bits)
+
+
+def lognormal_segments(seed: int, T: int, n_tenants: int, sub: int = 0, shrink: int = 1):
+    """Per-tenant training segments: lengths clip(round(exp(N(ln 1024, 0.6^2))), 128, 4096) drawn until
+    they cover T tokens; the last one is shortened to fit and, if that leaves fewer than 128 tokens,
+    merged into its predecessor.  Segment j (after a seeded shuffle of the order) belongs to tenant
+    j mod n_tenants.  ``shrink`` divides median and clip bounds (scaled-down test cases)."""
+    med, lo_len, hi_len = 1024.0 / shrink, max(1, 128 // shrink), max(1, 4096 // shrink)
+    lens = []
+    total, c = 0, 0
+    while total < T:
+        idx = np.array([2 * c, 2 * c + 1], dtype=np.uint64)
+        u = uniform01(seed, TID_TABLE, idx, sub)
+        z = math.sqrt(-2.0 * math.log(u[0])) * math.cos(2.0 * math.pi * u[1])
+        L = int(min(hi_len, max(lo_len, round(math.exp(math.log(med) + 0.6 * z)))))
+        lens.append(L)
+        total += L
+        c += 1
+    lens[-1] -= total - T
+    if lens[-1] < lo_len and len(lens) > 1:
+        lens[-2] += lens[-1]
+        lens.pop()
+    S = len(lens)
+    slots = np.arange(S, dtype=np.int64) % n_tenants
+    # seeded Fisher-Yates shuffle of the (length, tenant) pairs
+    order = np.arange(S)
+    for i in range(S - 1, 0, -1):
+        h = int(hash_u64(seed, TID_TABLE, np.array([1_000_000 + i], dtype=np.uint64), sub)[0])
+        j = h % (i + 1)
+        order[i], order[j] = order[j], order[i]
+    lens = np.asarray(lens, dtype=np.int64)[order]
+    slots = slots[order]
+    offsets = np.zeros(S + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum(lens)
+    return offsets, slots.astype(np.int32)
+
+
+def uniform_token_slots(seed: int, T: int, n_tenants: int, sub: int = 0) -> np.ndarray:
+    """Decode batch: one tenant id per token, uniform over the tenants, unsorted."""
+    h = hash_u64(seed, TID_TABLE, np.arange(T, dtype=np.uint64), sub + 77)
+    return (h % np.uint64(n_tenants)).astype(np.int32)
+
+
+def zipf_segments(seed: int, T: int, n_tenants: int, s: float = 1.1, max_len: int = 2048, sub: int = 0):
+    # scaled-down callers pass a smaller max_len
+    """Skewed mixed batch: each segment's tenant ~ Zipf(s) over the tenants (P(t) ~ (t+1)^-s) and its
+    length is a log-uniform integer in [1, max_len]; the last segment is truncated to fit T."""
+    p = np.arange(1, n_tenants + 1, dtype=np.float64) ** (-s)
+    cdf = np.cumsum(p / p.sum())
+    lens, slots = [], []
+    total, c = 0, 0
+    while total < T:
+        u = uniform01(seed, TID_TABLE, np.array([2 * c, 2 * c + 1], dtype=np.uint64), sub + 31)
+        t = int(min(n_tenants - 1, np.searchsorted(cdf, u[0], side="right")))
+        L = int(min(max_len, max(1, math.floor(math.exp(u[1] * math.log(max_len + 1.0))))))
+        L = min(L, T - total)
+        lens.append(L)
+        slots.append(t)
+        total += L
+        c += 1
+    offsets = np.zeros(len(lens) + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum(lens)
+    return offsets, np.asarray(slots, dtype=np.int32)
+
+
+def per_token_table(tok_slot: np.ndarray):
+    T = len(tok_slot)
+    return np.arange(T + 1, dtype=np.int32), np.asarray(tok_slot, dtype=np.int32)
+
+
+def make_workload(cfg: int, scale_down: int = 1, seed: Optional[int] = None) -> Workload:
+    """Build workload ``cfg`` in 1..5.  ``scale_down`` > 1 divides the token count and the weight
+    dimensions by that factor (kept multiples of 64) to get a same-structure case the oracle can
+    finish quickly; 1 gives the full-size configuration."""
+    seed = BASE_SEED + cfg if seed is None else seed
+    sd = scale_down
+
+    def dim(v):
+        return max(64, (v // sd) // 64 * 64)
+
+    if cfg == 1:
+        K = N = dim(512)
+        n, T = 4, max(8, 256 // sd)
+        q = T // 4
+        offsets = np.array([0, q, 2 * q, 3 * q, T], dtype=np.int32)
+        slots = np.arange(4, dtype=np.int32)
+        ranks, alphas = [8] * n, [16.0] * n
+        projs = [_make_projection(seed, "proj", K, N, n, ranks, alphas, T, T, 0, 0)]
+        return Workload("cfg1-tiny", T, T, offsets, slots, projs, n, 8)
+    if cfg == 2:
+        K = N = dim(4096)
+        n, T = 32, max(8, 256 // sd)
+        offsets, slots = per_token_table(uniform_token_slots(seed, T, n))
+        ranks, alphas = [16] * n, [32.0] * n
+        projs = [_make_projection(seed, "proj", K, N, n, ranks, alphas, T, 0, 0, 0)]
+        return Workload("cfg2-decode", T, 0, offsets, slots, projs, n, 16)
+    if cfg == 3:
+        K, N = dim(4096), dim(11008)
+        n, T = 10, 16384 // sd
+        offsets, slots = lognormal_segments(seed, T, n, shrink=sd)
+        ranks, alphas = [32] * n, [64.0] * n
+        projs = [_make_projection(seed, "up", K, N, n, ranks, alphas, T, T, 0, 0)]
+        return Workload("cfg3-train", T, T, offsets, slots, projs, n, 32)
+    if cfg == 4:
+        K = N = dim(5120)
+        n, T = 32, 8192 // sd
+        offsets, slots = zipf_segments(seed, T, n, max_len=max(1, 2048 // sd))
+        rk = hash_u64(seed, TID_RANKS, np.arange(n, dtype=np.uint64)) % np.uint64(4)
+        ranks = [int((8, 16, 32, 64)[int(v)]) for v in rk]
+        alphas = [16.0] * n
+        projs = [_make_projection(seed, "proj", K, N, n, ranks, alphas, T, T, 0, 0)]
+        return Workload("cfg4-hetero", T, T, offsets, slots, projs, n, 64)
+    if cfg == 5:
+        H, F = dim(4096), dim(11008)
+        n = 32
+        Tt, Td = 4096 // sd, max(8, 256 // sd)
+        o1, s1 = lognormal_segments(seed, Tt, n, shrink=sd)
+        o2, s2 = per_token_table(uniform_token_slots(seed, Td, n))
+        offsets = np.concatenate([o1, (o2[1:] + Tt).astype(np.int32)]).astype(np.int32)
+        slots = np.concatenate([s1, s2]).astype(np.int32)
+        T = Tt + Td
+        ranks, alphas = [16] * n, [32.0] * n
+        shapes = [("q", H, H, 0), ("k", H, H, 0), ("v", H, H, 0), ("o", H, H, 1),
+                  ("gate", H, F, 2), ("up", H, F, 2), ("down", F, H, 3)]
+        projs = [_make_projection(seed, nm, di, do, n, ranks, alphas, T, Tt, pi, xg)
+                 for pi, (nm, di, do, xg) in enumerate(shapes)]
+        return Workload("cfg5-layer", T, Tt, offsets, slots, projs, n, 16)
+    raise ValueError(f"unknown config {cfg}")
+
+
+def small_random_case(seed: int, T: int, K: int, N: int, ranks, alphas=None, n_segments: int = 6,
+                      with_base_only: bool = True, sigma_w: float = 0.02) -> Workload:
+    """Small ragged case for tests: random segment boundaries (zero-length segments allowed), tenants may
+    recur in non-adjacent segments, one tenant may get no tokens, optional slot -1 segment."""
+    n = len(ranks)
+    alphas = [16.0] * n if alphas is None else alphas
+    cuts = np.sort(hash_u64(seed, TID_TABLE, np.arange(n_segments - 1, dtype=np.uint64), 5) % np.uint64(T + 1))
+    offsets = np.concatenate([[0], cuts.astype(np.int64), [T]]).astype(np.int32)
+    pick = hash_u64(seed, TID_TABLE, np.arange(n_segments, dtype=np.uint64), 6)
+    lo = -1 if with_base_only else 0
+    span = max(1, n - 1) - lo            # the last tenant never appears: exercises "registered but absent"
+    slots = (pick % np.uint64(span)).astype(np.int64) + lo
+    w_bits, _ = normal_bf16(seed, TID_W, (K, N), sigma_w)
+    x_bits, _ = normal_bf16(seed, TID_X, (T, K), 1.0)
+    dy_bits, _ = normal_bf16(seed, TID_DY, (T, N), 1.0)
+    proj = Projection("proj", K, N, w_bits, _make_adapters(seed, n, ranks, alphas, K, N, 0), x_bits, dy_bits)
+    return Workload(f"small-{seed}", T, T, offsets, slots.astype(np.int32), [proj], n, max(ranks) if ranks else 0)
