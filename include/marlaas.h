@@ -1,0 +1,163 @@
+/* marlaas.h -- C ABI of the B200 multi-tenant LoRA linear layer.
+ *
+ * The layer is the one every adapted projection of the shared base model runs when many tenants
+ * share one frozen base weight through lightweight LoRA adapters (paper: abstract; Introduction;
+ * Methods, "Multi-Task Manager" -- per-task LoRA parameters theta_t^(v) with a version counter --
+ * and "Multi-LoRA Rollout with Single-Task Training" -- rollouts batched across tasks by multi-LoRA
+ * kernels; Algorithm 1 "Commit updated parameters").  For a token i routed to tenant slot t:
+ *
+ *     y_i  = x_i W + s_t (x_i A_t) B_t                              (forward: rollout decode and training)
+ *     dx_i = dy_i W^T + s_t (dy_i B_t^T) A_t^T                      (backward)
+ *     dA_t = s_t sum_{i:t(i)=t} x_i^T (dy_i B_t^T)      dB_t = s_t sum_{i:t(i)=t} (x_i A_t)^T dy_i
+ *
+ * W is d_in x d_out (K x N), A_t is K x r_t, B_t is r_t x N, s_t = alpha_t / r_t; everything is
+ * row-major; x, W, A, B, y, dy, dx are bf16 (1-8-7, round-to-nearest-even on output), sums are
+ * carried in fp32, dA_t and dB_t are fp32.  W is frozen: there is no dW.
+ *
+ * Conventions
+ *  - All data pointers are DEVICE pointers on the pool's device unless a comment says HOST.
+ *  - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *    stream) and the calls return without synchronising unless MARLAAS_FLAG_VALIDATE_SYNC is given.
+ *    The caller keeps every buffer alive and unmodified until the stream has passed the call.
+ *  - The library never allocates or frees device memory: the adapter store and the per-call workspace
+ *    are caller-provided (sizes from the *_bytes functions).
+ *  - Every function returns MARLAAS_OK (0) or a negative marlaas_status_t; nothing throws or aborts.
+ *    marlaas_last_error() gives a thread-local message for the last failure on this thread.
+ *  - Arguments are validated on the host BEFORE anything is launched; a failing call launches nothing.
+ *  - A pool may be used from one host thread at a time.
+ *  - Required alignment: every bf16 pointer 16-byte aligned, every leading dimension a multiple of 8
+ *    elements, d_in and d_out multiples of 8.
+ */
+#ifndef MARLAAS_H_
+#define MARLAAS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct marlaas_pool marlaas_pool_t; /* opaque; one pool per adapted projection (d_in, d_out) */
+typedef int32_t marlaas_status_t;
+
+enum {
+    MARLAAS_OK = 0,
+    MARLAAS_ERR_INVALID_ARG = -1,        /* null / misaligned pointer, negative size, leading dim too small */
+    MARLAAS_ERR_BAD_SEGMENT_TABLE = -2,  /* offsets not 0..T non-decreasing (host tables: before launch; device
+                                            tables: reported by marlaas_check_status) */
+    MARLAAS_ERR_UNKNOWN_TENANT = -3,
+    MARLAAS_ERR_RANK_TOO_LARGE = -4,
+    MARLAAS_ERR_POOL_FULL = -5,
+    MARLAAS_ERR_UNSUPPORTED_DEVICE = -6, /* not an sm_100 device, or no CUDA device */
+    MARLAAS_ERR_CUDA = -7,               /* a CUDA runtime / driver call failed */
+    MARLAAS_ERR_DEVICE_TIMEOUT = -8,     /* a bounded wait inside a kernel ran out; results of that call are invalid */
+    MARLAAS_ERR_DEVICE_BAD_INDEX = -9,   /* a device-side check met a slot outside [-1, capacity): that token was
+                                            computed with the base weight only */
+    MARLAAS_ERR_WORKSPACE_TOO_SMALL = -10
+};
+
+enum {
+    MARLAAS_FLAG_ACCUMULATE = 1u,     /* backward: dA_t, dB_t += instead of overwrite */
+    MARLAAS_FLAG_HOST_TABLE = 2u,     /* seg_offsets / seg_slot are HOST arrays: validated on the host, then copied
+                                         into the workspace in stream order */
+    MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
+    MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
+};
+
+/* Token-to-adapter segment table of one mixed batch: segment s covers tokens
+ * [seg_offsets[s], seg_offsets[s+1]) and routes them to pool slot seg_slot[s] (-1 = base weight only).
+ * seg_offsets[0] = 0, non-decreasing, seg_offsets[S] = T; zero-length segments are allowed; a slot may
+ * recur in any number of non-adjacent segments.  An unsorted decode batch is T segments of one token.
+ * The arrays are device memory unless MARLAAS_FLAG_HOST_TABLE is set. */
+typedef struct {
+    int32_t num_segments;       /* S >= 0 */
+    const int32_t* seg_offsets; /* [S+1] */
+    const int32_t* seg_slot;    /* [S]   */
+} marlaas_segments_t;
+
+/* ---- pooled adapter store (the manager's per-task parameters theta_t^(v), "Multi-Task Manager") ---- */
+
+/* Bytes of device memory a pool of `capacity` slots needs (0 if the arguments are invalid).
+ * max_rank in [1,128]; ranks are stored padded to a multiple of 16 with zero rows (exact). */
+size_t marlaas_adapter_pool_storage_bytes(int64_t d_in, int64_t d_out, int32_t max_rank, int32_t capacity);
+
+/* Create a pool over caller-owned device memory `storage` (256-byte aligned, >= storage_bytes, on
+ * `device`); clears it in stream order.  The pool object itself is host memory freed by _destroy; the
+ * storage stays the caller's.  Fails with UNSUPPORTED_DEVICE unless `device` has compute capability 10.x. */
+marlaas_status_t marlaas_adapter_pool_create(marlaas_pool_t** out, int device, int64_t d_in, int64_t d_out,
+                                             int32_t max_rank, int32_t capacity, void* storage,
+                                             size_t storage_bytes, void* cuda_stream);
+marlaas_status_t marlaas_adapter_pool_destroy(marlaas_pool_t* pool);
+
+/* Commit adapter version `version` of tenant `tenant_id` into the pool ("Commit updated parameters to M",
+ * Algorithm 1; Asynchronous Execution, training step).  A: bf16 [d_in][rank], B: bf16 [rank][d_out],
+ * both row-major device memory, copied and re-laid-out in stream order (the caller may reuse them once the
+ * stream has passed the call).  The layer uses s = alpha / rank formed in fp32.  A tenant that is already
+ * registered keeps its slot and is overwritten in stream order; a new tenant takes the lowest free slot.
+ * rank = 0 (A, B may be NULL) makes the slot behave as "no adapter".  *slot_out (HOST) receives the slot. */
+marlaas_status_t marlaas_adapter_pool_register(marlaas_pool_t* pool, uint64_t tenant_id, uint64_t version,
+                                               int32_t rank, float alpha, const void* A, const void* B,
+                                               int32_t* slot_out, void* cuda_stream);
+/* Free the tenant's slot (its rank becomes 0 in stream order). */
+marlaas_status_t marlaas_adapter_pool_unregister(marlaas_pool_t* pool, uint64_t tenant_id, void* cuda_stream);
+/* Host-side lookup: slot / rank / scale / version of a tenant (any out pointer may be NULL). */
+marlaas_status_t marlaas_adapter_pool_lookup(const marlaas_pool_t* pool, uint64_t tenant_id, int32_t* slot_out,
+                                             int32_t* rank_out, float* scale_out, uint64_t* version_out);
+/* Copy a slot's adapter back out in the caller's layout (A_out bf16 [d_in][rank], B_out bf16 [rank][d_out],
+ * device memory; either may be NULL).  Used to check the store's re-layout bit for bit. */
+marlaas_status_t marlaas_adapter_pool_export(marlaas_pool_t* pool, int32_t slot, void* A_out, void* B_out,
+                                             void* cuda_stream);
+/* Row stride (in floats) of the h_save / h_saved arrays: max_rank rounded up to a multiple of 16. */
+int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool);
+
+/* ---- the layer ---- */
+
+/* Bytes of workspace forward/backward need for a batch of T tokens on this pool (device memory, 256-byte
+ * aligned, contents need not be preserved between calls; two calls in flight need two workspaces). */
+size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
+
+/* Forward: y[T][d_out] = x[T][d_in] W + s_t (x A_t) B_t with t from the segment table.
+ * x (ldx >= d_in), W (ldw >= d_out), y (ldy >= d_out): bf16 row-major.  h_save: optional fp32
+ * [T][rank_stride] that receives h_i = x_i A_t (zero beyond r_t) for reuse by backward; NULL = not kept.
+ * T = 0 is a no-op. */
+marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx,
+                                      const void* W, int64_t ldw, void* y, int64_t ldy,
+                                      const marlaas_segments_t* seg, float* h_save, void* workspace,
+                                      size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/* Backward for the policy-training stage: dx[T][d_in] bf16 (NULL = skip) and per-slot fp32 adapter gradients.
+ * dA_slots / dB_slots: HOST arrays of `capacity` device pointers (either table, or any entry, may be NULL =
+ * skip); dA_t is [d_in][r_t], dB_t is [r_t][d_out], row-major, at the slot's true rank.  Without
+ * MARLAAS_FLAG_ACCUMULATE every non-NULL slot is overwritten (tenants with no token in the batch get exact
+ * zeros); with it the batch's contribution is added.  The sums over a tenant's tokens run over all of its
+ * segments.  h_saved: what forward wrote to h_save for the same batch and adapters, or NULL = recompute. */
+marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx,
+                                       const void* W, int64_t ldw, const void* dy, int64_t lddy,
+                                       void* dx, int64_t lddx, float* const* dA_slots, float* const* dB_slots,
+                                       const marlaas_segments_t* seg, const float* h_saved, void* workspace,
+                                       size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/* The indexing contract, bit-exact: tok_slot[T] (slot of the segment containing each token),
+ * slot_count[capacity+1] (tokens per slot; the last entry counts slot -1), slot_offset[capacity+2]
+ * (exclusive prefix sum in the order 0..capacity-1, then -1; last entry = T) and perm[T] (token indices
+ * stably sorted by that key).  All four are device int32 arrays; any may be NULL. */
+marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const marlaas_segments_t* seg,
+                                          int32_t* tok_slot, int32_t* slot_count, int32_t* slot_offset,
+                                          int32_t* perm, void* workspace, size_t workspace_bytes,
+                                          uint32_t flags, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, read and clear the pool's device status word: MARLAAS_OK, or the first
+ * device-side finding since the last check (BAD_SEGMENT_TABLE, DEVICE_BAD_INDEX, DEVICE_TIMEOUT). */
+marlaas_status_t marlaas_check_status(marlaas_pool_t* pool, void* cuda_stream);
+
+/* Message for the last non-OK status returned on the calling thread ("" if none). */
+const char* marlaas_last_error(void);
+
+/* Number of kernels the library has launched in this process (all pools, all threads). */
+uint64_t marlaas_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARLAAS_H_ */

@@ -1,0 +1,287 @@
+"""Python binding of the C-ABI library: same names as include/marlaas.h, argument marshalling only.
+
+Every step of the layer runs in the library's CUDA kernels; torch is used here for device memory
+(tensors own the buffers) and for the current stream.  There is no CPU fallback: if the library is
+missing or the device is not a B200-class (sm_100) GPU, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmarlaas.so")
+
+MARLAAS_OK = 0
+MARLAAS_ERR_INVALID_ARG = -1
+MARLAAS_ERR_BAD_SEGMENT_TABLE = -2
+MARLAAS_ERR_UNKNOWN_TENANT = -3
+MARLAAS_ERR_RANK_TOO_LARGE = -4
+MARLAAS_ERR_POOL_FULL = -5
+MARLAAS_ERR_UNSUPPORTED_DEVICE = -6
+MARLAAS_ERR_CUDA = -7
+MARLAAS_ERR_DEVICE_TIMEOUT = -8
+MARLAAS_ERR_DEVICE_BAD_INDEX = -9
+MARLAAS_ERR_WORKSPACE_TOO_SMALL = -10
+
+MARLAAS_FLAG_ACCUMULATE = 1
+MARLAAS_FLAG_HOST_TABLE = 2
+MARLAAS_FLAG_VALIDATE_SYNC = 4
+MARLAAS_FLAG_CUDA_CORE_PATH = 8
+
+EXPORTED_SYMBOLS = [
+    "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",
+    "marlaas_adapter_pool_register", "marlaas_adapter_pool_unregister", "marlaas_adapter_pool_lookup",
+    "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
+    "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
+    "marlaas_last_error", "marlaas_kernel_launch_count",
+]
+
+
+class MarlaasError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"marlaas status {status}: {message}")
+        self.status = status
+
+
+class marlaas_segments_t(ctypes.Structure):
+    _fields_ = [("num_segments", ctypes.c_int32), ("seg_offsets", ctypes.c_void_p), ("seg_slot", ctypes.c_void_p)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen the in-tree libmarlaas.so (built by paper_2605_08527_b200/build.py); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise MarlaasError(MARLAAS_ERR_CUDA, f"{LIB_PATH} is not built; run `python -m paper_2605_08527_b200.build` "
+                           "(needs nvcc); there is no fallback path")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u32, u64, f32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32,
+                                       ctypes.c_uint64, ctypes.c_float, ctypes.c_size_t)
+    P = ctypes.POINTER
+    L.marlaas_adapter_pool_storage_bytes.restype = sz
+    L.marlaas_adapter_pool_storage_bytes.argtypes = [i64, i64, i32, i32]
+    L.marlaas_adapter_pool_create.restype = i32
+    L.marlaas_adapter_pool_create.argtypes = [P(vp), ctypes.c_int, i64, i64, i32, i32, vp, sz, vp]
+    L.marlaas_adapter_pool_destroy.restype = i32
+    L.marlaas_adapter_pool_destroy.argtypes = [vp]
+    L.marlaas_adapter_pool_register.restype = i32
+    L.marlaas_adapter_pool_register.argtypes = [vp, u64, u64, i32, f32, vp, vp, P(i32), vp]
+    L.marlaas_adapter_pool_unregister.restype = i32
+    L.marlaas_adapter_pool_unregister.argtypes = [vp, u64, vp]
+    L.marlaas_adapter_pool_lookup.restype = i32
+    L.marlaas_adapter_pool_lookup.argtypes = [vp, u64, P(i32), P(i32), P(f32), P(u64)]
+    L.marlaas_adapter_pool_export.restype = i32
+    L.marlaas_adapter_pool_export.argtypes = [vp, i32, vp, vp, vp]
+    L.marlaas_adapter_pool_rank_stride.restype = i32
+    L.marlaas_adapter_pool_rank_stride.argtypes = [vp]
+    L.marlaas_lora_workspace_bytes.restype = sz
+    L.marlaas_lora_workspace_bytes.argtypes = [vp, i64]
+    L.marlaas_lora_forward.restype = i32
+    L.marlaas_lora_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, P(marlaas_segments_t), vp, vp, sz, u32, vp]
+    L.marlaas_lora_backward.restype = i32
+    L.marlaas_lora_backward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, vp,
+                                        P(marlaas_segments_t), vp, vp, sz, u32, vp]
+    L.marlaas_lora_build_index.restype = i32
+    L.marlaas_lora_build_index.argtypes = [vp, i64, P(marlaas_segments_t), vp, vp, vp, vp, vp, sz, u32, vp]
+    L.marlaas_check_status.restype = i32
+    L.marlaas_check_status.argtypes = [vp, vp]
+    L.marlaas_last_error.restype = ctypes.c_char_p
+    L.marlaas_last_error.argtypes = []
+    L.marlaas_kernel_launch_count.restype = u64
+    L.marlaas_kernel_launch_count.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(rc: int) -> None:
+    if rc != MARLAAS_OK:
+        raise MarlaasError(rc, load_library().marlaas_last_error().decode())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _dptr(t: Optional[torch.Tensor]) -> ctypes.c_void_p:
+    return ctypes.c_void_p(None if t is None else t.data_ptr())
+
+
+def marlaas_last_error() -> str:
+    return load_library().marlaas_last_error().decode()
+
+
+def marlaas_kernel_launch_count() -> int:
+    return int(load_library().marlaas_kernel_launch_count())
+
+
+class Segments:
+    """The token-to-adapter segment table of one mixed batch (int32 tensors, on the device or -- with
+    MARLAAS_FLAG_HOST_TABLE -- on the host)."""
+
+    def __init__(self, seg_offsets: torch.Tensor, seg_slot: torch.Tensor):
+        assert seg_offsets.dtype == torch.int32 and seg_slot.dtype == torch.int32
+        assert seg_offsets.is_contiguous() and seg_slot.is_contiguous()
+        assert seg_offsets.numel() == seg_slot.numel() + 1
+        assert seg_offsets.device == seg_slot.device
+        self.seg_offsets, self.seg_slot = seg_offsets, seg_slot
+        self.on_host = seg_offsets.device.type == "cpu"
+        self.c = marlaas_segments_t(seg_slot.numel(), seg_offsets.data_ptr(), seg_slot.data_ptr())
+
+    @property
+    def flags(self) -> int:
+        return MARLAAS_FLAG_HOST_TABLE if self.on_host else 0
+
+
+class AdapterPool:
+    """marlaas_pool_t plus the torch tensor that owns its device storage."""
+
+    def __init__(self, d_in: int, d_out: int, max_rank: int, capacity: int, device="cuda:0", stream=None):
+        L = load_library()
+        self.device = torch.device(device)
+        if self.device.type != "cuda":
+            raise MarlaasError(MARLAAS_ERR_UNSUPPORTED_DEVICE, "the layer runs on a CUDA device only")
+        idx = self.device.index if self.device.index is not None else torch.cuda.current_device()
+        self.d_in, self.d_out, self.max_rank, self.capacity = d_in, d_out, max_rank, capacity
+        nbytes = L.marlaas_adapter_pool_storage_bytes(d_in, d_out, max_rank, capacity)
+        if nbytes == 0:
+            raise MarlaasError(MARLAAS_ERR_INVALID_ARG, "invalid pool dimensions")
+        with torch.cuda.device(idx):
+            self.storage = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            h = ctypes.c_void_p()
+            _check(L.marlaas_adapter_pool_create(ctypes.byref(h), idx, d_in, d_out, max_rank, capacity,
+                                                 _dptr(self.storage), nbytes, _stream(stream)))
+        self.handle = h
+        self.rank_stride = int(L.marlaas_adapter_pool_rank_stride(h))
+        self._workspaces = {}
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load_library().marlaas_adapter_pool_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace(self, T: int) -> torch.Tensor:
+        """A cached workspace tensor large enough for T tokens (one per pool; not for overlapping calls)."""
+        need = marlaas_lora_workspace_bytes(self, T)
+        ws = self._workspaces.get("ws")
+        if ws is None or ws.numel() < need:
+            ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+            self._workspaces["ws"] = ws
+        return ws
+
+
+def marlaas_adapter_pool_register(pool: AdapterPool, tenant_id: int, version: int, rank: int, alpha: float,
+                                  A: Optional[torch.Tensor], B: Optional[torch.Tensor], stream=None) -> int:
+    if rank > 0:
+        assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.is_contiguous() and B.is_contiguous()
+        assert tuple(A.shape) == (pool.d_in, rank) and tuple(B.shape) == (rank, pool.d_out)
+        assert A.device == pool.device and B.device == pool.device
+    slot = ctypes.c_int32(-1)
+    _check(load_library().marlaas_adapter_pool_register(pool.handle, tenant_id, version, rank, alpha, _dptr(A), _dptr(B),
+                                                        ctypes.byref(slot), _stream(stream)))
+    return int(slot.value)
+
+
+def marlaas_adapter_pool_unregister(pool: AdapterPool, tenant_id: int, stream=None) -> None:
+    _check(load_library().marlaas_adapter_pool_unregister(pool.handle, tenant_id, _stream(stream)))
+
+
+def marlaas_adapter_pool_lookup(pool: AdapterPool, tenant_id: int):
+    s, r, sc, v = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_float(), ctypes.c_uint64()
+    _check(load_library().marlaas_adapter_pool_lookup(pool.handle, tenant_id, ctypes.byref(s), ctypes.byref(r),
+                                                      ctypes.byref(sc), ctypes.byref(v)))
+    return int(s.value), int(r.value), float(sc.value), int(v.value)
+
+
+def marlaas_adapter_pool_export(pool: AdapterPool, slot: int, rank: int, stream=None):
+    A = torch.empty((pool.d_in, rank), dtype=torch.bfloat16, device=pool.device)
+    B = torch.empty((rank, pool.d_out), dtype=torch.bfloat16, device=pool.device)
+    _check(load_library().marlaas_adapter_pool_export(pool.handle, slot, _dptr(A), _dptr(B), _stream(stream)))
+    return A, B
+
+
+def marlaas_lora_workspace_bytes(pool: AdapterPool, T: int) -> int:
+    return int(load_library().marlaas_lora_workspace_bytes(pool.handle, T))
+
+
+def _mat(t: torch.Tensor, cols: int, name: str):
+    assert t.dtype == torch.bfloat16 and t.dim() == 2 and t.shape[1] == cols and t.stride(1) == 1, name
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), cols)
+
+
+def marlaas_lora_forward(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, seg: Segments,
+                         y: Optional[torch.Tensor] = None, h_save: Optional[torch.Tensor] = None,
+                         workspace: Optional[torch.Tensor] = None, flags: int = 0, stream=None) -> torch.Tensor:
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, pool.d_out), dtype=torch.bfloat16, device=x.device)
+    ws = workspace if workspace is not None else pool.workspace(T)
+    ldx, ldw, ldy = _mat(x, pool.d_in, "x"), _mat(W, pool.d_out, "W"), _mat(y, pool.d_out, "y")
+    assert W.shape[0] == pool.d_in
+    if h_save is not None:
+        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and tuple(h_save.shape) == (T, pool.rank_stride)
+    _check(load_library().marlaas_lora_forward(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(y), ldy,
+                                               ctypes.byref(seg.c), _dptr(h_save), _dptr(ws), ws.numel(),
+                                               flags | seg.flags, _stream(stream)))
+    return y
+
+
+def _ptr_table(ts: Optional[Sequence[Optional[torch.Tensor]]], cap: int):
+    if ts is None:
+        return None
+    tab = (ctypes.c_void_p * cap)()
+    for i in range(cap):
+        t = ts[i] if i < len(ts) else None
+        if t is not None:
+            assert t.dtype == torch.float32 and t.is_contiguous()
+            tab[i] = t.data_ptr()
+    return tab
+
+
+def marlaas_lora_backward(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, dy: torch.Tensor, seg: Segments,
+                          dx: Optional[torch.Tensor] = None, dA: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                          dB: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                          h_saved: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                          flags: int = 0, stream=None) -> None:
+    T = dy.shape[0]
+    ws = workspace if workspace is not None else pool.workspace(T)
+    ldx = _mat(x, pool.d_in, "x") if x is not None else 0
+    ldw, lddy = _mat(W, pool.d_out, "W"), _mat(dy, pool.d_out, "dy")
+    lddx = _mat(dx, pool.d_in, "dx") if dx is not None else 0
+    ta, tb = _ptr_table(dA, pool.capacity), _ptr_table(dB, pool.capacity)
+    _check(load_library().marlaas_lora_backward(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(dy), lddy,
+                                                _dptr(dx), lddx, ta, tb, ctypes.byref(seg.c), _dptr(h_saved),
+                                                _dptr(ws), ws.numel(), flags | seg.flags, _stream(stream)))
+
+
+def marlaas_lora_build_index(pool: AdapterPool, T: int, seg: Segments, workspace: Optional[torch.Tensor] = None,
+                             flags: int = 0, stream=None):
+    dev = pool.device
+    tok_slot = torch.empty(max(T, 1), dtype=torch.int32, device=dev)
+    slot_count = torch.empty(pool.capacity + 1, dtype=torch.int32, device=dev)
+    slot_offset = torch.empty(pool.capacity + 2, dtype=torch.int32, device=dev)
+    perm = torch.empty(max(T, 1), dtype=torch.int32, device=dev)
+    ws = workspace if workspace is not None else pool.workspace(T)
+    _check(load_library().marlaas_lora_build_index(pool.handle, T, ctypes.byref(seg.c), _dptr(tok_slot),
+                                                   _dptr(slot_count), _dptr(slot_offset), _dptr(perm), _dptr(ws),
+                                                   ws.numel(), flags | seg.flags, _stream(stream)))
+    return tok_slot[:T], slot_count, slot_offset, perm[:T]
+
+
+def marlaas_check_status(pool: AdapterPool, stream=None) -> None:
+    _check(load_library().marlaas_check_status(pool.handle, _stream(stream)))

@@ -1,0 +1,215 @@
+// The exported layer calls: argument validation on the host, then the kernel sequence on the caller's stream.
+#include <string.h>
+
+#include "internal.cuh"
+
+namespace marlaas {
+
+Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
+    Workspace w;
+    char* p = (char*)base;
+    size_t o = 0;
+    const size_t Tn = (size_t)(T > 0 ? T : 1);
+    auto take = [&](size_t bytes) { char* q = p ? p + o : nullptr; o += align_up(bytes, 256); return q; };
+    w.tok_slot = (int32_t*)take(sizeof(int32_t) * Tn);
+    w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
+    w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
+    w.slot_offset = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 2));
+    w.h = (float*)take(sizeof(float) * Tn * pool->RP);
+    w.g = (float*)take(sizeof(float) * Tn * pool->RP);
+    w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
+    w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
+    w.total = o;
+    return w;
+}
+
+static bool aligned16(const void* p) { return (((uintptr_t)p) & 15) == 0; }
+
+static marlaas_status_t check_matrix(const char* fn, const char* name, const void* p, int64_t ld, int64_t cols) {
+    if (!p) return fail(MARLAAS_ERR_INVALID_ARG, "%s: %s is NULL", fn, name);
+    if (!aligned16(p)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: %s is not 16-byte aligned", fn, name);
+    if (ld < cols || (ld % 8) != 0)
+        return fail(MARLAAS_ERR_INVALID_ARG, "%s: leading dimension of %s (%lld) must be >= %lld and a multiple of 8",
+                    fn, name, (long long)ld, (long long)cols);
+    return MARLAAS_OK;
+}
+
+// Validates the table argument; for host tables also validates the contents and expands them into
+// host_tok_slot (so that nothing is launched for a malformed table).
+static marlaas_status_t check_segments(const char* fn, const marlaas_pool* pool, int64_t T,
+                                       const marlaas_segments_t* seg, uint32_t flags,
+                                       std::vector<int32_t>* host_tok_slot) {
+    if (!seg) return fail(MARLAAS_ERR_INVALID_ARG, "%s: segment table is NULL", fn);
+    if (seg->num_segments < 0) return fail(MARLAAS_ERR_INVALID_ARG, "%s: negative segment count", fn);
+    if (T > 0 && (seg->num_segments == 0 || !seg->seg_offsets || !seg->seg_slot))
+        return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: empty segment table for %lld tokens", fn, (long long)T);
+    if (!(flags & MARLAAS_FLAG_HOST_TABLE)) return MARLAAS_OK;
+    const int32_t S = seg->num_segments;
+    if (S > 0 && (!seg->seg_offsets || !seg->seg_slot))
+        return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: segment arrays are NULL", fn);
+    if (S > 0 && seg->seg_offsets[0] != 0)
+        return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: seg_offsets[0] = %d, expected 0", fn, seg->seg_offsets[0]);
+    if (S > 0 && seg->seg_offsets[S] != T)
+        return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: seg_offsets[S] = %d, expected T = %lld", fn,
+                    seg->seg_offsets[S], (long long)T);
+    host_tok_slot->assign((size_t)T, -1);
+    for (int32_t s = 0; s < S; ++s) {
+        const int32_t a = seg->seg_offsets[s], b = seg->seg_offsets[s + 1];
+        if (b < a) return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: seg_offsets decreases at segment %d", fn, s);
+        const int32_t t = seg->seg_slot[s];
+        if (t < -1 || t >= pool->cap)
+            return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "%s: segment %d names slot %d outside [-1,%d)", fn, s, t,
+                        pool->cap);
+        if (t >= 0 && !pool->slots[t].used)
+            return fail(MARLAAS_ERR_UNKNOWN_TENANT, "%s: segment %d names slot %d, which holds no adapter", fn, s, t);
+        for (int32_t i = a; i < b; ++i) (*host_tok_slot)[i] = t;
+    }
+    return MARLAAS_OK;
+}
+
+static marlaas_status_t make_tok_slot(const marlaas_pool* pool, int64_t T, const marlaas_segments_t* seg,
+                                      uint32_t flags, const std::vector<int32_t>& host_tok_slot, int32_t* tok_slot,
+                                      cudaStream_t st) {
+    if (T <= 0) return MARLAAS_OK;
+    if (flags & MARLAAS_FLAG_HOST_TABLE) {
+        // pageable source: the runtime stages it before returning, so the vector may die after this call
+        MARLAAS_CUDA_TRY(cudaMemcpyAsync(tok_slot, host_tok_slot.data(), sizeof(int32_t) * (size_t)T,
+                                         cudaMemcpyHostToDevice, st));
+        return MARLAAS_OK;
+    }
+    return launch_tok_slot(pool, T, seg->num_segments, seg->seg_offsets, seg->seg_slot, tok_slot, st);
+}
+
+static marlaas_status_t finish(marlaas_pool* pool, uint32_t flags, cudaStream_t st) {
+    if (flags & MARLAAS_FLAG_VALIDATE_SYNC) return marlaas_check_status(pool, (void*)st);
+    return MARLAAS_OK;
+}
+
+}  // namespace marlaas
+
+using namespace marlaas;
+
+extern "C" {
+
+size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T) {
+    if (!pool || T < 0) return 0;
+    return carve_workspace(pool, T, nullptr).total;
+}
+
+marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const marlaas_segments_t* seg,
+                                          int32_t* tok_slot, int32_t* slot_count, int32_t* slot_offset,
+                                          int32_t* perm, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                          void* cuda_stream) {
+    const char* fn = "lora_build_index";
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
+    if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
+    std::vector<int32_t> host_ts;
+    marlaas_status_t rc = check_segments(fn, pool, T, seg, flags, &host_ts);
+    if (rc != MARLAAS_OK) return rc;
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
+    const Workspace ws = carve_workspace(pool, T, workspace);
+    if (workspace_bytes < ws.total)
+        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    int32_t* ts = tok_slot ? tok_slot : ws.tok_slot;
+    rc = make_tok_slot(pool, T, seg, flags, host_ts, ts, st);
+    if (rc != MARLAAS_OK) return rc;
+    if (slot_count || slot_offset || perm) {
+        rc = launch_slot_sort(pool, T, ts, slot_count, slot_offset, perm, st);
+        if (rc != MARLAAS_OK) return rc;
+    }
+    return finish(pool, flags, st);
+}
+
+marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
+                                      int64_t ldw, void* y, int64_t ldy, const marlaas_segments_t* seg,
+                                      float* h_save, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                      void* cuda_stream) {
+    const char* fn = "lora_forward";
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
+    if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
+    if (T == 0) return MARLAAS_OK;
+    marlaas_status_t rc;
+    if ((rc = check_matrix(fn, "x", x, ldx, pool->K)) != MARLAAS_OK) return rc;
+    if ((rc = check_matrix(fn, "W", W, ldw, pool->N)) != MARLAAS_OK) return rc;
+    if ((rc = check_matrix(fn, "y", y, ldy, pool->N)) != MARLAAS_OK) return rc;
+    if (h_save && !aligned16(h_save)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: h_save is not 16-byte aligned", fn);
+    std::vector<int32_t> host_ts;
+    if ((rc = check_segments(fn, pool, T, seg, flags, &host_ts)) != MARLAAS_OK) return rc;
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
+    const Workspace ws = carve_workspace(pool, T, workspace);
+    if (workspace_bytes < ws.total)
+        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+
+    if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    float* h = h_save ? h_save : ws.h;
+    if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, h, st)) != MARLAAS_OK) return rc;
+    if ((rc = launch_gemm_cuda_core(pool, T, pool->N, pool->K, (const bf16*)x, ldx, (const bf16*)W, ldw, false,
+                                    (bf16*)y, ldy, h, pool->d_Bs, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    return finish(pool, flags, st);
+}
+
+marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
+                                       int64_t ldw, const void* dy, int64_t lddy, void* dx, int64_t lddx,
+                                       float* const* dA_slots, float* const* dB_slots,
+                                       const marlaas_segments_t* seg, const float* h_saved, void* workspace,
+                                       size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
+    const char* fn = "lora_backward";
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
+    if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
+    marlaas_status_t rc;
+    const bool want_dA = dA_slots != nullptr, want_dB = dB_slots != nullptr;
+    if (T > 0) {
+        if ((rc = check_matrix(fn, "W", W, ldw, pool->N)) != MARLAAS_OK) return rc;
+        if ((rc = check_matrix(fn, "dy", dy, lddy, pool->N)) != MARLAAS_OK) return rc;
+        if (dx && (rc = check_matrix(fn, "dx", dx, lddx, pool->K)) != MARLAAS_OK) return rc;
+        if ((want_dA || (want_dB && !h_saved)) && (rc = check_matrix(fn, "x", x, ldx, pool->K)) != MARLAAS_OK) return rc;
+    }
+    if (h_saved && !aligned16(h_saved)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: h_saved is not 16-byte aligned", fn);
+    for (int s = 0; s < pool->cap; ++s) {
+        if (want_dA && dA_slots[s] && ((uintptr_t)dA_slots[s] & 3)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: dA_slots[%d] misaligned", fn, s);
+        if (want_dB && dB_slots[s] && ((uintptr_t)dB_slots[s] & 3)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: dB_slots[%d] misaligned", fn, s);
+    }
+    std::vector<int32_t> host_ts;
+    if ((rc = check_segments(fn, pool, T, seg, flags, &host_ts)) != MARLAAS_OK) return rc;
+    if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
+    const Workspace ws = carve_workspace(pool, T, workspace);
+    if (workspace_bytes < ws.total)
+        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    const bool acc = (flags & MARLAAS_FLAG_ACCUMULATE) != 0;
+
+    if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    if (T > 0 && (dx || want_dA)) {
+        if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
+    }
+    if (T > 0 && dx) {
+        if ((rc = launch_gemm_cuda_core(pool, T, pool->K, pool->N, (const bf16*)dy, lddy, (const bf16*)W, ldw, true,
+                                        (bf16*)dx, lddx, ws.g, pool->d_At, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    }
+    if (want_dA || want_dB) {
+        if ((rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st)) != MARLAAS_OK) return rc;
+        if (want_dB) {
+            const float* h = h_saved;
+            if (!h && T > 0) {
+                if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, ws.h, st)) != MARLAAS_OK) return rc;
+                h = ws.h;
+            }
+            MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if ((rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
+                                         false, acc, st)) != MARLAAS_OK) return rc;
+        }
+        if (want_dA) {
+            MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if ((rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
+                                         true, acc, st)) != MARLAAS_OK) return rc;
+        }
+    }
+    return finish(pool, flags, st);
+}
+
+}  // extern "C"

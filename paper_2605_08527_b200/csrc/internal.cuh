@@ -1,0 +1,117 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <string>
+#include <vector>
+
+#include "marlaas.h"
+
+namespace marlaas {
+
+typedef __nv_bfloat16 bf16;
+
+// ---- error plumbing -------------------------------------------------------------------------------
+marlaas_status_t fail(marlaas_status_t code, const char* fmt, ...);
+void count_launch(int n = 1);
+
+#define MARLAAS_CUDA_TRY(expr)                                                                       \
+    do {                                                                                             \
+        cudaError_t e__ = (expr);                                                                    \
+        if (e__ != cudaSuccess)                                                                      \
+            return ::marlaas::fail(MARLAAS_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+#define MARLAAS_LAUNCH_CHECK(name)                                                                   \
+    do {                                                                                             \
+        cudaError_t e__ = cudaGetLastError();                                                        \
+        if (e__ != cudaSuccess)                                                                      \
+            return ::marlaas::fail(MARLAAS_ERR_CUDA, "launch of %s failed: %s", name, cudaGetErrorString(e__)); \
+        ::marlaas::count_launch();                                                                   \
+    } while (0)
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// device status word values (written with atomicCAS from 0, so the first finding wins)
+enum { DEV_OK = 0, DEV_BAD_TABLE = 1, DEV_BAD_INDEX = 2, DEV_TIMEOUT = 3 };
+
+struct SlotMeta {
+    bool used = false;
+    uint64_t tenant_id = 0;
+    uint64_t version = 0;
+    int32_t rank = 0;
+    float alpha = 0.f;
+    float scale = 0.f;
+};
+
+}  // namespace marlaas
+
+// The pool: host bookkeeping plus pointers into the caller-provided device storage.
+//   At : bf16 [capacity*RP][K]   row (slot*RP + j) = column j of A_t   (zero rows for j >= r_t)
+//   Bs : bf16 [capacity*RP][N]   row (slot*RP + j) = row j of B_t      (zero rows for j >= r_t)
+// Both serve as gather sources for the shrink (dot products along a contiguous row) and as tensor-core
+// operands for the extra k-steps of the fused expand (rows = rank index).
+struct marlaas_pool {
+    int device = 0;
+    int64_t K = 0, N = 0;
+    int32_t max_rank = 0, RP = 0, cap = 0;
+    char* storage = nullptr;
+    size_t storage_bytes = 0;
+    int32_t* d_status = nullptr;
+    int32_t* d_rank = nullptr;
+    float* d_scale = nullptr;
+    marlaas::bf16* d_At = nullptr;
+    marlaas::bf16* d_Bs = nullptr;
+    std::vector<marlaas::SlotMeta> slots;
+    int sm_count = 0;
+};
+
+namespace marlaas {
+
+struct StorageLayout {
+    size_t off_status, off_rank, off_scale, off_At, off_Bs, total;
+};
+StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap);
+
+// Per-call workspace (device), carved from the caller's buffer.
+struct Workspace {
+    int32_t* tok_slot;     // [T]
+    int32_t* perm;         // [T]
+    int32_t* slot_count;   // [cap+1]
+    int32_t* slot_offset;  // [cap+2]
+    float* h;              // [T][RP]
+    float* g;              // [T][RP]
+    float** dA_ptrs;       // [cap]
+    float** dB_ptrs;       // [cap]
+    size_t total;
+};
+Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base);
+
+// ---- kernels launched by api.cu ---------------------------------------------------------------------
+// plan.cu
+marlaas_status_t launch_tok_slot(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
+                                 const int32_t* seg_slot, int32_t* tok_slot, cudaStream_t st);
+marlaas_status_t launch_slot_sort(const marlaas_pool* pool, int64_t T, const int32_t* tok_slot,
+                                  int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st);
+
+// cuda_core_kernels.cu
+// out[i][j] = sum_d src[i][d] * store[(slot_i*RP + j)][d] for j < RP (zeros for inactive tokens / padded rows)
+marlaas_status_t launch_rowdot(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                               const bf16* store, const int32_t* tok_slot, float* out, cudaStream_t st);
+// C[T][Nout] = bf16( A[T][Kc] * op(W) + s_t * sum_j hg[i][j] * store[(slot*RP+j)][c] );
+// trans_w = false: op(W) = W[Kc][Nout] (ldw);  true: op(W) = W^T with W stored [Nout][Kc] (ldw)
+marlaas_status_t launch_gemm_cuda_core(const marlaas_pool* pool, int64_t T, int64_t Nout, int64_t Kc,
+                                       const bf16* A, int64_t lda, const bf16* W, int64_t ldw, bool trans_w,
+                                       bf16* C, int64_t ldc, const float* hg, const bf16* store,
+                                       const int32_t* tok_slot, cudaStream_t st);
+// out_t[j][c] (transpose_out = false, ld = C) or out_t[c][j] (true, ld = r_t) (+)= s_t * sum_{i in t} hg[i][j] * src[i][c]
+marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const bf16* src, int64_t ld,
+                                    const float* hg, const int32_t* perm, const int32_t* slot_offset,
+                                    float* const* out_ptrs, bool transpose_out, bool accumulate, cudaStream_t st);
+
+}  // namespace marlaas

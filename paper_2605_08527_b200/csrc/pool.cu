@@ -1,0 +1,254 @@
+// Pooled adapter store: one slot per tenant, holding the tenant's current policy version
+// (paper: Methods, "Multi-Task Manager": per-task LoRA parameters theta_t^(v) and version counter;
+// Algorithm 1: "Commit updated parameters to M").
+#include <stdarg.h>
+#include <stdio.h>
+
+#include <new>
+
+#include "internal.cuh"
+
+namespace marlaas {
+
+static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+marlaas_status_t fail(marlaas_status_t code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap) {
+    StorageLayout L;
+    size_t o = 0;
+    L.off_status = o; o += 256;
+    L.off_rank = o;   o += align_up(sizeof(int32_t) * (size_t)cap, 256);
+    L.off_scale = o;  o += align_up(sizeof(float) * (size_t)cap, 256);
+    L.off_At = o;     o += align_up(sizeof(bf16) * (size_t)cap * RP * (size_t)K, 256);
+    L.off_Bs = o;     o += align_up(sizeof(bf16) * (size_t)cap * RP * (size_t)N, 256);
+    L.total = o;
+    return L;
+}
+
+static bool pool_args_ok(int64_t K, int64_t N, int32_t max_rank, int32_t cap) {
+    return K > 0 && N > 0 && (K % 8) == 0 && (N % 8) == 0 && max_rank >= 1 && max_rank <= 128 && cap >= 1 &&
+           cap <= 4096 && K < (1ll << 31) && N < (1ll << 31);
+}
+
+// A [K][r] row-major -> At rows (slot*RP + j)[k]; B [r][N] -> Bs rows; rows r..RP-1 cleared.
+__global__ void k_register(const bf16* __restrict__ A, const bf16* __restrict__ B, bf16* __restrict__ At,
+                           bf16* __restrict__ Bs, int32_t* d_rank, float* d_scale, int slot, int r, int RP,
+                           int64_t K, int64_t N, float scale) {
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nth = (int64_t)gridDim.x * blockDim.x;
+    bf16* at = At + (size_t)slot * RP * K;
+    bf16* bs = Bs + (size_t)slot * RP * N;
+    const bf16 zero = __float2bfloat16(0.f);
+    for (int64_t e = tid; e < (int64_t)RP * K; e += nth) {
+        const int64_t j = e / K, k = e - j * K;
+        at[e] = (j < r) ? A[k * r + j] : zero;
+    }
+    for (int64_t e = tid; e < (int64_t)RP * N; e += nth) {
+        const int64_t j = e / N;
+        bs[e] = (j < r) ? B[e] : zero;
+    }
+    if (tid == 0) {
+        d_rank[slot] = r;
+        d_scale[slot] = scale;
+    }
+}
+
+__global__ void k_export(const bf16* __restrict__ At, const bf16* __restrict__ Bs, bf16* A_out, bf16* B_out,
+                         int slot, int r, int RP, int64_t K, int64_t N) {
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nth = (int64_t)gridDim.x * blockDim.x;
+    const bf16* at = At + (size_t)slot * RP * K;
+    const bf16* bs = Bs + (size_t)slot * RP * N;
+    if (A_out)
+        for (int64_t e = tid; e < (int64_t)r * K; e += nth) {
+            const int64_t k = e / r, j = e - k * r;
+            A_out[e] = at[j * K + k];
+        }
+    if (B_out)
+        for (int64_t e = tid; e < (int64_t)r * N; e += nth) B_out[e] = bs[e];
+}
+
+}  // namespace marlaas
+
+using namespace marlaas;
+
+extern "C" {
+
+const char* marlaas_last_error(void) { return g_err; }
+uint64_t marlaas_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t marlaas_adapter_pool_storage_bytes(int64_t d_in, int64_t d_out, int32_t max_rank, int32_t capacity) {
+    if (!pool_args_ok(d_in, d_out, max_rank, capacity)) return 0;
+    return storage_layout(d_in, d_out, (max_rank + 15) / 16 * 16, capacity).total;
+}
+
+marlaas_status_t marlaas_adapter_pool_create(marlaas_pool_t** out, int device, int64_t d_in, int64_t d_out,
+                                             int32_t max_rank, int32_t capacity, void* storage,
+                                             size_t storage_bytes, void* cuda_stream) {
+    if (!out) return fail(MARLAAS_ERR_INVALID_ARG, "pool_create: out is NULL");
+    *out = nullptr;
+    if (!pool_args_ok(d_in, d_out, max_rank, capacity))
+        return fail(MARLAAS_ERR_INVALID_ARG,
+                    "pool_create: need d_in, d_out > 0 and multiples of 8, max_rank in [1,128], capacity in [1,4096]");
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+        cudaGetLastError();
+        return fail(MARLAAS_ERR_UNSUPPORTED_DEVICE, "pool_create: no CUDA device %d", device);
+    }
+    int major = 0, sms = 0;
+    MARLAAS_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+    MARLAAS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    if (major != 10)
+        return fail(MARLAAS_ERR_UNSUPPORTED_DEVICE, "pool_create: device %d is sm_%d0, this library is sm_100a only",
+                    device, major);
+    const int32_t RP = (max_rank + 15) / 16 * 16;
+    const StorageLayout L = storage_layout(d_in, d_out, RP, capacity);
+    if (!storage || ((uintptr_t)storage & 255) != 0)
+        return fail(MARLAAS_ERR_INVALID_ARG, "pool_create: storage must be a 256-byte aligned device pointer");
+    if (storage_bytes < L.total)
+        return fail(MARLAAS_ERR_INVALID_ARG, "pool_create: storage_bytes %zu < required %zu", storage_bytes, L.total);
+    MARLAAS_CUDA_TRY(cudaSetDevice(device));
+    MARLAAS_CUDA_TRY(cudaMemsetAsync(storage, 0, L.total, (cudaStream_t)cuda_stream));
+    marlaas_pool* p = new (std::nothrow) marlaas_pool();
+    if (!p) return fail(MARLAAS_ERR_INVALID_ARG, "pool_create: out of host memory");
+    p->device = device;
+    p->K = d_in;
+    p->N = d_out;
+    p->max_rank = max_rank;
+    p->RP = RP;
+    p->cap = capacity;
+    p->storage = (char*)storage;
+    p->storage_bytes = storage_bytes;
+    p->d_status = (int32_t*)(p->storage + L.off_status);
+    p->d_rank = (int32_t*)(p->storage + L.off_rank);
+    p->d_scale = (float*)(p->storage + L.off_scale);
+    p->d_At = (bf16*)(p->storage + L.off_At);
+    p->d_Bs = (bf16*)(p->storage + L.off_Bs);
+    p->slots.resize((size_t)capacity);
+    p->sm_count = sms;
+    *out = p;
+    return MARLAAS_OK;
+}
+
+marlaas_status_t marlaas_adapter_pool_destroy(marlaas_pool_t* pool) {
+    delete pool;
+    return MARLAAS_OK;
+}
+
+int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool) { return pool ? pool->RP : 0; }
+
+marlaas_status_t marlaas_adapter_pool_register(marlaas_pool_t* pool, uint64_t tenant_id, uint64_t version,
+                                               int32_t rank, float alpha, const void* A, const void* B,
+                                               int32_t* slot_out, void* cuda_stream) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "pool_register: pool is NULL");
+    if (rank < 0) return fail(MARLAAS_ERR_INVALID_ARG, "pool_register: negative rank");
+    if (rank > pool->max_rank)
+        return fail(MARLAAS_ERR_RANK_TOO_LARGE, "pool_register: rank %d > pool max_rank %d", rank, pool->max_rank);
+    if (rank > 0 && (!A || !B)) return fail(MARLAAS_ERR_INVALID_ARG, "pool_register: A or B is NULL");
+    if (rank > 0 && ((((uintptr_t)A) | ((uintptr_t)B)) & 1))
+        return fail(MARLAAS_ERR_INVALID_ARG, "pool_register: A and B must be 2-byte aligned");
+    int slot = -1, free_slot = -1;
+    for (int s = 0; s < pool->cap; ++s) {
+        if (pool->slots[s].used && pool->slots[s].tenant_id == tenant_id) { slot = s; break; }
+        if (!pool->slots[s].used && free_slot < 0) free_slot = s;
+    }
+    if (slot < 0) slot = free_slot;
+    if (slot < 0) return fail(MARLAAS_ERR_POOL_FULL, "pool_register: all %d slots in use", pool->cap);
+    const float scale = rank > 0 ? alpha / (float)rank : 0.f;
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    const int64_t work = (int64_t)pool->RP * (pool->K > pool->N ? pool->K : pool->N);
+    const int blocks = (int)(cdiv(work, 256) < 4 * pool->sm_count ? cdiv(work, 256) : 4 * pool->sm_count);
+    k_register<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>((const bf16*)A, (const bf16*)B, pool->d_At, pool->d_Bs,
+                                                              pool->d_rank, pool->d_scale, slot, rank, pool->RP,
+                                                              pool->K, pool->N, scale);
+    MARLAAS_LAUNCH_CHECK("k_register");
+    SlotMeta& m = pool->slots[slot];
+    m.used = true;
+    m.tenant_id = tenant_id;
+    m.version = version;
+    m.rank = rank;
+    m.alpha = alpha;
+    m.scale = scale;
+    if (slot_out) *slot_out = slot;
+    return MARLAAS_OK;
+}
+
+marlaas_status_t marlaas_adapter_pool_unregister(marlaas_pool_t* pool, uint64_t tenant_id, void* cuda_stream) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "pool_unregister: pool is NULL");
+    for (int s = 0; s < pool->cap; ++s) {
+        if (pool->slots[s].used && pool->slots[s].tenant_id == tenant_id) {
+            MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+            k_register<<<1, 256, 0, (cudaStream_t)cuda_stream>>>(nullptr, nullptr, pool->d_At, pool->d_Bs, pool->d_rank,
+                                                                 pool->d_scale, s, 0, pool->RP, pool->K, pool->N, 0.f);
+            MARLAAS_LAUNCH_CHECK("k_register(unregister)");
+            pool->slots[s] = SlotMeta();
+            return MARLAAS_OK;
+        }
+    }
+    return fail(MARLAAS_ERR_UNKNOWN_TENANT, "pool_unregister: tenant %llu is not registered",
+                (unsigned long long)tenant_id);
+}
+
+marlaas_status_t marlaas_adapter_pool_lookup(const marlaas_pool_t* pool, uint64_t tenant_id, int32_t* slot_out,
+                                             int32_t* rank_out, float* scale_out, uint64_t* version_out) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "pool_lookup: pool is NULL");
+    for (int s = 0; s < pool->cap; ++s) {
+        const SlotMeta& m = pool->slots[s];
+        if (m.used && m.tenant_id == tenant_id) {
+            if (slot_out) *slot_out = s;
+            if (rank_out) *rank_out = m.rank;
+            if (scale_out) *scale_out = m.scale;
+            if (version_out) *version_out = m.version;
+            return MARLAAS_OK;
+        }
+    }
+    return fail(MARLAAS_ERR_UNKNOWN_TENANT, "pool_lookup: tenant %llu is not registered", (unsigned long long)tenant_id);
+}
+
+marlaas_status_t marlaas_adapter_pool_export(marlaas_pool_t* pool, int32_t slot, void* A_out, void* B_out,
+                                             void* cuda_stream) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "pool_export: pool is NULL");
+    if (slot < 0 || slot >= pool->cap || !pool->slots[slot].used)
+        return fail(MARLAAS_ERR_UNKNOWN_TENANT, "pool_export: slot %d is not in use", slot);
+    const int r = pool->slots[slot].rank;
+    if (r == 0 || (!A_out && !B_out)) return MARLAAS_OK;
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    const int64_t work = (int64_t)r * (pool->K > pool->N ? pool->K : pool->N);
+    const int blocks = (int)(cdiv(work, 256) < 4 * pool->sm_count ? cdiv(work, 256) : 4 * pool->sm_count);
+    k_export<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(pool->d_At, pool->d_Bs, (bf16*)A_out, (bf16*)B_out, slot, r,
+                                                            pool->RP, pool->K, pool->N);
+    MARLAAS_LAUNCH_CHECK("k_export");
+    return MARLAAS_OK;
+}
+
+marlaas_status_t marlaas_check_status(marlaas_pool_t* pool, void* cuda_stream) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "check_status: pool is NULL");
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    int32_t w[4] = {0, 0, 0, 0};
+    MARLAAS_CUDA_TRY(cudaMemcpyAsync(w, pool->d_status, sizeof(w), cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream));
+    MARLAAS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    if (w[0] == DEV_OK) return MARLAAS_OK;
+    MARLAAS_CUDA_TRY(cudaMemsetAsync(pool->d_status, 0, 16, (cudaStream_t)cuda_stream));
+    MARLAAS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    switch (w[0]) {
+        case DEV_BAD_TABLE:
+            return fail(MARLAAS_ERR_BAD_SEGMENT_TABLE, "device check: malformed segment table (detail %d)", w[1]);
+        case DEV_BAD_INDEX:
+            return fail(MARLAAS_ERR_DEVICE_BAD_INDEX, "device check: slot outside [-1, capacity) at token %d", w[1]);
+        case DEV_TIMEOUT:
+            return fail(MARLAAS_ERR_DEVICE_TIMEOUT, "device check: a bounded wait ran out (site %d)", w[1]);
+        default:
+            return fail(MARLAAS_ERR_CUDA, "device check: unknown status word %d", w[0]);
+    }
+}
+
+}  // extern "C"

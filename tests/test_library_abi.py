@@ -1,0 +1,61 @@
+"""CPU-side checks of the boundary: the library loads and exports every symbol include/marlaas.h declares,
+and host-side argument validation answers with status codes without needing a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2605_08527_b200 as ml
+from paper_2605_08527_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "marlaas.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(marlaas_[a-z_]+)\s*\(", text)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2605_08527_b200 import build
+    build.build()
+    return B.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert "marlaas_lora_forward" in names and "marlaas_lora_backward" in names
+    assert "marlaas_adapter_pool_register" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in marlaas.h but not exported"
+    assert sorted(B.EXPORTED_SYMBOLS) == names
+
+
+def test_storage_bytes_and_argument_checks(lib):
+    assert lib.marlaas_adapter_pool_storage_bytes(4096, 4096, 16, 32) > 2 * 32 * 16 * 4096 * 2
+    assert lib.marlaas_adapter_pool_storage_bytes(4096, 4097, 16, 32) == 0      # d_out not a multiple of 8
+    assert lib.marlaas_adapter_pool_storage_bytes(4096, 4096, 0, 32) == 0
+    assert lib.marlaas_adapter_pool_storage_bytes(4096, 4096, 129, 32) == 0
+    h = ctypes.c_void_p()
+    rc = lib.marlaas_adapter_pool_create(ctypes.byref(h), 0, 512, 511, 8, 4, None, 0, None)
+    assert rc == B.MARLAAS_ERR_INVALID_ARG and "multiples of 8" in B.marlaas_last_error()
+    rc = lib.marlaas_adapter_pool_create(ctypes.byref(h), 0, 512, 512, 8, 4, None, 0, None)
+    # without a GPU the device check answers; with one, the NULL storage does
+    assert rc in (B.MARLAAS_ERR_UNSUPPORTED_DEVICE, B.MARLAAS_ERR_INVALID_ARG)
+    assert lib.marlaas_lora_forward(None, 1, None, 0, None, 0, None, 0, None, None, None, 0, 0, None) == B.MARLAAS_ERR_INVALID_ARG
+    assert lib.marlaas_lora_backward(None, 1, None, 0, None, 0, None, 0, None, 0, None, None, None, None, None, 0, 0,
+                                     None) == B.MARLAAS_ERR_INVALID_ARG
+    assert lib.marlaas_lora_workspace_bytes(None, 5) == 0
+
+
+def test_product_path_has_no_oracle_or_cpu_fallback():
+    pkg = os.path.join(ROOT, "paper_2605_08527_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in src and "from oracle" not in src, f
+                assert "marlaas_oracle" not in src, f
