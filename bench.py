@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""Benchmark of the multi-tenant LoRA linear layer (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: index build, shrink,
+base GEMM with the fused LoRA expand (forward), then g-shrink, dx GEMM with its fused expand and the dA/dB
+reductions (backward).  The default workload is the training-shaped configuration (base W 4096x11008,
+10 tenants of rank 32, 16384 tokens in lognormal per-tenant segments), the only single-projection
+configuration that exercises every step; --workload cfg2 times the decode-shaped forward, cfg4 the
+heterogeneous one, cfg5 the 7-projection decoder-layer set.
+
+Prints ONE JSON line (rank 0).  `value` is whole-job tokens/s with inputs resident in HBM; `e2e` is the same
+metric through the same calls with HOST inputs and outputs (pinned buffers, copies inside the timed region).
+`--impl reference` times the CPU oracle on the host cores instead (a deliberately plain program).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_08527_b200 import workloads as wl  # noqa: E402
+
+METRIC = "multi-LoRA layer tokens/s (fwd+bwd)"
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
+CFG_OF = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
+CFG_DESC = {
+    "cfg1": "tiny: W 512x512, 4 tenants r=8, 256 tokens, fwd+bwd",
+    "cfg2": "rollout-decode shaped: W 4096x4096, 32 tenants r=16, 256 unsorted decode tokens, fwd only",
+    "cfg3": "training shaped: W 4096x11008, 10 tenants r=32, 16384 tokens in lognormal segments, fwd+bwd",
+    "cfg4": "heterogeneous tenants: W 5120x5120, 32 tenants r in {8,16,32,64}, 8192 Zipf tokens, fwd+bwd",
+    "cfg5": "7B decoder-layer adapter set: 7 projections, 32 tenants r=16, 4096 training + 256 decode tokens",
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return {"bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    "hbm_gbs": float(d["hbm_gbs"])}, "measured"
+        except Exception:
+            pass
+    return {"bf16_tflops": FALLBACK["bf16_tflops"], "bf16_tflops_sustained": 1400.0, "hbm_gbs": FALLBACK["hbm_gbs"]}, "fallback"
+
+
+def algorithmic_work(w):
+    """Flops and minimum bytes of one step (each operand touched once), per projection and summed.
+    fwd: 2TKN + sum_i 2 r(K+N); bwd: 2TKN + sum_i r(4N+4K); rank padding and recomputation are not counted."""
+    ts = w.tok_slot()
+    out = {"fwd_flops": 0.0, "bwd_flops": 0.0, "fwd_bytes": 0.0, "bwd_bytes": 0.0, "gemm_flops": []}
+    for p in w.projections:
+        K, N = p.d_in, p.d_out
+        ranks = np.array([a.rank for a in p.adapters] + [0])
+        r_tok = ranks[ts]
+        Tb = 0 if p.dy_bits is None else p.dy_bits.shape[0]
+        present = np.unique(ts[ts >= 0])
+        ad_bytes = sum(2 * ranks[t] * (K + N) for t in present)
+        out["fwd_flops"] += 2.0 * w.T * K * N + float(np.sum(2.0 * r_tok * (K + N)))
+        out["fwd_bytes"] += 2.0 * (K * N + w.T * K + w.T * N) + ad_bytes
+        out["gemm_flops"].append(2.0 * w.T * K * N + float(np.sum(2.0 * r_tok * N)))
+        if Tb:
+            rb = r_tok[:Tb]
+            pres_b = np.unique(ts[:Tb][ts[:Tb] >= 0])
+            out["bwd_flops"] += 2.0 * Tb * K * N + float(np.sum(rb * (4.0 * N + 4.0 * K)))
+            out["bwd_bytes"] += 2.0 * (K * N + 2 * Tb * K + Tb * N) + sum(2 * ranks[t] * (K + N) for t in pres_b) \
+                + sum(4 * ranks[t] * (K + N) for t in pres_b)
+            out["gemm_flops"].append(2.0 * Tb * K * N + float(np.sum(2.0 * rb * K)))
+    return out
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc, self.path = None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                c = [v.strip() for v in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, c[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(pw)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_step_sample(w, n_tok):
+    """Time the oracle (as it stands) on the first n_tok tokens of every projection; returns seconds."""
+    import oracle
+    ts = w.tok_slot()
+    total = 0.0
+    for p in w.projections:
+        r, s, A, Bm = oracle.adapters_of(p)
+        n = min(n_tok, w.T)
+        x = p.x[:n]
+        t0 = time.perf_counter()
+        oracle.forward(x, p.W, r, s, A, Bm, ts[:n])
+        if p.dy_bits is not None:
+            nb = min(n, p.dy_bits.shape[0])
+            dy = p.dy[:nb]
+            oracle.backward_dx(dy, p.W, r, s, A, Bm, ts[:nb])
+            oracle.backward_dAdB(x[:nb], dy, r, s, A, Bm, ts[:nb])
+        total += time.perf_counter() - t0
+    return total
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the CPU oracle on the host cores, a bounded sample of the workload per step."""
+    if rank != 0:
+        return
+    import oracle
+    w = wl.make_workload(CFG_OF[args.workload])
+    n_tok = min(w.T, args.reference_tokens)
+    for _ in range(args.warmup):
+        oracle_step_sample(w, min(n_tok, 32))
+    times = [oracle_step_sample(w, n_tok) for _ in range(args.steps)]
+    sec = float(np.mean(times))
+    val = n_tok / sec
+    cores = oracle.num_threads()
+    sample = f"first {n_tok} of {w.T} tokens of {args.workload}, all projections, forward" + \
+             ("+backward" if w.T_bwd else "") + " per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32 storage / f64 accumulate", "data": "synthetic",
+        "config": {"workload": args.workload, "desc": CFG_DESC[args.workload], "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg3", choices=sorted(CFG_OF))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--reference-tokens", type=int, default=1024)
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--flags", type=int, default=0, help="extra MARLAAS_FLAG_* bits for every call (diagnostics)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    from paper_2605_08527_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the layer has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = wl.make_workload(CFG_OF[args.workload])
+    work = algorithmic_work(w)
+    ts_np = w.tok_slot()
+
+    def dev_bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+
+    def pinned_bf16(bits):
+        t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+        return t.pin_memory()
+
+    # ---- device-resident state: one pool per projection, adapters registered, inputs uploaded -------------
+    projs = []
+    seg = B.Segments(torch.from_numpy(w.seg_offsets.astype(np.int32)).to(dev), torch.from_numpy(w.seg_slot.astype(np.int32)).to(dev))
+    Tb = w.T_bwd
+    seg_b = seg
+    if 0 < Tb < w.T:
+        keep = [s for s in range(len(w.seg_slot)) if w.seg_offsets[s] < Tb]
+        off = np.array([min(int(w.seg_offsets[s]), Tb) for s in keep] + [Tb], dtype=np.int32)
+        seg_b = B.Segments(torch.from_numpy(off).to(dev), torch.from_numpy(w.seg_slot[keep].astype(np.int32)).to(dev))
+    x_cache = {}
+    for p in w.projections:
+        pool = B.AdapterPool(p.d_in, p.d_out, w.max_rank, w.n_tenants, device=dev)
+        for a in p.adapters:
+            B.marlaas_adapter_pool_register(pool, a.tenant_id, 0, a.rank, a.alpha, dev_bf16(a.A_bits), dev_bf16(a.B_bits))
+        key = p.x_bits.ctypes.data if False else (p.d_in, p.x_bits[0, :8].tobytes())
+        if key not in x_cache:
+            x_cache[key] = (dev_bf16(p.x_bits), pinned_bf16(p.x_bits))
+        x_d, x_h = x_cache[key]
+        st = {"p": p, "pool": pool, "W": dev_bf16(p.W_bits), "x": x_d, "x_host": x_h,
+              "y": torch.empty((w.T, p.d_out), dtype=torch.bfloat16, device=dev),
+              "h": torch.empty((w.T, pool.rank_stride), dtype=torch.float32, device=dev),
+              "ws": torch.empty(B.marlaas_lora_workspace_bytes(pool, w.T), dtype=torch.uint8, device=dev)}
+        if Tb:
+            st["dy"] = dev_bf16(p.dy_bits)
+            st["dy_host"] = pinned_bf16(p.dy_bits)
+            st["dx"] = torch.empty((Tb, p.d_in), dtype=torch.bfloat16, device=dev)
+            st["dA"] = [torch.empty((p.d_in, a.rank), dtype=torch.float32, device=dev) for a in p.adapters]
+            st["dB"] = [torch.empty((a.rank, p.d_out), dtype=torch.float32, device=dev) for a in p.adapters]
+        projs.append(st)
+
+    def step(x_of=lambda s: s["x"], dy_of=lambda s: s["dy"]):
+        for s in projs:
+            B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=args.flags)
+            if Tb:
+                B.marlaas_lora_backward(s["pool"], x_of(s)[:Tb], s["W"], dy_of(s), seg_b, dx=s["dx"], dA=s["dA"], dB=s["dB"],
+                                        h_saved=s["h"][:Tb], workspace=s["ws"], flags=args.flags)
+
+    # L2 hygiene: every step streams operands larger than the 126 MB L2 except on the small configs, where a
+    # flush buffer is written between steps.
+    resident = sum(s["W"].numel() * 2 + s["x"].numel() * 2 for s in projs)
+    l2_note = "inputs larger than L2"
+    flush = None
+    if resident < 3 * 126e6:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        l2_note = "L2 flushed between steps (256 MiB write)"
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    for s in projs:
+        B.marlaas_check_status(s["pool"])
+    barrier()
+
+    # ---- timed region: device-resident inputs ------------------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    n0 = B.marlaas_kernel_launch_count()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for a, b in evs:
+        if flush is not None:
+            flush.fill_(1)
+        a.record()
+        step()
+        b.record()
+    barrier()
+    launches = B.marlaas_kernel_launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = float(sum(step_ms))
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = w.T * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- dominant kernel (base GEMM + fused expand), timed live with events on the launching stream -------
+    for s in projs:
+        B.marlaas_kernel_timing_begin(s["pool"])
+    for _ in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        step()
+    gemm_ms, gemm_n = 0.0, 0
+    for s in projs:
+        ms, n = B.marlaas_kernel_timing_end(s["pool"])
+        gemm_ms += ms
+        gemm_n += n
+    peaks, peak_src = measured_peaks()
+    gemm_flops_per_step = float(sum(work["gemm_flops"]))
+    avg_launch_ms = gemm_ms / max(gemm_n, 1)
+    flops_per_launch = gemm_flops_per_step / max(len(work["gemm_flops"]), 1)
+    step_bytes = work["fwd_bytes"] + work["bwd_bytes"]
+    if args.workload == "cfg2":
+        ach = work["fwd_bytes"] / (ms_per_step * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peak_src}",
+                    "kernel": "whole forward call (index + shrink + GEMM with fused expand)",
+                    "frac_of_nominal_8TBs": ach / NOMINAL["hbm_gbs"]}
+    else:
+        ach = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12 if gemm_n else 0.0
+        roofline = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": f"of {peak_src} (burst)",
+                    "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)",
+                    "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms,
+                    "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
+                    "whole_step_tflops": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12,
+                    "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+
+    # ---- end to end: host inputs -> device -> layer -> host outputs, all inside the timed region ------------
+    e2e = None
+    if args.e2e_steps > 0:
+        host_out = []
+        for s in projs:
+            o = {"y": torch.empty((w.T, s["p"].d_out), dtype=torch.bfloat16).pin_memory()}
+            if Tb:
+                o["dx"] = torch.empty((Tb, s["p"].d_in), dtype=torch.bfloat16).pin_memory()
+                o["dA"] = [torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in s["dA"]]
+                o["dB"] = [torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in s["dB"]]
+            host_out.append(o)
+        seg_off_h = torch.from_numpy(w.seg_offsets.astype(np.int32)).pin_memory()
+        seg_slot_h = torch.from_numpy(w.seg_slot.astype(np.int32)).pin_memory()
+
+        def e2e_step():
+            h2d = d2h = 0
+            seg.seg_offsets.copy_(seg_off_h, non_blocking=True)
+            seg.seg_slot.copy_(seg_slot_h, non_blocking=True)
+            h2d += seg_off_h.numel() * 4 + seg_slot_h.numel() * 4
+            done = set()
+            for s in projs:
+                if id(s["x"]) not in done:
+                    s["x"].copy_(s["x_host"], non_blocking=True)
+                    h2d += s["x"].numel() * 2
+                    done.add(id(s["x"]))
+                if Tb:
+                    s["dy"].copy_(s["dy_host"], non_blocking=True)
+                    h2d += s["dy"].numel() * 2
+            step()
+            for s, o in zip(projs, host_out):
+                o["y"].copy_(s["y"], non_blocking=True)
+                d2h += s["y"].numel() * 2
+                if Tb:
+                    o["dx"].copy_(s["dx"], non_blocking=True)
+                    d2h += s["dx"].numel() * 2
+                    for hbuf, dbuf in zip(o["dA"] + o["dB"], s["dA"] + s["dB"]):
+                        hbuf.copy_(dbuf, non_blocking=True)
+                        d2h += dbuf.numel() * 4
+            return h2d, d2h
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            h2d, d2h = e2e_step()
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": tokens_per_step / (e_ms / args.e2e_steps * 1e-3), "unit": "tokens/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
+               "ms_per_step": e_ms / args.e2e_steps}
+
+    for s in projs:
+        B.marlaas_check_status(s["pool"])
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only) ------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_tok = min(w.T, args.cpu_baseline_tokens)
+        sec = oracle_step_sample(w, n_tok)
+        cpu_baseline = {"value": n_tok / sec, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"first {n_tok} of {w.T} tokens of {args.workload}, all projections, one timed execution "
+                                  f"({sec:.1f} s)"}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC if Tb else "multi-LoRA layer tokens/s (fwd)", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "desc": CFG_DESC[args.workload], "tokens_per_step_per_gpu": w.T,
+                       "backward_tokens": Tb, "segments": int(len(w.seg_slot)), "l2": l2_note,
+                       "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks,
+            "work_per_step": {"fwd_gflop": work["fwd_flops"] / 1e9, "bwd_gflop": work["bwd_flops"] / 1e9,
+                              "fwd_mb": work["fwd_bytes"] / 1e6, "bwd_mb": work["bwd_bytes"] / 1e6},
+            "ms_per_step_min": float(min(step_ms)), "ms_per_step_median": float(np.median(step_ms)),
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -154,6 +154,13 @@ marlaas_status_t marlaas_check_status(marlaas_pool_t* pool, void* cuda_stream);
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char* marlaas_last_error(void);
 
+/* Measurement aid (no counterpart in the paper): between _begin and _end the library brackets every launch of
+ * the layer's dominant kernel (the base GEMM with the fused low-rank term, forward and dx) with CUDA events on
+ * the launching stream.  _end synchronises those events and returns the summed device time in milliseconds
+ * and the number of bracketed launches (either out pointer may be NULL). */
+marlaas_status_t marlaas_kernel_timing_begin(marlaas_pool_t* pool);
+marlaas_status_t marlaas_kernel_timing_end(marlaas_pool_t* pool, float* gemm_ms, int32_t* gemm_launches);
+
 /* Number of kernels the library has launched in this process (all pools, all threads). */
 uint64_t marlaas_kernel_launch_count(void);
 

@@ -37,7 +37,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_register", "marlaas_adapter_pool_unregister", "marlaas_adapter_pool_lookup",
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
-    "marlaas_last_error", "marlaas_kernel_launch_count",
+    "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
 ]
 
 
@@ -93,6 +93,10 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_lora_build_index.argtypes = [vp, i64, P(marlaas_segments_t), vp, vp, vp, vp, vp, sz, u32, vp]
     L.marlaas_check_status.restype = i32
     L.marlaas_check_status.argtypes = [vp, vp]
+    L.marlaas_kernel_timing_begin.restype = i32
+    L.marlaas_kernel_timing_begin.argtypes = [vp]
+    L.marlaas_kernel_timing_end.restype = i32
+    L.marlaas_kernel_timing_end.argtypes = [vp, P(f32), P(i32)]
     L.marlaas_last_error.restype = ctypes.c_char_p
     L.marlaas_last_error.argtypes = []
     L.marlaas_kernel_launch_count.restype = u64
@@ -285,3 +289,14 @@ def marlaas_lora_build_index(pool: AdapterPool, T: int, seg: Segments, workspace
 
 def marlaas_check_status(pool: AdapterPool, stream=None) -> None:
     _check(load_library().marlaas_check_status(pool.handle, _stream(stream)))
+
+
+def marlaas_kernel_timing_begin(pool: AdapterPool) -> None:
+    _check(load_library().marlaas_kernel_timing_begin(pool.handle))
+
+
+def marlaas_kernel_timing_end(pool: AdapterPool):
+    """(summed device milliseconds, launches) of the dominant kernel since marlaas_kernel_timing_begin."""
+    ms, n = ctypes.c_float(), ctypes.c_int32()
+    _check(load_library().marlaas_kernel_timing_end(pool.handle, ctypes.byref(ms), ctypes.byref(n)))
+    return float(ms.value), int(n.value)

@@ -147,8 +147,11 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     float* h = h_save ? h_save : ws.h;
     if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, h, st)) != MARLAAS_OK) return rc;
-    if ((rc = launch_gemm_cuda_core(pool, T, pool->N, pool->K, (const bf16*)x, ldx, (const bf16*)W, ldw, false,
-                                    (bf16*)y, ldy, h, pool->d_Bs, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    {
+        TimedLaunch timed(pool, st);
+        if ((rc = launch_gemm_cuda_core(pool, T, pool->N, pool->K, (const bf16*)x, ldx, (const bf16*)W, ldw, false,
+                                        (bf16*)y, ldy, h, pool->d_Bs, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+    }
     return finish(pool, flags, st);
 }
 
@@ -188,6 +191,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
     }
     if (T > 0 && dx) {
+        TimedLaunch timed(pool, st);
         if ((rc = launch_gemm_cuda_core(pool, T, pool->K, pool->N, (const bf16*)dy, lddy, (const bf16*)W, ldw, true,
                                         (bf16*)dx, lddx, ws.g, pool->d_At, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }

@@ -34,6 +34,15 @@ void count_launch(int n = 1);
         ::marlaas::count_launch();                                                                   \
     } while (0)
 
+// Brackets one launch of the dominant kernel with events while the pool's timing mode is on.
+struct TimedLaunch {
+    marlaas_pool* pool;
+    cudaStream_t st;
+    bool on;
+    TimedLaunch(marlaas_pool* p, cudaStream_t s);
+    ~TimedLaunch();
+};
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -69,6 +78,10 @@ struct marlaas_pool {
     marlaas::bf16* d_Bs = nullptr;
     std::vector<marlaas::SlotMeta> slots;
     int sm_count = 0;
+    // kernel timing (marlaas_kernel_timing_begin/_end): event pairs around the dominant kernel
+    bool timing = false;
+    std::vector<cudaEvent_t> timing_events;
+    size_t timing_used = 0;
 };
 
 namespace marlaas {

@@ -22,6 +22,22 @@ marlaas_status_t fail(marlaas_status_t code, const char* fmt, ...) {
 }
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+TimedLaunch::TimedLaunch(marlaas_pool* p, cudaStream_t s) : pool(p), st(s), on(false) {
+    if (!p->timing) return;
+    if (p->timing_used + 2 > p->timing_events.size()) {
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+        p->timing_events.push_back(a);
+        p->timing_events.push_back(b);
+    }
+    on = cudaEventRecord(p->timing_events[p->timing_used], st) == cudaSuccess;
+}
+TimedLaunch::~TimedLaunch() {
+    if (!on) return;
+    cudaEventRecord(pool->timing_events[pool->timing_used + 1], st);
+    pool->timing_used += 2;
+}
+
 StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap) {
     StorageLayout L;
     size_t o = 0;
@@ -139,7 +155,32 @@ marlaas_status_t marlaas_adapter_pool_create(marlaas_pool_t** out, int device, i
     return MARLAAS_OK;
 }
 
+marlaas_status_t marlaas_kernel_timing_begin(marlaas_pool_t* pool) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "kernel_timing_begin: pool is NULL");
+    pool->timing = true;
+    pool->timing_used = 0;
+    return MARLAAS_OK;
+}
+
+marlaas_status_t marlaas_kernel_timing_end(marlaas_pool_t* pool, float* gemm_ms, int32_t* gemm_launches) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "kernel_timing_end: pool is NULL");
+    pool->timing = false;
+    float total = 0.f;
+    for (size_t i = 0; i + 1 < pool->timing_used; i += 2) {
+        MARLAAS_CUDA_TRY(cudaEventSynchronize(pool->timing_events[i + 1]));
+        float ms = 0.f;
+        MARLAAS_CUDA_TRY(cudaEventElapsedTime(&ms, pool->timing_events[i], pool->timing_events[i + 1]));
+        total += ms;
+    }
+    if (gemm_ms) *gemm_ms = total;
+    if (gemm_launches) *gemm_launches = (int32_t)(pool->timing_used / 2);
+    pool->timing_used = 0;
+    return MARLAAS_OK;
+}
+
 marlaas_status_t marlaas_adapter_pool_destroy(marlaas_pool_t* pool) {
+    if (pool)
+        for (cudaEvent_t e : pool->timing_events) cudaEventDestroy(e);
     delete pool;
     return MARLAAS_OK;
 }

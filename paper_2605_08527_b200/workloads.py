@@ -16,8 +16,10 @@ the same values widened exactly to ``float32``.
 """
 from __future__ import annotations
 
+import concurrent.futures
 import dataclasses
 import math
+import os
 from typing import Dict, List, Optional
 
 import numpy as np
@@ -69,18 +71,28 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
-def normal_bf16(seed: int, tensor_id: int, shape, sigma: float, sub: int = 0, chunk: int = 1 << 22):
+def normal_bf16(seed: int, tensor_id: int, shape, sigma: float, sub: int = 0, chunk: int = 1 << 21):
     """bf16-rounded N(0, sigma^2) tensor -> (bits uint16, values float32), element i of the
-    flattened tensor uses counters 2i and 2i+1."""
+    flattened tensor uses counters 2i and 2i+1.  Chunks are drawn on a thread pool (the result does
+    not depend on the chunking: every element is a pure function of its index)."""
     n = int(np.prod(shape))
     bits = np.empty(n, dtype=np.uint16)
-    for lo in range(0, n, chunk):
+
+    def fill(lo):
         hi = min(n, lo + chunk)
         idx = np.arange(lo, hi, dtype=np.uint64)
         u1 = uniform01(seed, tensor_id, idx * np.uint64(2), sub)
         u2 = uniform01(seed, tensor_id, idx * np.uint64(2) + np.uint64(1), sub)
         z = np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)
         bits[lo:hi] = f32_to_bf16_bits((z * sigma).astype(np.float32))
+
+    starts = list(range(0, n, chunk))
+    if len(starts) <= 1:
+        for lo in starts:
+            fill(lo)
+    else:
+        with concurrent.futures.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, starts))
     bits = bits.reshape(shape)
     return bits, bf16_bits_to_f32(bits)
 
