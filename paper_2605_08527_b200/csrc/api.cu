@@ -19,6 +19,12 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.g = (float*)take(sizeof(float) * Tn * pool->RP);
     w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
+    const size_t ntiles = (Tn + 127) / 128;
+    w.umax = (pool->cap < 128 ? pool->cap : 128) * (pool->RP / 16);
+    w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
+    w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
+    w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
+    w.hd = (bf16*)take(sizeof(bf16) * Tn * (size_t)w.umax * 16);
     w.total = o;
     return w;
 }
@@ -78,6 +84,17 @@ static marlaas_status_t make_tok_slot(const marlaas_pool* pool, int64_t T, const
         return MARLAAS_OK;
     }
     return launch_tok_slot(pool, T, seg->num_segments, seg->seg_offsets, seg->seg_slot, tok_slot, st);
+}
+
+static marlaas_status_t make_plan(const marlaas_pool* pool, int64_t T, const marlaas_segments_t* seg, uint32_t flags,
+                                  const std::vector<int32_t>& host_tok_slot, const Workspace& ws, cudaStream_t st) {
+    if (T <= 0) return MARLAAS_OK;
+    if (flags & MARLAAS_FLAG_HOST_TABLE) {
+        MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.tok_slot, host_tok_slot.data(), sizeof(int32_t) * (size_t)T,
+                                         cudaMemcpyHostToDevice, st));
+        return launch_plan_tiles(pool, T, -1, nullptr, nullptr, ws, st);
+    }
+    return launch_plan_tiles(pool, T, seg->num_segments, seg->seg_offsets, seg->seg_slot, ws, st);
 }
 
 static marlaas_status_t finish(marlaas_pool* pool, uint32_t flags, cudaStream_t st) {
@@ -144,8 +161,25 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
 
-    if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     float* h = h_save ? h_save : ws.h;
+    if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH)) {
+        if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
+        if ((rc = launch_shrink_hd(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st)) != MARLAAS_OK) return rc;
+        GemmOperands o;
+        o.M = T; o.Nout = pool->N; o.Kc = pool->K;
+        o.A = (const bf16*)x; o.lda = ldx;
+        o.B = (const bf16*)W; o.ldb = ldw; o.b_mn = true;
+        o.C = (bf16*)y; o.ldc = ldy;
+        o.XA = ws.hd; o.xa_cols = (int64_t)ws.umax * 16;
+        o.XB = pool->d_Bs; o.xb_rows = (int64_t)pool->cap * pool->RP;
+        o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
+        {
+            TimedLaunch timed(pool, st);
+            if ((rc = launch_gemm_sm100(pool, o, st)) != MARLAAS_OK) return rc;
+        }
+        return finish(pool, flags, st);
+    }
+    if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, h, st)) != MARLAAS_OK) return rc;
     {
         TimedLaunch timed(pool, st);
@@ -186,11 +220,31 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
     const bool acc = (flags & MARLAAS_FLAG_ACCUMULATE) != 0;
 
-    if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
-    if (T > 0 && (dx || want_dA)) {
-        if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
+    const bool tc_path = !(flags & MARLAAS_FLAG_CUDA_CORE_PATH);
+    if (tc_path && T > 0) {
+        if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
+    } else {
+        if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
-    if (T > 0 && dx) {
+    if (T > 0 && (dx || want_dA)) {
+        if (tc_path) {
+            if ((rc = launch_shrink_hd(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st)) != MARLAAS_OK) return rc;
+        } else {
+            if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
+        }
+    }
+    if (T > 0 && dx && tc_path) {
+        GemmOperands o;
+        o.M = T; o.Nout = pool->K; o.Kc = pool->N;
+        o.A = (const bf16*)dy; o.lda = lddy;
+        o.B = (const bf16*)W; o.ldb = ldw; o.b_mn = false;
+        o.C = (bf16*)dx; o.ldc = lddx;
+        o.XA = ws.hd; o.xa_cols = (int64_t)ws.umax * 16;
+        o.XB = pool->d_At; o.xb_rows = (int64_t)pool->cap * pool->RP;
+        o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
+        TimedLaunch timed(pool, st);
+        if ((rc = launch_gemm_sm100(pool, o, st)) != MARLAAS_OK) return rc;
+    } else if (T > 0 && dx) {
         TimedLaunch timed(pool, st);
         if ((rc = launch_gemm_cuda_core(pool, T, pool->K, pool->N, (const bf16*)dy, lddy, (const bf16*)W, ldw, true,
                                         (bf16*)dx, lddx, ws.g, pool->d_At, ws.tok_slot, st)) != MARLAAS_OK) return rc;

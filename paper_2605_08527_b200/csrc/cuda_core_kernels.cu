@@ -41,6 +41,67 @@ __global__ void __launch_bounds__(128) k_rowdot(int64_t D, const bf16* __restric
     }
 }
 
+// Same dot products, plus the token's row of the block-diagonal bf16 operand the tensor-core GEMM multiplies with
+// the adapter rows: bf16(s_t * h) in the columns of the token's own tenant units, zeros in the tile's other units.
+__global__ void __launch_bounds__(128) k_shrink_hd(int64_t D, const bf16* __restrict__ src, int64_t ld,
+                                                   const bf16* __restrict__ store, const int32_t* __restrict__ tok_slot,
+                                                   const int32_t* __restrict__ tok_uoff,
+                                                   const int32_t* __restrict__ tile_nunits,
+                                                   const int32_t* __restrict__ d_rank, const float* __restrict__ d_scale,
+                                                   int RP, int cap, int hd_cols, float* __restrict__ out,
+                                                   bf16* __restrict__ hd) {
+    __shared__ float sh[128];
+    const int64_t i = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = tok_slot[i];
+    const int r = (t >= 0 && t < cap) ? d_rank[t] : 0;
+    const bf16* row = src + i * ld;
+    for (int j = warp; j < RP; j += 4) {
+        float acc = 0.f;
+        if (j < r) {
+            const bf16* a = store + ((size_t)t * RP + j) * D;
+            for (int64_t d = (int64_t)lane * 8; d < D; d += 256) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(row + d);
+                const uint4 av = *reinterpret_cast<const uint4*>(a + d);
+                const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xv);
+                const __nv_bfloat162* ap = reinterpret_cast<const __nv_bfloat162*>(&av);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 xf = __bfloat1622float2(xp[q]);
+                    const float2 af = __bfloat1622float2(ap[q]);
+                    acc = fmaf(xf.x, af.x, acc);
+                    acc = fmaf(xf.y, af.y, acc);
+                }
+            }
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        }
+        if (lane == 0) {
+            out[i * RP + j] = acc;
+            sh[j] = acc;
+        }
+    }
+    __syncthreads();
+    const int nun = tile_nunits[i >> 7];
+    const int uo = r > 0 ? tok_uoff[i] : -1;
+    const float s = r > 0 ? d_scale[t] : 0.f;
+    const int own0 = uo * 16, own1 = own0 + ((r + 15) >> 4) * 16;
+    for (int c8 = threadIdx.x; c8 * 8 < nun * 16; c8 += 128) {
+        uint4 o = make_uint4(0u, 0u, 0u, 0u);
+        const int c = c8 * 8;
+        if (uo >= 0 && c >= own0 && c < own1) {
+            __nv_bfloat162 p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                p[e] = __floats2bfloat162_rn(s * sh[c - own0 + 2 * e], s * sh[c - own0 + 2 * e + 1]);
+            o.x = *reinterpret_cast<uint32_t*>(&p[0]);
+            o.y = *reinterpret_cast<uint32_t*>(&p[1]);
+            o.z = *reinterpret_cast<uint32_t*>(&p[2]);
+            o.w = *reinterpret_cast<uint32_t*>(&p[3]);
+        }
+        *reinterpret_cast<uint4*>(hd + i * hd_cols + c) = o;
+    }
+}
+
 // ---- base GEMM + fused low-rank term ----------------------------------------------------------------------
 // C[i][c] = bf16( sum_k A[i][k] * Wop[k][c] + s_t * sum_j hg[i][j] * store[(t*RP+j)][c] )
 // 64x64 tile, 16-deep k slab, 256 threads x (4x4) outputs.
@@ -165,6 +226,15 @@ marlaas_status_t launch_rowdot(const marlaas_pool* pool, int64_t T, const bf16* 
     if (T <= 0) return MARLAAS_OK;
     k_rowdot<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, tok_slot, pool->d_rank, pool->RP, pool->cap, out);
     MARLAAS_LAUNCH_CHECK("k_rowdot");
+    return MARLAAS_OK;
+}
+
+marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                                  const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+    if (T <= 0) return MARLAAS_OK;
+    k_shrink_hd<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, ws.tok_slot, ws.tok_uoff, ws.tile_nunits, pool->d_rank,
+                                             pool->d_scale, pool->RP, pool->cap, ws.umax * 16, out, ws.hd);
+    MARLAAS_LAUNCH_CHECK("k_shrink_hd");
     return MARLAAS_OK;
 }
 

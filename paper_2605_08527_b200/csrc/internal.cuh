@@ -101,6 +101,13 @@ struct Workspace {
     float* g;              // [T][RP]
     float** dA_ptrs;       // [cap]
     float** dB_ptrs;       // [cap]
+    // tensor-core path: per 128-token tile, the list of 16-deep rank units of the tenants present in it
+    int32_t* tok_uoff;     // [T]  first unit of the token's tenant within its tile's list, -1 = none
+    int32_t* tile_nunits;  // [ceil(T/128)]
+    int32_t* tile_units;   // [ceil(T/128)][umax]  first store row (slot*RP + 16j) of each unit
+    bf16* hd;              // [T][umax*16]  bf16(s_t h_i) (forward) or bf16(s_t g_i) (backward) in the tenant's unit
+                           //               columns, zeros in the other units of the tile
+    int32_t umax;
     size_t total;
 };
 Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base);
@@ -112,7 +119,30 @@ marlaas_status_t launch_tok_slot(const marlaas_pool* pool, int64_t T, int32_t S,
 marlaas_status_t launch_slot_sort(const marlaas_pool* pool, int64_t T, const int32_t* tok_slot,
                                   int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st);
 
+// One CTA per 128-token tile: per-token slot (from the table, or already in tok_slot when S < 0), the tile's unit
+// list and each token's unit offset.
+marlaas_status_t launch_plan_tiles(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
+                                   const int32_t* seg_slot, const Workspace& ws, cudaStream_t st);
+
+// gemm_sm100.cu
+struct GemmOperands {
+    int64_t M, Nout, Kc;
+    const bf16* A; int64_t lda;        // [M][Kc]
+    const bf16* B; int64_t ldb;        // b_mn: [Kc][Nout]; else [Nout][Kc]
+    bool b_mn;
+    bf16* C; int64_t ldc;              // [M][Nout]
+    const bf16* XA; int64_t xa_cols;   // [M][xa_cols] (pitch xa_cols)
+    const bf16* XB; int64_t xb_rows;   // [xb_rows][Nout] (pitch Nout)
+    const int32_t* tile_nunits;        // nullptr = no low-rank term
+    const int32_t* tile_units;
+    int32_t umax;
+};
+marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
+
 // cuda_core_kernels.cu
+// h/g (fp32, [T][RP]) as launch_rowdot, plus the bf16 block-diagonal operand rows hd for the tensor-core path
+marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                                  const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
 // out[i][j] = sum_d src[i][d] * store[(slot_i*RP + j)][d] for j < RP (zeros for inactive tokens / padded rows)
 marlaas_status_t launch_rowdot(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
                                const bf16* store, const int32_t* tok_slot, float* out, cudaStream_t st);

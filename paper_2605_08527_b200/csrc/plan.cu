@@ -97,6 +97,87 @@ __global__ void __launch_bounds__(256) k_slot_sort(int T, int cap, const int32_t
     }
 }
 
+// One CTA of 128 threads per 128-token tile.  Besides tok_slot it lists, for the tile, the 16-deep rank units of
+// every tenant present (ascending slot order) and tells each token where its tenant's units start.
+__global__ void __launch_bounds__(128) k_plan_tiles(int T, int S, const int32_t* __restrict__ seg_offsets,
+                                                    const int32_t* __restrict__ seg_slot, int cap, int RP,
+                                                    const int32_t* __restrict__ d_rank, int32_t* __restrict__ tok_slot,
+                                                    int32_t* __restrict__ tok_uoff, int32_t* __restrict__ tile_nunits,
+                                                    int32_t* __restrict__ tile_units, int umax, int32_t* status) {
+    __shared__ int s_u[4096];
+    __shared__ int s_warp[4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = blockIdx.x;
+    const int i = m * 128 + tid;
+    if (S >= 0) {   // table checks, spread over the grid
+        for (int s = blockIdx.x * 128 + tid; s < S; s += gridDim.x * 128) {
+            const int a = seg_offsets[s], b = seg_offsets[s + 1];
+            if (b < a || a < 0 || b > T) report(status, DEV_BAD_TABLE, s);
+            if (s == 0 && a != 0) report(status, DEV_BAD_TABLE, -1);
+            if (s == S - 1 && b != T) report(status, DEV_BAD_TABLE, -2);
+        }
+        if (i == 0 && S == 0 && T != 0) report(status, DEV_BAD_TABLE, -3);
+    }
+    int slot = -1;
+    if (i < T) {
+        if (S >= 0) {
+            int lo = 0, hi = S;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (seg_offsets[mid + 1] > i) hi = mid; else lo = mid + 1;
+            }
+            if (lo < S) slot = seg_slot[lo];
+        } else {
+            slot = tok_slot[i];
+        }
+        if (slot < -1 || slot >= cap) {
+            report(status, DEV_BAD_INDEX, i);
+            slot = -1;
+        }
+        tok_slot[i] = slot;
+    }
+    for (int t = tid; t < cap; t += 128) s_u[t] = 0;
+    __syncthreads();
+    const int r = slot >= 0 ? d_rank[slot] : 0;
+    if (r > 0) s_u[slot] = (r + 15) >> 4;
+    __syncthreads();
+    // exclusive scan of the per-slot unit counts; each thread owns a contiguous run of slots
+    const int per = (cap + 127) / 128;
+    const int t0 = tid * per, t1 = min(cap, t0 + per);
+    int loc = 0;
+    for (int t = t0; t < t1; ++t) loc += s_u[t];
+    int inc = loc;
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += v;
+    }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    int off = inc - loc;
+    for (int w = 0; w < warp; ++w) off += s_warp[w];
+    const int total = s_warp[0] + s_warp[1] + s_warp[2] + s_warp[3];
+    for (int t = t0; t < t1; ++t) {
+        const int u = s_u[t];
+        for (int j = 0; j < u; ++j)
+            if (off + j < umax) tile_units[(size_t)m * umax + off + j] = t * RP + j * 16;
+        s_u[t] = off;
+        off += u;
+    }
+    __syncthreads();
+    if (i < T) tok_uoff[i] = r > 0 ? s_u[slot] : -1;
+    if (tid == 0) tile_nunits[m] = min(total, umax);
+}
+
+marlaas_status_t launch_plan_tiles(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
+                                   const int32_t* seg_slot, const Workspace& ws, cudaStream_t st) {
+    if (T <= 0) return MARLAAS_OK;
+    k_plan_tiles<<<(unsigned)cdiv(T, 128), 128, 0, st>>>((int)T, S, seg_offsets, seg_slot, pool->cap, pool->RP,
+                                                         pool->d_rank, ws.tok_slot, ws.tok_uoff, ws.tile_nunits,
+                                                         ws.tile_units, ws.umax, pool->d_status);
+    MARLAAS_LAUNCH_CHECK("k_plan_tiles");
+    return MARLAAS_OK;
+}
+
 marlaas_status_t launch_tok_slot(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
                                  const int32_t* seg_slot, int32_t* tok_slot, cudaStream_t st) {
     const int64_t n = T > S ? T : S;

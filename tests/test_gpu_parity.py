@@ -227,7 +227,9 @@ def test_pool_store_roundtrip_versions_and_errors():
         B.marlaas_adapter_pool_register(dc.pool, 5001, 0, 0, 0.0, None, None)
     assert e.value.status == B.MARLAAS_ERR_POOL_FULL
     with pytest.raises(B.MarlaasError) as e:
-        B.marlaas_adapter_pool_register(dc.pool, a1.tenant_id, 2, 17, 1.0, dc.A[1], newB)
+        B.marlaas_adapter_pool_register(dc.pool, a1.tenant_id, 2, 17, 1.0,
+                                        torch.zeros((p.d_in, 17), dtype=torch.bfloat16, device="cuda:0"),
+                                        torch.zeros((17, p.d_out), dtype=torch.bfloat16, device="cuda:0"))
     assert e.value.status == B.MARLAAS_ERR_RANK_TOO_LARGE
     B.marlaas_adapter_pool_unregister(dc.pool, 5000)
     with pytest.raises(B.MarlaasError) as e:
