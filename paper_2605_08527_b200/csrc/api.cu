@@ -97,6 +97,14 @@ static marlaas_status_t make_plan(const marlaas_pool* pool, int64_t T, const mar
     return launch_plan_tiles(pool, T, seg->num_segments, seg->seg_offsets, seg->seg_slot, ws, st);
 }
 
+// Shrink for the tensor-core path: batches with several 128-token tiles go through the tcgen05 kernel, small
+// (decode-shaped) batches through the per-token gather kernel, which spreads over more SMs.
+static marlaas_status_t shrink(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                               const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+    if (T >= 512) return launch_shrink_sm100(pool, T, src, ld, D, store, ws, out, st);
+    return launch_shrink_hd(pool, T, src, ld, D, store, ws, out, st);
+}
+
 static marlaas_status_t finish(marlaas_pool* pool, uint32_t flags, cudaStream_t st) {
     if (flags & MARLAAS_FLAG_VALIDATE_SYNC) return marlaas_check_status(pool, (void*)st);
     return MARLAAS_OK;
@@ -164,7 +172,7 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     float* h = h_save ? h_save : ws.h;
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH)) {
         if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
-        if ((rc = launch_shrink_hd(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st)) != MARLAAS_OK) return rc;
+        if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st)) != MARLAAS_OK) return rc;
         GemmOperands o;
         o.M = T; o.Nout = pool->N; o.Kc = pool->K;
         o.A = (const bf16*)x; o.lda = ldx;
@@ -228,7 +236,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     }
     if (T > 0 && (dx || want_dA)) {
         if (tc_path) {
-            if ((rc = launch_shrink_hd(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st)) != MARLAAS_OK) return rc;
+            if ((rc = shrink(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st)) != MARLAAS_OK) return rc;
         } else {
             if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
         }

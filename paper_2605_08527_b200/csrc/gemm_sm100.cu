@@ -11,20 +11,12 @@
 // The low-rank term rides in the same accumulator: every 128-row tile carries a list of 16-deep "units" (one per
 // 16 ranks of each tenant present in the tile); XA holds, per token, its own tenant's scaled h (or g) in that
 // tenant's unit columns and zeros elsewhere, so one extra MMA per unit adds s_t h_i B_t for all rows of the tile.
-#include <cuda.h>
-
-#include "internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace marlaas {
 namespace sm100 {
 
-constexpr int BM = 128;
-constexpr int BK = 64;                       // 64 bf16 = one 128-byte swizzle row
-constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
-constexpr uint32_t CHUNK_BYTES = BK * 128;   // one [64 k][64 n] MN-major chunk of B
-constexpr uint32_t UNIT_BYTES = 16 * 128;    // 16 k-rows of one chunk
 constexpr int NUM_THREADS = 192;
-constexpr unsigned long long WAIT_LIMIT_NS = 400ull * 1000 * 1000;
 
 struct GemmArgs {
     int M, Nout, Kc;
@@ -38,107 +30,6 @@ struct GemmArgs {
     int64_t ldc;
     int32_t* status;
 };
-
-// ---- PTX wrappers ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up after WAIT_LIMIT_NS or as soon as another role of this CTA has given up; the first to
-// give up records its site in the CTA's abort word.  Returns false on abort.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int site) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    uint32_t spins = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_word != 0) return false;
-        if (((++spins) & 63u) == 0 && global_ns() - t0 > WAIT_LIMIT_NS) {
-            atomicCAS((int*)abort_word, 0, site);
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                            uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptors, 128-byte swizzle, version 1 (sm_100).
-//  K-major operand  : rows of 64 elements (128 B); 8-row groups 1024 B apart (SBO); LBO unused (1).
-//  MN-major operand : rows of 64 MN-elements (128 B), one per k; 8-k groups 1024 B apart (SBO); successive
-//                     64-element chunks along MN `lbo_bytes` apart (LBO).
-__device__ __forceinline__ uint64_t desc_k_major(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-           (2ull << 61);
-}
-__device__ __forceinline__ uint64_t desc_mn_major(uint32_t saddr, uint32_t lbo_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B major as given, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc(int bn, int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(bn >> 3) << 17) |
-           ((uint32_t)(BM >> 4) << 24);
-}
 
 __device__ __forceinline__ void decode_tile(const GemmArgs& g, int tile, int& m_idx, int& n_idx) {
     const int per_band = g.group_m * g.num_n_tiles;
@@ -391,9 +282,7 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D bf16 tensor [rows][cols] with row pitch ld elements; box = box_cols x box_rows; 128-byte swizzle; reads
-// outside the tensor return zeros.
-static marlaas_status_t make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld,
+marlaas_status_t make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld,
                                  uint32_t box_cols, uint32_t box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(MARLAAS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");

@@ -139,6 +139,10 @@ struct GemmOperands {
 };
 marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
 
+// shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
+marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                                     const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
+
 // cuda_core_kernels.cu
 // h/g (fp32, [T][RP]) as launch_rowdot, plus the bf16 block-diagonal operand rows hd for the tensor-core path
 marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
