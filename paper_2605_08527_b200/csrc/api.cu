@@ -25,6 +25,19 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
     w.hd = (bf16*)take(sizeof(bf16) * Tn * (size_t)w.umax * 16);
+    const size_t nblk = (Tn + 63) / 64;
+    const bool grad_tc = grad_sm100_eligible(pool, (int64_t)Tn);
+    w.HW = ((2 * pool->RP + 63) / 64) * 64;
+    w.max_copies = grad_tc ? (int32_t)(3 * nblk + 2 * (size_t)pool->cap) : 0;
+    const size_t gb = grad_tc ? nblk : 0, gc = grad_tc ? (size_t)pool->cap : 0;
+    w.blk_np = (int32_t*)take(sizeof(int32_t) * gb);
+    w.blk_base = (int32_t*)take(sizeof(int32_t) * (gb + 1));
+    w.blk_rank = (int32_t*)take(sizeof(int32_t) * gb * gc);
+    w.ten_nblk = (int32_t*)take(sizeof(int32_t) * gc);
+    w.ten_blks = (int32_t*)take(sizeof(int32_t) * gb * gc);
+    w.ten_pos = (int32_t*)take(sizeof(int32_t) * gb * gc);
+    w.gflag = (int32_t*)take(16);
+    w.hm = (bf16*)take(sizeof(bf16) * (size_t)w.max_copies * 64 * (size_t)w.HW);
     w.total = o;
     return w;
 }
@@ -258,21 +271,28 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
                                         (bf16*)dx, lddx, ws.g, pool->d_At, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
     if (want_dA || want_dB) {
-        if ((rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st)) != MARLAAS_OK) return rc;
+        const bool tc_grad = tc_path && grad_sm100_eligible(pool, T);
+        const int32_t* run_flag = tc_grad ? ws.gflag : nullptr;   // the CUDA-core kernels run only if the flag is set
+        if (tc_grad && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
+        if ((rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
         if (want_dB) {
             const float* h = h_saved;
             if (!h && T > 0) {
-                if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, ws.h, st)) != MARLAAS_OK) return rc;
+                if (tc_path) rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, ws.h, st);
+                else rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, ws.h, st);
+                if (rc != MARLAAS_OK) return rc;
                 h = ws.h;
             }
             MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, false, acc, ws, st)) != MARLAAS_OK) return rc;
             if ((rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
-                                         false, acc, st)) != MARLAAS_OK) return rc;
+                                         false, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }
         if (want_dA) {
             MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, true, acc, ws, st)) != MARLAAS_OK) return rc;
             if ((rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
-                                         true, acc, st)) != MARLAAS_OK) return rc;
+                                         true, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }
     }
     return finish(pool, flags, st);

@@ -182,7 +182,8 @@ __global__ void __launch_bounds__(128) k_grad_reduce(int64_t C, const bf16* __re
                                                      const int32_t* __restrict__ d_rank,
                                                      const float* __restrict__ d_scale, int RP,
                                                      float* const* __restrict__ out_ptrs, int transpose_out,
-                                                     int accumulate) {
+                                                     int accumulate, const int32_t* __restrict__ run_flag) {
+    if (run_flag != nullptr && run_flag[0] == 0) return;
     const int t = blockIdx.y;
     float* out = out_ptrs[t];
     const int r = d_rank[t];
@@ -256,10 +257,11 @@ marlaas_status_t launch_gemm_cuda_core(const marlaas_pool* pool, int64_t T, int6
 
 marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const bf16* src, int64_t ld,
                                     const float* hg, const int32_t* perm, const int32_t* slot_offset,
-                                    float* const* out_ptrs, bool transpose_out, bool accumulate, cudaStream_t st) {
+                                    float* const* out_ptrs, bool transpose_out, bool accumulate, cudaStream_t st,
+                                    const int32_t* run_flag) {
     dim3 grid((unsigned)cdiv(C, 128), (unsigned)pool->cap, (unsigned)(pool->RP / 16));
     k_grad_reduce<<<grid, 128, 0, st>>>(C, src, ld, hg, perm, slot_offset, pool->d_rank, pool->d_scale, pool->RP,
-                                        out_ptrs, transpose_out ? 1 : 0, accumulate ? 1 : 0);
+                                        out_ptrs, transpose_out ? 1 : 0, accumulate ? 1 : 0, run_flag);
     MARLAAS_LAUNCH_CHECK("k_grad_reduce");
     return MARLAAS_OK;
 }

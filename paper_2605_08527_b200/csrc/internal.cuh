@@ -108,6 +108,16 @@ struct Workspace {
     bf16* hd;              // [T][umax*16]  bf16(s_t h_i) (forward) or bf16(s_t g_i) (backward) in the tenant's unit
                            //               columns, zeros in the other units of the tile
     int32_t umax;
+    // tensor-core gradient reductions: 64-token blocks, one masked copy of the block's r-vectors per tenant present
+    int32_t* blk_np;       // [nblk]        tenants present in the block
+    int32_t* blk_base;     // [nblk+1]      exclusive scan of blk_np (= first copy of the block)
+    int32_t* blk_rank;     // [nblk][cap]   rank of the tenant among the block's present tenants, -1 = absent
+    int32_t* ten_nblk;     // [cap]         copies of the tenant
+    int32_t* ten_blks;     // [cap][nblk]   the tenant's blocks, ascending
+    int32_t* ten_pos;      // [cap][nblk]   the matching copy positions
+    int32_t* gflag;        // [4]           [0] = 1 when the copies do not fit (CUDA-core reduction runs instead)
+    bf16* hm;              // [max_copies*64][HW]  hi | lo split r-vectors
+    int32_t max_copies, HW;
     size_t total;
 };
 Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base);
@@ -116,8 +126,10 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base);
 // plan.cu
 marlaas_status_t launch_tok_slot(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
                                  const int32_t* seg_slot, int32_t* tok_slot, cudaStream_t st);
+// run_flag (optional, device): the kernel returns at once unless run_flag[0] != 0
 marlaas_status_t launch_slot_sort(const marlaas_pool* pool, int64_t T, const int32_t* tok_slot,
-                                  int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st);
+                                  int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st,
+                                  const int32_t* run_flag = nullptr);
 
 // One CTA per 128-token tile: per-token slot (from the table, or already in tok_slot when S < 0), the tile's unit
 // list and each token's unit offset.
@@ -159,6 +171,14 @@ marlaas_status_t launch_gemm_cuda_core(const marlaas_pool* pool, int64_t T, int6
 // out_t[j][c] (transpose_out = false, ld = C) or out_t[c][j] (true, ld = r_t) (+)= s_t * sum_{i in t} hg[i][j] * src[i][c]
 marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const bf16* src, int64_t ld,
                                     const float* hg, const int32_t* perm, const int32_t* slot_offset,
-                                    float* const* out_ptrs, bool transpose_out, bool accumulate, cudaStream_t st);
+                                    float* const* out_ptrs, bool transpose_out, bool accumulate, cudaStream_t st,
+                                    const int32_t* run_flag = nullptr);
+
+// grad_sm100.cu: the same reductions on the tensor cores
+bool grad_sm100_eligible(const marlaas_pool* pool, int64_t T);
+marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Workspace& ws, cudaStream_t st);
+marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
+                                   const float* hg, float* const* out_ptrs, bool transpose_out, bool accumulate,
+                                   const Workspace& ws, cudaStream_t st);
 
 }  // namespace marlaas

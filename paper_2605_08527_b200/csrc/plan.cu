@@ -44,7 +44,9 @@ __global__ void k_tok_slot(int T, int S, const int32_t* __restrict__ seg_offsets
 // this key's tokens in ascending token order.  Stable by construction.
 __global__ void __launch_bounds__(256) k_slot_sort(int T, int cap, const int32_t* __restrict__ tok_slot,
                                                    int32_t* __restrict__ slot_count,
-                                                   int32_t* __restrict__ slot_offset, int32_t* __restrict__ perm) {
+                                                   int32_t* __restrict__ slot_offset, int32_t* __restrict__ perm,
+                                                   const int32_t* __restrict__ run_flag) {
+    if (run_flag != nullptr && run_flag[0] == 0) return;
     const int key = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ int s_warp[8];
@@ -189,8 +191,9 @@ marlaas_status_t launch_tok_slot(const marlaas_pool* pool, int64_t T, int32_t S,
 }
 
 marlaas_status_t launch_slot_sort(const marlaas_pool* pool, int64_t T, const int32_t* tok_slot,
-                                  int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st) {
-    k_slot_sort<<<pool->cap + 1, 256, 0, st>>>((int)T, pool->cap, tok_slot, slot_count, slot_offset, perm);
+                                  int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st,
+                                  const int32_t* run_flag) {
+    k_slot_sort<<<pool->cap + 1, 256, 0, st>>>((int)T, pool->cap, tok_slot, slot_count, slot_offset, perm, run_flag);
     MARLAAS_LAUNCH_CHECK("k_slot_sort");
     return MARLAAS_OK;
 }

@@ -74,6 +74,15 @@ def test_small_ragged_cases(flags, seed, T, K, N, ranks):
     _check_case(w, w.projections[0], flags=flags, capacity=len(ranks) + 2)
 
 
+def test_finely_interleaved_tenants_with_backward():
+    # every token its own segment, tenants drawn uniformly: the per-block tenant copies of the tensor-core gradient
+    # reduction do not fit, so the device-side switch to the CUDA-core reduction is exercised
+    T, n = 700, 12
+    w = wl.small_random_case(61, T, 128, 136, [8] * n, n_segments=4)
+    w.seg_offsets, w.seg_slot = wl.per_token_table(wl.uniform_token_slots(61, T, n))
+    _check_case(w, w.projections[0])
+
+
 def test_cfg2_decode_full_size():
     w = wl.make_workload(2)
     _check_case(w, w.projections[0])
