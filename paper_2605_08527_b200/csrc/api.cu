@@ -19,8 +19,8 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.g = (float*)take(sizeof(float) * Tn * pool->RP);
     w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
-    const size_t ntiles = (Tn + 127) / 128;
-    w.umax = (pool->cap < 128 ? pool->cap : 128) * (pool->RP / 16);
+    const size_t ntiles = (Tn + 255) / 256;
+    w.umax = (pool->cap < 256 ? pool->cap : 256) * (pool->RP / 16);
     w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
@@ -196,7 +196,8 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
         {
             TimedLaunch timed(pool, st);
-            if ((rc = launch_gemm_sm100(pool, o, st)) != MARLAAS_OK) return rc;
+            rc = gemm2_sm100_eligible(pool, T) ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
+            if (rc != MARLAAS_OK) return rc;
         }
         return finish(pool, flags, st);
     }
@@ -264,7 +265,8 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         o.XB = pool->d_At; o.xb_rows = (int64_t)pool->cap * pool->RP;
         o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
         TimedLaunch timed(pool, st);
-        if ((rc = launch_gemm_sm100(pool, o, st)) != MARLAAS_OK) return rc;
+        rc = gemm2_sm100_eligible(pool, T) ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
+        if (rc != MARLAAS_OK) return rc;
     } else if (T > 0 && dx) {
         TimedLaunch timed(pool, st);
         if ((rc = launch_gemm_cuda_core(pool, T, pool->K, pool->N, (const bf16*)dy, lddy, (const bf16*)W, ldw, true,

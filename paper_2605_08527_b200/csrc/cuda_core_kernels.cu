@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(128) k_shrink_hd(int64_t D, const bf16* __rest
         }
     }
     __syncthreads();
-    const int nun = tile_nunits[i >> 7];
+    const int nun = tile_nunits[i >> 8];
     const int uo = r > 0 ? tok_uoff[i] : -1;
     const float s = r > 0 ? d_scale[t] : 0.f;
     const int own0 = uo * 16, own1 = own0 + ((r + 15) >> 4) * 16;

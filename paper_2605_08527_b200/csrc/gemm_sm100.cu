@@ -8,7 +8,7 @@
 // forward : A = x,  B = W        (W is [Kc][Nout] row-major: an MN-major B operand),  XA = bf16(s_t h), XB = B_t rows
 // backward: A = dy, B = W^T      (W is [Nout][Kc] row-major: a K-major B operand),    XA = bf16(s_t g), XB = A_t^T rows
 //
-// The low-rank term rides in the same accumulator: every 128-row tile carries a list of 16-deep "units" (one per
+// The low-rank term rides in the same accumulator: every 256-row plan tile carries a list of 16-deep "units" (one per
 // 16 ranks of each tenant present in the tile); XA holds, per token, its own tenant's scaled h (or g) in that
 // tenant's unit columns and zeros elsewhere, so one extra MMA per unit adds s_t h_i B_t for all rows of the tile.
 #include "sm100_ptx.cuh"
@@ -23,8 +23,8 @@ struct GemmArgs {
     int num_m_tiles, num_n_tiles, num_kb;
     int group_m;
     int b_mn;                      // 1: B is MN-major in memory ([Kc][Nout]); 0: K-major ([Nout][Kc])
-    const int32_t* tile_nunits;    // [num_m_tiles] or nullptr
-    const int32_t* tile_units;     // [num_m_tiles][umax]: first row of the unit in the XB store
+    const int32_t* tile_nunits;    // [ceil(M/256)] (one list per 256-row plan tile) or nullptr
+    const int32_t* tile_units;     // [ceil(M/256)][umax]: first row of the unit in the XB store
     int umax;
     bf16* C;
     int64_t ldc;
@@ -122,7 +122,7 @@ k_gemm_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         tma_load_2d(sB + s * B_STAGE_BYTES, &tmB, full, kb * BK, n0);
                     }
                 }
-                const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
+                const int nun = g.tile_nunits ? g.tile_nunits[m_idx >> 1] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 2))) break;
@@ -131,7 +131,7 @@ k_gemm_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     mbar_expect_tx(full, A_STAGE_BYTES + nv * nchunk * UNIT_BYTES);
                     tma_load_2d(sA + s * A_STAGE_BYTES, &tmXA, full, x0 * 16, m0);
                     for (int u = 0; u < nv; ++u) {
-                        const int row = g.tile_units[(size_t)m_idx * g.umax + x0 + u];
+                        const int row = g.tile_units[(size_t)(m_idx >> 1) * g.umax + x0 + u];
                         for (int c = 0; c < nchunk; ++c)
                             tma_load_2d(sB + s * B_STAGE_BYTES + c * CHUNK_BYTES + u * UNIT_BYTES, &tmXB, full,
                                         n0 + c * 64, row);
@@ -181,7 +181,7 @@ k_gemm_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     }
                     tc_commit(bar_empty + 8 * s);
                 }
-                const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
+                const int nun = g.tile_nunits ? g.tile_nunits[m_idx >> 1] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 5))) break;

@@ -101,10 +101,10 @@ struct Workspace {
     float* g;              // [T][RP]
     float** dA_ptrs;       // [cap]
     float** dB_ptrs;       // [cap]
-    // tensor-core path: per 128-token tile, the list of 16-deep rank units of the tenants present in it
+    // tensor-core path: per 256-token plan tile, the list of 16-deep rank units of the tenants present in it
     int32_t* tok_uoff;     // [T]  first unit of the token's tenant within its tile's list, -1 = none
-    int32_t* tile_nunits;  // [ceil(T/128)]
-    int32_t* tile_units;   // [ceil(T/128)][umax]  first store row (slot*RP + 16j) of each unit
+    int32_t* tile_nunits;  // [ceil(T/256)]
+    int32_t* tile_units;   // [ceil(T/256)][umax]  first store row (slot*RP + 16j) of each unit
     bf16* hd;              // [T][umax*16]  bf16(s_t h_i) (forward) or bf16(s_t g_i) (backward) in the tenant's unit
                            //               columns, zeros in the other units of the tile
     int32_t umax;
@@ -131,7 +131,7 @@ marlaas_status_t launch_slot_sort(const marlaas_pool* pool, int64_t T, const int
                                   int32_t* slot_count, int32_t* slot_offset, int32_t* perm, cudaStream_t st,
                                   const int32_t* run_flag = nullptr);
 
-// One CTA per 128-token tile: per-token slot (from the table, or already in tok_slot when S < 0), the tile's unit
+// One CTA per 256-token plan tile: per-token slot (from the table, or already in tok_slot when S < 0), the tile's unit
 // list and each token's unit offset.
 marlaas_status_t launch_plan_tiles(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
                                    const int32_t* seg_slot, const Workspace& ws, cudaStream_t st);
@@ -150,6 +150,9 @@ struct GemmOperands {
     int32_t umax;
 };
 marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
+// gemm2_sm100.cu: the same product with 2-CTA clusters (256 x 256 tiles), for batches of at least 1024 rows
+bool gemm2_sm100_eligible(const marlaas_pool* pool, int64_t M);
+marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
 
 // shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,

@@ -99,20 +99,20 @@ __global__ void __launch_bounds__(256) k_slot_sort(int T, int cap, const int32_t
     }
 }
 
-// One CTA of 128 threads per 128-token tile.  Besides tok_slot it lists, for the tile, the 16-deep rank units of
+// One CTA of 256 threads per 256-token plan tile.  Besides tok_slot it lists, for the tile, the 16-deep rank units of
 // every tenant present (ascending slot order) and tells each token where its tenant's units start.
-__global__ void __launch_bounds__(128) k_plan_tiles(int T, int S, const int32_t* __restrict__ seg_offsets,
+__global__ void __launch_bounds__(256) k_plan_tiles(int T, int S, const int32_t* __restrict__ seg_offsets,
                                                     const int32_t* __restrict__ seg_slot, int cap, int RP,
                                                     const int32_t* __restrict__ d_rank, int32_t* __restrict__ tok_slot,
                                                     int32_t* __restrict__ tok_uoff, int32_t* __restrict__ tile_nunits,
                                                     int32_t* __restrict__ tile_units, int umax, int32_t* status) {
     __shared__ int s_u[4096];
-    __shared__ int s_warp[4];
+    __shared__ int s_warp[8];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = blockIdx.x;
-    const int i = m * 128 + tid;
+    const int i = m * 256 + tid;
     if (S >= 0) {   // table checks, spread over the grid
-        for (int s = blockIdx.x * 128 + tid; s < S; s += gridDim.x * 128) {
+        for (int s = blockIdx.x * 256 + tid; s < S; s += gridDim.x * 256) {
             const int a = seg_offsets[s], b = seg_offsets[s + 1];
             if (b < a || a < 0 || b > T) report(status, DEV_BAD_TABLE, s);
             if (s == 0 && a != 0) report(status, DEV_BAD_TABLE, -1);
@@ -138,13 +138,13 @@ __global__ void __launch_bounds__(128) k_plan_tiles(int T, int S, const int32_t*
         }
         tok_slot[i] = slot;
     }
-    for (int t = tid; t < cap; t += 128) s_u[t] = 0;
+    for (int t = tid; t < cap; t += 256) s_u[t] = 0;
     __syncthreads();
     const int r = slot >= 0 ? d_rank[slot] : 0;
     if (r > 0) s_u[slot] = (r + 15) >> 4;
     __syncthreads();
     // exclusive scan of the per-slot unit counts; each thread owns a contiguous run of slots
-    const int per = (cap + 127) / 128;
+    const int per = (cap + 255) / 256;
     const int t0 = tid * per, t1 = min(cap, t0 + per);
     int loc = 0;
     for (int t = t0; t < t1; ++t) loc += s_u[t];
@@ -157,7 +157,8 @@ __global__ void __launch_bounds__(128) k_plan_tiles(int T, int S, const int32_t*
     __syncthreads();
     int off = inc - loc;
     for (int w = 0; w < warp; ++w) off += s_warp[w];
-    const int total = s_warp[0] + s_warp[1] + s_warp[2] + s_warp[3];
+    int total = 0;
+    for (int w = 0; w < 8; ++w) total += s_warp[w];
     for (int t = t0; t < t1; ++t) {
         const int u = s_u[t];
         for (int j = 0; j < u; ++j)
@@ -173,7 +174,7 @@ __global__ void __launch_bounds__(128) k_plan_tiles(int T, int S, const int32_t*
 marlaas_status_t launch_plan_tiles(const marlaas_pool* pool, int64_t T, int32_t S, const int32_t* seg_offsets,
                                    const int32_t* seg_slot, const Workspace& ws, cudaStream_t st) {
     if (T <= 0) return MARLAAS_OK;
-    k_plan_tiles<<<(unsigned)cdiv(T, 128), 128, 0, st>>>((int)T, S, seg_offsets, seg_slot, pool->cap, pool->RP,
+    k_plan_tiles<<<(unsigned)cdiv(T, 256), 256, 0, st>>>((int)T, S, seg_offsets, seg_slot, pool->cap, pool->RP,
                                                          pool->d_rank, ws.tok_slot, ws.tok_uoff, ws.tile_nunits,
                                                          ws.tile_units, ws.umax, pool->d_status);
     MARLAAS_LAUNCH_CHECK("k_plan_tiles");

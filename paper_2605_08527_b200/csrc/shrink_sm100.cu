@@ -1,4 +1,4 @@
-// Segmented shrink on the tensor cores (sm_100a): per 128-token tile, h = x A_t (or g = dy B_t^T) for every tenant
+// Segmented shrink on the tensor cores (sm_100a): per 128-token tile (half of a 256-token plan tile), h = x A_t (or g = dy B_t^T) for every tenant
 // present in the tile at once.
 //
 // The tile's unit list (16 ranks of one tenant per unit, built by the plan kernel) names the adapter rows to
@@ -96,10 +96,10 @@ k_shrink_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant_
             uint32_t it = 0;
             bool ok = true;
             for (int m = blockIdx.x; m < g.num_m_tiles && ok; m += gridDim.x) {
-                const int nun = g.tile_nunits[m];
+                const int nun = g.tile_nunits[m >> 1];
                 for (int g0 = 0; g0 < nun && ok; g0 += GROUP_UNITS) {
                     const int nug = min(GROUP_UNITS, nun - g0);
-                    const int32_t* rows = g.tile_units + (size_t)m * g.umax + g0;
+                    const int32_t* rows = g.tile_units + (size_t)(m >> 1) * g.umax + g0;
                     for (int kb = 0; kb < g.num_kb && ok; ++kb, ++it) {
                         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                         if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 11))) break;
@@ -128,7 +128,7 @@ k_shrink_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant_
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int m = blockIdx.x; m < g.num_m_tiles && ok; m += gridDim.x) {
-                const int nun = g.tile_nunits[m];
+                const int nun = g.tile_nunits[m >> 1];
                 for (int g0 = 0; g0 < nun && ok; g0 += GROUP_UNITS, ++lt) {
                     const int nug = min(GROUP_UNITS, nun - g0);
                     const uint32_t idesc = make_idesc(nug * 16, 0);
@@ -166,7 +166,7 @@ k_shrink_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant_
         uint32_t lt = 0;
         bool ok = true;
         for (int m = blockIdx.x; m < g.num_m_tiles && ok; m += gridDim.x) {
-            const int nun = g.tile_nunits[m];
+            const int nun = g.tile_nunits[m >> 1];
             const int row = m * BM + q * 32 + lane;
             int uo = -1, nu = 0;
             float sc = 0.f;

@@ -68,6 +68,8 @@ def test_cfg1_tiny_forward_backward(flags):
     (3, 129, 512, 72, (16, 16, 7)),           # one token past a 128-row tile
     (4, 1, 64, 64, (4,)),                     # single token
     (5, 640, 200, 328, (64, 33, 1, 12, 9)),   # several row tiles, odd ranks
+    (6, 1100, 264, 392, (16, 8, 32, 5)),      # 2-CTA tiles with ragged tails in rows, columns and depth
+    (7, 1290, 128, 136, (8, 64)),             # second CTA of the last pair has only 10 rows; its column half is empty
 ])
 def test_small_ragged_cases(flags, seed, T, K, N, ranks):
     w = wl.small_random_case(seed, T, K, N, list(ranks), n_segments=min(9, T + 1))
