@@ -183,6 +183,21 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
 
     float* h = h_save ? h_save : ws.h;
+    if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH) && decode_sm100_eligible(pool, T)) {
+        int32_t S = seg->num_segments;
+        if (flags & MARLAAS_FLAG_HOST_TABLE) {
+            MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.tok_slot, host_ts.data(), sizeof(int32_t) * (size_t)T,
+                                             cudaMemcpyHostToDevice, st));
+            S = -1;
+        }
+        {
+            TimedLaunch timed(pool, st);
+            rc = launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
+                                     seg->seg_offsets, seg->seg_slot, ws, h, st);
+            if (rc != MARLAAS_OK) return rc;
+        }
+        return finish(pool, flags, st);
+    }
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH)) {
         if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
         if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st)) != MARLAAS_OK) return rc;

@@ -154,6 +154,13 @@ marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands&
 bool gemm2_sm100_eligible(const marlaas_pool* pool, int64_t M);
 marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
 
+// decode_sm100.cu: the whole forward for batches of at most 256 tokens (two overlapping kernels).
+// S < 0: ws.tok_slot already holds the per-token slots.
+bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T);
+marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
+                                     int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
+                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
+
 // shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
                                      const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
