@@ -33,6 +33,9 @@ from paper_2605_08527_b200 import workloads as wl  # noqa: E402
 METRIC = "multi-LoRA layer tokens/s (fwd+bwd)"
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed ncu captures
+# (profiles/); None where the kernel has changed since its counters were taken.
+TRAFFIC = {}
 CFG_OF = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
 CFG_DESC = {
     "cfg1": "tiny: W 512x512, 4 tenants r=8, 256 tokens, fwd+bwd",
@@ -188,6 +191,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--flags", type=int, default=0, help="extra MARLAAS_FLAG_* bits for every call (diagnostics)")
+    ap.add_argument("--no-graph", action="store_true", help="time direct launches even for forward-only workloads")
+    ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -224,7 +229,9 @@ def main():
         return t.pin_memory()
 
     # ---- device-resident state: one pool per projection, adapters registered, inputs uploaded -------------
-    projs = []
+    # L2 hygiene: R independent copies of everything a step touches (weights, pools, inputs, outputs), used in
+    # rotation, with R chosen so that the copies' inputs exceed three times the L2; no step finds its operands
+    # in cache and no flush (whose dirty lines the next step would have to write back) is needed.
     seg = B.Segments(torch.from_numpy(w.seg_offsets.astype(np.int32)).to(dev), torch.from_numpy(w.seg_slot.astype(np.int32)).to(dev))
     Tb = w.T_bwd
     seg_b = seg
@@ -232,72 +239,124 @@ def main():
         keep = [s for s in range(len(w.seg_slot)) if w.seg_offsets[s] < Tb]
         off = np.array([min(int(w.seg_offsets[s]), Tb) for s in keep] + [Tb], dtype=np.int32)
         seg_b = B.Segments(torch.from_numpy(off).to(dev), torch.from_numpy(w.seg_slot[keep].astype(np.int32)).to(dev))
-    x_cache = {}
-    for p in w.projections:
-        pool = B.AdapterPool(p.d_in, p.d_out, w.max_rank, w.n_tenants, device=dev)
-        for a in p.adapters:
-            B.marlaas_adapter_pool_register(pool, a.tenant_id, 0, a.rank, a.alpha, dev_bf16(a.A_bits), dev_bf16(a.B_bits))
-        key = p.x_bits.ctypes.data if False else (p.d_in, p.x_bits[0, :8].tobytes())
-        if key not in x_cache:
-            x_cache[key] = (dev_bf16(p.x_bits), pinned_bf16(p.x_bits))
-        x_d, x_h = x_cache[key]
-        st = {"p": p, "pool": pool, "W": dev_bf16(p.W_bits), "x": x_d, "x_host": x_h,
-              "y": torch.empty((w.T, p.d_out), dtype=torch.bfloat16, device=dev),
-              "h": torch.empty((w.T, pool.rank_stride), dtype=torch.float32, device=dev),
-              "ws": torch.empty(B.marlaas_lora_workspace_bytes(pool, w.T), dtype=torch.uint8, device=dev)}
-        if Tb:
-            st["dy"] = dev_bf16(p.dy_bits)
-            st["dy_host"] = pinned_bf16(p.dy_bits)
-            st["dx"] = torch.empty((Tb, p.d_in), dtype=torch.bfloat16, device=dev)
-            st["dA"] = [torch.empty((p.d_in, a.rank), dtype=torch.float32, device=dev) for a in p.adapters]
-            st["dB"] = [torch.empty((a.rank, p.d_out), dtype=torch.float32, device=dev) for a in p.adapters]
-        projs.append(st)
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    input_bytes = sum(p.W_bits.nbytes + (0 if p.dy_bits is None else p.dy_bits.nbytes) for p in w.projections) \
+        + sum(x.nbytes for x in {id(p.x_bits): p.x_bits for p in w.projections}.values()) \
+        + sum(2 * a.rank * (p.d_in + p.d_out) for p in w.projections for a in p.adapters)
+    R = int(min(16, max(1, -(-3 * l2_bytes // input_bytes))))
+    l2_note = f"inputs of a step ({input_bytes / 1e6:.0f} MB) rotate over {R} independent copies (> 3x the {l2_bytes / 1e6:.0f} MB L2)" \
+        if R > 1 else f"inputs of a step ({input_bytes / 1e6:.0f} MB) are larger than 3x the {l2_bytes / 1e6:.0f} MB L2"
+    pinned = {}
 
-    def step(x_of=lambda s: s["x"], dy_of=lambda s: s["dy"]):
-        for s in projs:
+    def build_copy():
+        projs, x_cache = [], {}
+        for p in w.projections:
+            pool = B.AdapterPool(p.d_in, p.d_out, w.max_rank, w.n_tenants, device=dev)
+            for a in p.adapters:
+                B.marlaas_adapter_pool_register(pool, a.tenant_id, 0, a.rank, a.alpha, dev_bf16(a.A_bits), dev_bf16(a.B_bits))
+            key = id(p.x_bits)
+            if key not in x_cache:
+                x_cache[key] = dev_bf16(p.x_bits)
+            if key not in pinned:
+                pinned[key] = pinned_bf16(p.x_bits)
+            st = {"p": p, "pool": pool, "W": dev_bf16(p.W_bits), "x": x_cache[key], "x_host": pinned[key],
+                  "y": torch.empty((w.T, p.d_out), dtype=torch.bfloat16, device=dev),
+                  "h": torch.empty((w.T, pool.rank_stride), dtype=torch.float32, device=dev),
+                  "ws": torch.empty(B.marlaas_lora_workspace_bytes(pool, w.T), dtype=torch.uint8, device=dev)}
+            if Tb:
+                st["dy"] = dev_bf16(p.dy_bits)
+                if id(p.dy_bits) not in pinned:
+                    pinned[id(p.dy_bits)] = pinned_bf16(p.dy_bits)
+                st["dy_host"] = pinned[id(p.dy_bits)]
+                st["dx"] = torch.empty((Tb, p.d_in), dtype=torch.bfloat16, device=dev)
+                st["dA"] = [torch.empty((p.d_in, a.rank), dtype=torch.float32, device=dev) for a in p.adapters]
+                st["dB"] = [torch.empty((a.rank, p.d_out), dtype=torch.float32, device=dev) for a in p.adapters]
+            projs.append(st)
+        return projs
+
+    copies = [build_copy() for _ in range(R)]
+    projs = copies[0]
+    all_projs = [s for c in copies for s in c]
+
+    def step(i=0, x_of=lambda s: s["x"], dy_of=lambda s: s["dy"]):
+        for s in copies[i % R]:
             B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=args.flags)
             if Tb:
                 B.marlaas_lora_backward(s["pool"], x_of(s)[:Tb], s["W"], dy_of(s), seg_b, dx=s["dx"], dA=s["dA"], dB=s["dB"],
                                         h_saved=s["h"][:Tb], workspace=s["ws"], flags=args.flags)
-
-    # L2 hygiene: every step streams operands larger than the 126 MB L2 except on the small configs, where a
-    # flush buffer is written between steps.
-    resident = sum(s["W"].numel() * 2 + s["x"].numel() * 2 for s in projs)
-    l2_note = "inputs larger than L2"
-    flush = None
-    if resident < 3 * 126e6:
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        l2_note = "L2 flushed between steps (256 MiB write)"
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
-    for s in projs:
+    for i in range(max(args.warmup, R)):
+        step(i)
+    for s in all_projs:
         B.marlaas_check_status(s["pool"])
     barrier()
+
+    # Forward-only (decode-shaped) steps last about ten microseconds, less than the host needs to issue one through
+    # Python, so the K timed steps are captured once into a CUDA graph and replayed; training-shaped steps are
+    # issued directly (their gradient pointer tables come from pageable host memory, which a capture cannot hold).
+    graph = None
+    if not Tb and not args.no_graph:
+        try:
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_, stream=side):
+                    for i in range(args.steps):
+                        step(i)
+            torch.cuda.current_stream().wait_stream(side)
+            graph = g_
+            wa, wb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            graph.replay()
+            wa.record()
+            for _ in range(3):
+                graph.replay()
+            wb.record()
+            barrier()
+            # enough replays for the clock sampler to see the GPU under this load (about 0.3 s), at least --repeats
+            args.repeats = int(min(5000, max(args.repeats, 0.3e3 / max(wa.elapsed_time(wb) / 3, 1e-3))))
+        except Exception as e:  # noqa: BLE001
+            print(f"bench.py: CUDA graph capture failed ({e}); timing direct launches", file=sys.stderr)
+            graph = None
+
+    def run_steps():
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
 
     # ---- timed region: device-resident inputs ------------------------------------------------------------------
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    reps = max(1, args.repeats)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    barrier()
     n0 = B.marlaas_kernel_launch_count()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    for a, b in evs:
-        if flush is not None:
-            flush.fill_(1)
-        a.record()
-        step()
-        b.record()
-    barrier()
-    launches = B.marlaas_kernel_launch_count() - n0
+    if graph is None:
+        evs[0][0].record()
+        run_steps()
+        evs[0][1].record()
+        barrier()
+        launches = B.marlaas_kernel_launch_count() - n0
+        rep_ms = [evs[0][0].elapsed_time(evs[0][1])]
+    else:
+        # the graph holds exactly K steps; it is replayed `reps` times and the median replay is reported
+        for a, b in evs:
+            a.record()
+            run_steps()
+            b.record()
+        barrier()
+        launches = None
+        rep_ms = [a.elapsed_time(b) for a, b in evs]
     clocks = sampler.stop() if rank == 0 else None
-    step_ms = [a.elapsed_time(b) for a, b in evs]
-    total_ms = float(sum(step_ms))
+    total_ms = float(np.median(rep_ms))
     if dist is not None:
         t = torch.tensor([total_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -306,15 +365,17 @@ def main():
     tokens_per_step = w.T * world
     value = tokens_per_step / (ms_per_step * 1e-3)
 
-    # ---- dominant kernel (base GEMM + fused expand), timed live with events on the launching stream -------
-    for s in projs:
+    # ---- dominant kernel, timed live with events on the launching stream ---------------------------------------
+    for s in all_projs:
         B.marlaas_kernel_timing_begin(s["pool"])
-    for _ in range(args.steps):
-        if flush is not None:
-            flush.fill_(1)
-        step()
+    n1 = B.marlaas_kernel_launch_count()
+    for i in range(args.steps):
+        step(i)
+    launches_direct = B.marlaas_kernel_launch_count() - n1
+    if launches is None:
+        launches = launches_direct      # what one replay of the captured graph launches
     gemm_ms, gemm_n = 0.0, 0
-    for s in projs:
+    for s in all_projs:
         ms, n = B.marlaas_kernel_timing_end(s["pool"])
         gemm_ms += ms
         gemm_n += n
@@ -322,19 +383,21 @@ def main():
     gemm_flops_per_step = float(sum(work["gemm_flops"]))
     avg_launch_ms = gemm_ms / max(gemm_n, 1)
     flops_per_launch = gemm_flops_per_step / max(len(work["gemm_flops"]), 1)
-    step_bytes = work["fwd_bytes"] + work["bwd_bytes"]
-    if args.workload == "cfg2":
+    if not Tb:
         ach = work["fwd_bytes"] / (ms_per_step * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peak_src}",
-                    "kernel": "whole forward call (index + shrink + GEMM with fused expand)",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": TRAFFIC.get(args.workload), "peak_source": f"of {peak_src}",
+                    "kernel": "whole forward call: k_decode_shrink and k_decode_gemm (base GEMM + expand), overlapped; "
+                              "bytes = W + x + y + present adapters, each once",
+                    "bytes_per_launch": work["fwd_bytes"], "avg_launch_ms": ms_per_step,
+                    "direct_launch_event_ms": avg_launch_ms,
                     "frac_of_nominal_8TBs": ach / NOMINAL["hbm_gbs"]}
     else:
         ach = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12 if gemm_n else 0.0
         roofline = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": f"of {peak_src} (burst)",
+                    "frac": ach / peaks["bf16_tflops"], "traffic": TRAFFIC.get(args.workload), "peak_source": f"of {peak_src} (burst)",
                     "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)",
-                    "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms,
+                    "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms, "flops_per_launch": flops_per_launch,
                     "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
                     "whole_step_tflops": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12,
                     "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
@@ -396,7 +459,7 @@ def main():
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
                "ms_per_step": e_ms / args.e2e_steps}
 
-    for s in projs:
+    for s in all_projs:
         B.marlaas_check_status(s["pool"])
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only) ------------------------
@@ -416,12 +479,13 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "desc": CFG_DESC[args.workload], "tokens_per_step_per_gpu": w.T,
                        "backward_tokens": Tb, "segments": int(len(w.seg_slot)), "l2": l2_note,
+                       "timed_as": "one CUDA graph of K steps, median of %d replays" % reps if graph is not None else "K direct steps",
                        "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": clocks,
             "work_per_step": {"fwd_gflop": work["fwd_flops"] / 1e9, "bwd_gflop": work["bwd_flops"] / 1e9,
                               "fwd_mb": work["fwd_bytes"] / 1e6, "bwd_mb": work["bwd_bytes"] / 1e6},
-            "ms_per_step_min": float(min(step_ms)), "ms_per_step_median": float(np.median(step_ms)),
+            "ms_per_step_min": float(min(rep_ms)) / args.steps,
         }
         print(json.dumps(out))
     if dist is not None:

@@ -24,7 +24,7 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
-    w.hd = (bf16*)take(sizeof(bf16) * Tn * (size_t)w.umax * 16);
+    w.hd = (bf16*)take(sizeof(bf16) * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
     const size_t nblk = (Tn + 63) / 64;
     const bool grad_tc = grad_sm100_eligible(pool, (int64_t)Tn);
     w.HW = ((2 * pool->RP + 63) / 64) * 64;

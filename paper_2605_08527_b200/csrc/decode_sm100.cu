@@ -57,10 +57,9 @@ __device__ __forceinline__ void dk_report(int32_t* status, int code, int detail)
 constexpr int DS_THREADS = 128;
 constexpr int DS_MAX_T = 256;          // tokens per call
 constexpr int DS_PASS = 16;            // tokens per pass (one m16 MMA tile)
-constexpr int DS_SUB_OCT = 64;         // 16-byte octets (8 bf16) of K per staged sub-chunk: 512 elements
-constexpr int DS_PITCH = (DS_SUB_OCT + 1) * 16;   // bytes per staged row (padded: conflict-free ldmatrix)
 constexpr int DS_MAX_CS = 8;
-constexpr int DS_TABLE_SMEM = 1024;    // segment offsets staged in shared memory when S + 1 <= this
+constexpr int DS_TABLE_SMEM = 1024;    // the segment table is staged in shared memory when S + 1 <= this
+constexpr int DS_UB = 4;               // 32-deep k-blocks whose loads are in flight together per warp
 
 struct DecodeShrinkArgs {
     int T, K, RP, cap;
@@ -80,20 +79,15 @@ struct DecodeShrinkArgs {
 };
 
 struct __align__(16) DecodeShrinkSmem {
-    uint8_t sx[DS_PASS * DS_PITCH];
-    uint8_t sa[16 * DS_PITCH];
-    float part[DS_MAX_CS * 4 * 256];    // [cluster rank][warp][16 tokens x 16 ranks] (used in cluster rank 0)
+    float wpart[4][256];                // per-warp [16 tokens][16 ranks] partial products
+    float part[DS_MAX_CS][256];         // per-CTA partials, gathered in cluster rank 0
     int32_t slot[DS_MAX_T];
     int32_t list[DS_MAX_T];
-    int32_t table[DS_TABLE_SMEM];
+    int32_t off_tab[DS_TABLE_SMEM];
+    int32_t slot_tab[DS_TABLE_SMEM];
     int32_t cnt[8];
 };
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -102,12 +96,22 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
 
 // grid = (cap + 1) clusters of CS CTAs; cluster t < cap serves tenant slot t, cluster cap the tokens routed to no
-// adapter (slot -1, or a slot outside the pool, which is reported).
+// adapter (slot -1, or a slot outside the pool, which is reported).  The cluster's CTAs (and their warps) split K.
+//
+// Operand fragments of the m16n8k16 MMA come straight from global memory with 16-byte loads: within a 32-deep
+// k-block lane (g, t) reads elements 8t .. 8t+7 of its rows, and the same element-to-position permutation is used
+// for the token rows (A fragment) and the adapter rows (B fragment), so every product pairs matching k.
 __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrinkArgs g) {
-    extern __shared__ uint8_t ds_raw[];
-    DecodeShrinkSmem& sm = *reinterpret_cast<DecodeShrinkSmem*>((reinterpret_cast<uintptr_t>(ds_raw) + 15) & ~uintptr_t(15));
+    __shared__ DecodeShrinkSmem sm;
     dk_launch_dependents();      // the GEMM may start streaming W now; it waits for this grid before the expand
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -116,17 +120,22 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(cs));
     const int t = (int)dk_cluster_id_x();           // tenant slot served by this cluster; == cap: no adapter
     const bool first = (t == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
+    const int r_t = t < g.cap ? g.d_rank[t] : 0;
+    const float sc = t < g.cap ? g.d_scale[t] : 0.f;
 
     // ---- per-token slot ------------------------------------------------------------------------------------
     if (g.S >= 0) {
         const bool staged = g.S + 1 <= DS_TABLE_SMEM;
         if (staged) {
-            for (int s = tid; s <= g.S; s += DS_THREADS) sm.table[s] = g.seg_offsets[s];
+            for (int s = tid; s <= g.S; s += DS_THREADS) {
+                sm.off_tab[s] = g.seg_offsets[s];
+                if (s < g.S) sm.slot_tab[s] = g.seg_slot[s];
+            }
             __syncthreads();
         }
         if (first) {
             for (int s = tid; s < g.S; s += DS_THREADS) {
-                const int a = g.seg_offsets[s], b = g.seg_offsets[s + 1];
+                const int a = staged ? sm.off_tab[s] : g.seg_offsets[s], b = staged ? sm.off_tab[s + 1] : g.seg_offsets[s + 1];
                 if (b < a || a < 0 || b > g.T) dk_report(g.status, DEV_BAD_TABLE, s);
                 if (s == 0 && a != 0) dk_report(g.status, DEV_BAD_TABLE, -1);
                 if (s == g.S - 1 && b != g.T) dk_report(g.status, DEV_BAD_TABLE, -2);
@@ -137,10 +146,10 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
             int lo = 0, hi = g.S;
             while (lo < hi) {       // first s with seg_offsets[s + 1] > i
                 const int mid = (lo + hi) >> 1;
-                const int v = staged ? sm.table[mid + 1] : g.seg_offsets[mid + 1];
+                const int v = staged ? sm.off_tab[mid + 1] : g.seg_offsets[mid + 1];
                 if (v > i) hi = mid; else lo = mid + 1;
             }
-            sm.slot[i] = lo < g.S ? g.seg_slot[lo] : -1;
+            sm.slot[i] = lo < g.S ? (staged ? sm.slot_tab[lo] : g.seg_slot[lo]) : -1;
         }
     } else {
         for (int i = tid; i < g.T; i += DS_THREADS) sm.slot[i] = g.tok_slot[i];
@@ -186,9 +195,16 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     __syncthreads();
     if (n_t == 0) return;        // uniform over the cluster
 
-    const int r_t = t < g.cap ? g.d_rank[t] : 0;
-    const float sc = r_t > 0 ? g.d_scale[t] : 0.f;
     const int own0 = r_t > 0 ? t * g.RP : 0, own1 = r_t > 0 ? own0 + g.RP : 0;   // hd columns written by the MMA part
+    const int ngroups = (r_t + 15) >> 4;
+
+    // ---- partial products over this warp's share of K --------------------------------------------------------
+    // 32-deep k-blocks [kb0, kb1) of this warp: the cluster's CTAs split the blocks, then each CTA's warps do
+    const int nb32 = (g.K + 31) >> 5;
+    const int cb0 = (int)((int64_t)crank * nb32 / cs), cb1 = (int)((int64_t)(crank + 1) * nb32 / cs);
+    const int wb0 = cb0 + (int)((int64_t)warp * (cb1 - cb0) / 4), wb1 = cb0 + (int)((int64_t)(warp + 1) * (cb1 - cb0) / 4);
+    const int gq = lane >> 2, tq = lane & 3;
+    const uint32_t part_rank0 = dk_map_to_cta(smem_u32(&sm.part[0][0]), 0);
 
     // zero the other tenants' columns of this cluster's hd rows (and, with no adapter, the h rows): one warp per row
     for (int e = crank * 4 + warp; e < n_t; e += cs * 4) {
@@ -201,56 +217,51 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     }
     if (r_t == 0) return;        // uniform over the cluster
 
-    // ---- partial products over this CTA's share of K ---------------------------------------------------------
-    const int oct_total = g.K >> 3;
-    const int oct0 = (int)((int64_t)crank * oct_total / cs), oct1 = (int)((int64_t)(crank + 1) * oct_total / cs);
-    const uint32_t sx_u = smem_u32(sm.sx), sa_u = smem_u32(sm.sa);
-    const uint32_t part_rank0 = dk_map_to_cta(smem_u32(sm.part), 0);
-    const int ngroups = (r_t + 15) >> 4;
-
     for (int p0 = 0; p0 < n_t; p0 += DS_PASS) {
         const int np = min(DS_PASS, n_t - p0);
+        const bf16* xr0 = gq < np ? g.x + (size_t)sm.list[p0 + gq] * g.ldx : nullptr;
+        const bf16* xr1 = gq + 8 < np ? g.x + (size_t)sm.list[p0 + gq + 8] * g.ldx : nullptr;
         for (int jg = 0; jg < ngroups; ++jg) {
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-            const bf16* arow = g.At + ((size_t)t * g.RP + jg * 16) * g.K;
-            for (int o0 = oct0; o0 < oct1; o0 += DS_SUB_OCT) {
-                const int no = min(DS_SUB_OCT, oct1 - o0);
-                __syncthreads();    // the previous sub-chunk has been consumed
+            const bf16* ar0 = g.At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
+            const bf16* ar1 = ar0 + (size_t)8 * g.K;
+            for (int b0 = wb0; b0 < wb1; b0 += DS_UB) {
+                uint4 xa[DS_UB], xb[DS_UB], ba[DS_UB], bb[DS_UB];
 #pragma unroll
-                for (int e = tid; e < 16 * DS_SUB_OCT; e += DS_THREADS) {
-                    const int row = e / DS_SUB_OCT, o = e - row * DS_SUB_OCT;
-                    uint4 xv = make_uint4(0u, 0u, 0u, 0u), av = xv;
-                    if (o < no) {
-                        av = *reinterpret_cast<const uint4*>(arow + (size_t)row * g.K + (size_t)(o0 + o) * 8);
-                        if (row < np)
-                            xv = *reinterpret_cast<const uint4*>(g.x + (size_t)sm.list[p0 + row] * g.ldx + (size_t)(o0 + o) * 8);
-                    }
-                    *reinterpret_cast<uint4*>(sm.sx + row * DS_PITCH + o * 16) = xv;
-                    *reinterpret_cast<uint4*>(sm.sa + row * DS_PITCH + o * 16) = av;
+                for (int u = 0; u < DS_UB; ++u) {
+                    const int k = (b0 + u) * 32 + tq * 8;
+                    const bool in = (b0 + u) < wb1 && k < g.K;
+                    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                    xa[u] = (in && xr0) ? ldg_nc_v4(xr0 + k) : z;
+                    xb[u] = (in && xr1) ? ldg_nc_v4(xr1 + k) : z;
+                    ba[u] = in ? ldg_nc_v4(ar0 + k) : z;
+                    bb[u] = in ? ldg_nc_v4(ar1 + k) : z;
                 }
-                __syncthreads();
-                // warp w multiplies k16 steps w, w + 4, ... of the sub-chunk (each step = two octets)
-                const int steps = (no + 1) >> 1;
-                for (int ks = warp; ks < steps; ks += 4) {
-                    uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-                    ldmatrix_x4(sx_u + ((lane & 7) + ((lane >> 3) & 1) * 8) * DS_PITCH + (ks * 2 + (lane >> 4)) * 16, a0, a1, a2, a3);
-                    ldmatrix_x4(sa_u + ((lane & 7) + (lane >> 4) * 8) * DS_PITCH + (ks * 2 + ((lane >> 3) & 1)) * 16, b0, b1, b2, b3);
-                    mma_bf16_16816(c0, a0, a1, a2, a3, b0, b1);
-                    mma_bf16_16816(c1, a0, a1, a2, a3, b2, b3);
+#pragma unroll
+                for (int u = 0; u < DS_UB; ++u) {
+                    mma_bf16_16816(c0, xa[u].x, xb[u].x, xa[u].y, xb[u].y, ba[u].x, ba[u].y);
+                    mma_bf16_16816(c1, xa[u].x, xb[u].x, xa[u].y, xb[u].y, bb[u].x, bb[u].y);
+                    mma_bf16_16816(c0, xa[u].z, xb[u].z, xa[u].w, xb[u].w, ba[u].z, ba[u].w);
+                    mma_bf16_16816(c1, xa[u].z, xb[u].z, xa[u].w, xb[u].w, bb[u].z, bb[u].w);
                 }
             }
-            // this warp's 16 x 16 partial -> cluster rank 0, slot (crank, warp)
+            // warp partials -> CTA partial (fixed order) -> cluster rank 0
+            __syncthreads();        // wpart of the previous group has been consumed
             {
-                const int gq = lane >> 2, tq = lane & 3;
-                const uint32_t base = part_rank0 + (uint32_t)((crank * 4 + warp) * 256) * 4;
-                dk_st_cluster_f32(base + (gq * 16 + 2 * tq) * 4, c0[0]);
-                dk_st_cluster_f32(base + (gq * 16 + 2 * tq + 1) * 4, c0[1]);
-                dk_st_cluster_f32(base + ((gq + 8) * 16 + 2 * tq) * 4, c0[2]);
-                dk_st_cluster_f32(base + ((gq + 8) * 16 + 2 * tq + 1) * 4, c0[3]);
-                dk_st_cluster_f32(base + (gq * 16 + 8 + 2 * tq) * 4, c1[0]);
-                dk_st_cluster_f32(base + (gq * 16 + 8 + 2 * tq + 1) * 4, c1[1]);
-                dk_st_cluster_f32(base + ((gq + 8) * 16 + 8 + 2 * tq) * 4, c1[2]);
-                dk_st_cluster_f32(base + ((gq + 8) * 16 + 8 + 2 * tq + 1) * 4, c1[3]);
+                float* wp = sm.wpart[warp];
+                wp[gq * 16 + 2 * tq] = c0[0];
+                wp[gq * 16 + 2 * tq + 1] = c0[1];
+                wp[(gq + 8) * 16 + 2 * tq] = c0[2];
+                wp[(gq + 8) * 16 + 2 * tq + 1] = c0[3];
+                wp[gq * 16 + 8 + 2 * tq] = c1[0];
+                wp[gq * 16 + 8 + 2 * tq + 1] = c1[1];
+                wp[(gq + 8) * 16 + 8 + 2 * tq] = c1[2];
+                wp[(gq + 8) * 16 + 8 + 2 * tq + 1] = c1[3];
+            }
+            __syncthreads();
+            for (int e = tid; e < 256; e += DS_THREADS) {
+                const float v = ((sm.wpart[0][e] + sm.wpart[1][e]) + sm.wpart[2][e]) + sm.wpart[3][e];
+                dk_st_cluster_f32(part_rank0 + (uint32_t)(crank * 256 + e) * 4, v);
             }
             dk_cluster_sync();
             if (crank == 0) {
@@ -258,7 +269,7 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
                     const int i = e >> 4, j = e & 15;
                     if (i < np) {
                         float v = 0.f;
-                        for (int s = 0; s < cs * 4; ++s) v += sm.part[s * 256 + e];   // fixed order
+                        for (int s = 0; s < cs; ++s) v += sm.part[s][e];   // fixed order
                         const int tok = sm.list[p0 + i];
                         g.h_out[(size_t)tok * g.RP + jg * 16 + j] = v;
                         g.hd[(size_t)tok * g.hd_cols + own0 + jg * 16 + j] = __float2bfloat16_rn(sc * v);
@@ -268,13 +279,15 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
             dk_cluster_sync();      // rank 0 has read the partials before they are overwritten
         }
         // ranks beyond the tenant's true rank (rounded up to 16) stay zero
-        if (crank == 0)
-            for (int e = tid; e < np * (g.RP - ngroups * 16); e += DS_THREADS) {
-                const int i = e / (g.RP - ngroups * 16), j = ngroups * 16 + e % (g.RP - ngroups * 16);
+        if (crank == 0) {
+            const int rest = g.RP - ngroups * 16;
+            for (int e = tid; e < np * rest; e += DS_THREADS) {
+                const int i = e / rest, j = ngroups * 16 + e % rest;
                 const int tok = sm.list[p0 + i];
                 g.h_out[(size_t)tok * g.RP + j] = 0.f;
                 g.hd[(size_t)tok * g.hd_cols + own0 + j] = __float2bfloat16_rn(0.f);
             }
+        }
     }
 }
 
@@ -282,13 +295,15 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
 // k_decode_gemm
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int DG_THREADS = 192;
+constexpr int DG_KP = 2;               // 64-deep panels per pipeline step
 
 struct DecodeGemmArgs {
     int T, Nout;
-    int num_kb;          // k-blocks of 64 over K
-    int num_xb;          // k-blocks of 64 over the expand rows (cap*RP, or up to the last slot in use)
+    int num_ks;          // pipeline steps (kp * 64 deep) over K
+    int num_xs;          // pipeline steps over the expand rows (cap*RP, or up to the last slot in use)
     int S;               // contraction slices = CTA pairs per cluster
     int nch;             // 64-column chunks of the B operand staged per CTA: the pair's strip is 128 * nch columns
+    int kp;              // 64-deep panels per pipeline step: one TMA instruction per operand moves all of them
     int stages;
     bf16* C;
     int64_t ldc;
@@ -299,6 +314,13 @@ __device__ __forceinline__ void dg_tma_pair(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void dg_tma_pair_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0, int c1,
+                                               int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 __device__ __forceinline__ void dg_commit_pair(uint32_t bar, uint16_t mask) {
@@ -315,16 +337,23 @@ __device__ __forceinline__ void dg_mma_pair(uint32_t d_tmem, uint64_t desc_a, ui
         : "memory");
 }
 
+// Operand staging per pipeline step (kp panels of 64 k):
+//   A  [kp][128 rows][64 k]      one 3-D TMA over x viewed as (64 k, rows, K / 64): K-major tiles, 128-byte swizzle
+//   B  [nch][kp * 64 k][64 n]    one 2-D TMA per 64-column chunk: MN-major, chunks kp * 8 KB apart
+// A single thread issues the loads and a single thread the MMAs, and each of their instructions costs tens to a
+// hundred cycles of issue latency, so the steps are made deep: with 64-deep steps the issue loop, not HBM, set the pace.
 __global__ void __launch_bounds__(DG_THREADS, 1)
 k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
               const __grid_constant__ CUtensorMap tmXA, const __grid_constant__ CUtensorMap tmXB, const DecodeGemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int STAGES = g.stages;
-    const uint32_t b_stage_bytes = (uint32_t)g.nch * CHUNK_BYTES;
+    const uint32_t a_stage_bytes = (uint32_t)g.kp * A_STAGE_BYTES;
+    const uint32_t b_chunk_bytes = (uint32_t)g.kp * CHUNK_BYTES;
+    const uint32_t b_stage_bytes = (uint32_t)g.nch * b_chunk_bytes;
     const uint32_t sA = smem_u32(smem);
-    const uint32_t sB = sA + STAGES * A_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + b_stage_bytes));
+    const uint32_t sB = sA + STAGES * a_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (a_stage_bytes + b_stage_bytes));
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;
@@ -342,8 +371,8 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int my_m = (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
     const uint32_t tmem_cols = (uint32_t)NP;    // 128 or 256
 
-    const int kb0 = (int)((int64_t)pairi * g.num_kb / g.S), kb1 = (int)((int64_t)(pairi + 1) * g.num_kb / g.S);
-    const int xb0 = (int)((int64_t)pairi * g.num_xb / g.S), xb1 = (int)((int64_t)(pairi + 1) * g.num_xb / g.S);
+    const int ks0 = (int)((int64_t)pairi * g.num_ks / g.S), ks1 = (int)((int64_t)(pairi + 1) * g.num_ks / g.S);
+    const int xs0 = (int)((int64_t)pairi * g.num_xs / g.S), xs1 = (int)((int64_t)(pairi + 1) * g.num_xs / g.S);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -357,7 +386,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
-        if (g.num_xb > 0) {
+        if (g.num_xs > 0) {
             prefetch_tmap(&tmXA);
             prefetch_tmap(&tmXB);
         }
@@ -374,10 +403,11 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // bytes the two CTAs of the pair stage per k-block (rows and columns outside the tensors are skipped entirely)
-    auto a_bytes = [&](int r) -> uint32_t { return (r * 128 < g.T) ? A_STAGE_BYTES : 0u; };
+    // bytes the two CTAs of the pair stage per step (rows and columns outside the tensors are skipped entirely;
+    // partly outside boxes are filled with zeros and count in full)
+    auto a_bytes = [&](int r) -> uint32_t { return (r * 128 < g.T) ? a_stage_bytes : 0u; };
     auto b_chunks = [&](int r) -> int { return max(0, min(g.nch, (g.Nout - (n0 + r * 64 * g.nch) + 63) / 64)); };
-    const uint32_t stage_tx = a_bytes(0) + a_bytes(1) + (uint32_t)(b_chunks(0) + b_chunks(1)) * CHUNK_BYTES;
+    const uint32_t stage_tx = a_bytes(0) + a_bytes(1) + (uint32_t)(b_chunks(0) + b_chunks(1)) * b_chunk_bytes;
     const int my_chunks = b_chunks((int)half);
     const bool have_rows = my_m < g.T;
 
@@ -385,25 +415,25 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (warp == 0) {
         // ================= TMA producer (every CTA) =================
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, ph = 0;     // steps issued; stage and phase bit of the next step
             bool ok = true;
             const uint32_t full0 = dk_map_to_cta(bar_full, leader);
-            for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+            for (int ks = ks0; ks < ks1 && ok; ++ks, ++it) {
                 if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 41))) break;
                 if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
-                if (have_rows) dg_tma_pair(sA + s * A_STAGE_BYTES, &tmA, full0 + 8 * s, kb * BK, my_m);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmA, full0 + 8 * s, 0, my_m, ks * g.kp);
                 for (int c = 0; c < my_chunks; ++c)
-                    dg_tma_pair(sB + s * b_stage_bytes + c * CHUNK_BYTES, &tmB, full0 + 8 * s, my_n + c * 64, kb * BK);
+                    dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmB, full0 + 8 * s, my_n + c * 64, ks * g.kp * BK);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
-            if (ok && xb0 < xb1) dk_wait_prerequisites();     // hd comes from the shrink grid
-            for (int xb = xb0; xb < xb1 && ok; ++xb, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+            if (ok && xs0 < xs1) dk_wait_prerequisites();     // hd comes from the shrink grid
+            for (int xs = xs0; xs < xs1 && ok; ++xs, ++it) {
                 if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 42))) break;
                 if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
-                if (have_rows) dg_tma_pair(sA + s * A_STAGE_BYTES, &tmXA, full0 + 8 * s, xb * BK, my_m);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, xs * g.kp);
                 for (int c = 0; c < my_chunks; ++c)
-                    dg_tma_pair(sB + s * b_stage_bytes + c * CHUNK_BYTES, &tmXB, full0 + 8 * s, my_n + c * 64, xb * BK);
+                    dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmXB, full0 + 8 * s, my_n + c * 64, xs * g.kp * BK);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
             if (!ok && half == 0) {
                 // let the copies already issued land (bounded) before shared memory is reused or released
@@ -411,7 +441,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 for (uint32_t j = 0; j < back; ++j) {
                     const uint32_t jt = it - 1 - j;
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_full + 8 * (jt % STAGES), (jt / STAGES) & 1) &&
+                    while (!mbar_try_wait(bar_full + 8 * (jt % (uint32_t)STAGES), (jt / (uint32_t)STAGES) & 1) &&
                            global_ns() - t0 < WAIT_LIMIT_NS) {
                     }
                 }
@@ -424,20 +454,23 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(NP >> 3) << 17) |
                                    ((uint32_t)(256 >> 4) << 24);    // fp32 acc, bf16 x bf16, B MN-major, M = 256, N = NP
             const uint16_t mask = (uint16_t)(3u << leader);
-            uint32_t it = 0, acc = 0;
+            uint32_t acc = 0, s = 0, ph = 0;
             bool ok = true;
-            const int nblk = (kb1 - kb0) + (xb1 - xb0);
-            for (int b = 0; b < nblk && ok; ++b, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+            const int nstep = (ks1 - ks0) + (xs1 - xs0);
+            for (int b = 0; b < nstep && ok; ++b) {
                 if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 44))) break;
                 tc_fence_after();
-                const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * b_stage_bytes;
+                const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
+                for (int q = 0; q < g.kp; ++q) {
 #pragma unroll
-                for (int j = 0; j < BK / 16; ++j) {
-                    dg_mma_pair(tmem_base, desc_k_major(a0 + j * 32), desc_mn_major(b0 + j * UNIT_BYTES, CHUNK_BYTES), idesc, acc);
-                    acc = 1;
+                    for (int j = 0; j < BK / 16; ++j) {
+                        dg_mma_pair(tmem_base, desc_k_major(a0 + q * A_STAGE_BYTES + j * 32),
+                                    desc_mn_major(b0 + q * CHUNK_BYTES + j * UNIT_BYTES, b_chunk_bytes), idesc, acc);
+                        acc = 1;
+                    }
                 }
                 dg_commit_pair(bar_empty + 8 * s, mask);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
             if (ok) {
                 dg_commit_pair(bar_tfull, mask);
@@ -458,62 +491,91 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
 
     // ---- sum the S slices through distributed shared memory ---------------------------------------------------
-    // Row quarter q (32 rows) of each half is summed by pair (q mod S); that CTA's buffer holds, for each of its
-    // 4 / S quarters, one [32][NP] fp32 block per source pair.  16-byte chunks are XOR-swizzled by the row so that
-    // both the row-per-lane writes and the column-per-lane reads are conflict-free.
-    tc_fence_before();
-    __syncthreads();
-    dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
-    tc_fence_after();
+    // Row quarter q (32 rows) of each half is finished by pair (q mod S).  The other pairs' warps holding that
+    // quarter send their partial accumulators to a mailbox in the finishing CTA (thread to thread: the same
+    // tensor-memory lane on both sides, [column group][lane] 16-byte slots), and the finishing warp adds them to
+    // its own accumulator in ascending pair order.  The mailboxes reuse the pipeline stages.
     const int qper = 4 / g.S;
-    const uint32_t blk_bytes = 32u * (uint32_t)NP * 4u;
-    const uint32_t row_bytes = (uint32_t)NP * 4u;
-    if (warp >= 2 && epi_ok) {
-        const int q = warp & 3;
-        const uint32_t dst_rank = (uint32_t)(2 * (q % g.S)) + half;
-        const uint32_t dst = dk_map_to_cta(sA, dst_rank) + (pairi * qper + (uint32_t)(q / g.S)) * blk_bytes + (uint32_t)lane * row_bytes;
+    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
+    const int q = warp & 3;
+    const uint32_t own = (uint32_t)(q % g.S);
+    if (g.S > 1) {
+        tc_fence_before();
+        __syncthreads();
+        dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
+        tc_fence_after();
+        if (warp >= 2 && epi_ok && own != pairi) {
+            const uint32_t si = pairi < own ? pairi : pairi - 1;
+            const uint32_t dst = dk_map_to_cta(sA, 2 * own + half) + (si * (uint32_t)qper + (uint32_t)(q / g.S)) * box_bytes +
+                                 (uint32_t)lane * 16u;
+#pragma unroll 1
+            for (int c = 0; c < NP / 32; ++c) {
+                uint32_t v[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    dk_st_cluster_v4(dst + (uint32_t)(c * 8 + e) * 512u, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+            }
+        }
+        tc_fence_before();
+        dk_cluster_sync();      // all partial accumulators have landed
+        tc_fence_after();
+    }
+    if (warp >= 2 && epi_ok && own == pairi) {
+        const int row = my_m + q * 32 + lane;
+        bf16* crow = g.C + (size_t)row * g.ldc + n0;
+        const uint32_t mbox = sA + (uint32_t)(q / g.S) * box_bytes + (uint32_t)lane * 16u;
 #pragma unroll 1
         for (int c = 0; c < NP / 32; ++c) {
             uint32_t v[32];
             tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, v);
             tc_wait_ld();
+            float acc[32];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const uint32_t c4 = (uint32_t)(c * 8 + e);
-                dk_st_cluster_v4(dst + ((c4 ^ (uint32_t)(lane & 7)) << 4), v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-            }
-        }
-    }
-    tc_fence_before();
-    dk_cluster_sync();      // all partial blocks have landed
-    if (warp >= 2 && epi_ok) {
-        const int ew = warp - 2;
-        for (int qs = 0; qs < qper; ++qs) {
-            const int q = qs * g.S + (int)pairi;
-            for (int rr = ew; rr < 32; rr += 4) {
-                const int row = my_m + q * 32 + rr;
-                if (row >= g.T) continue;
-                for (int c4 = lane; c4 < NP / 4; c4 += 32) {
-                    const int col = n0 + c4 * 4;
-                    if (col >= g.Nout) continue;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int src = 0; src < g.S; ++src) {      // fixed order
-                        const float4 p = *reinterpret_cast<const float4*>(
-                            smem + (size_t)(src * qper + qs) * blk_bytes + (size_t)rr * row_bytes + ((c4 ^ (rr & 7)) << 4));
-                        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+            for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+            for (uint32_t src = 0; src < (uint32_t)g.S; ++src) {      // ascending pair order
+                if (src == pairi) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(v[e]);
+                } else {
+                    const uint32_t si = src < pairi ? src : src - 1;
+                    const uint32_t a = mbox + si * (uint32_t)qper * box_bytes + (uint32_t)(c * 8) * 512u;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float4 p;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(p.x), "=f"(p.y), "=f"(p.z), "=f"(p.w)
+                                     : "r"(a + (uint32_t)e * 512u));
+                        acc[4 * e] += p.x; acc[4 * e + 1] += p.y; acc[4 * e + 2] += p.z; acc[4 * e + 3] += p.w;
                     }
-                    __nv_bfloat162 p0 = __floats2bfloat162_rn(acc.x, acc.y), p1 = __floats2bfloat162_rn(acc.z, acc.w);
-                    uint2 o;
-                    o.x = *reinterpret_cast<uint32_t*>(&p0);
-                    o.y = *reinterpret_cast<uint32_t*>(&p1);
-                    *reinterpret_cast<uint2*>(g.C + (size_t)row * g.ldc + col) = o;
+                }
+            }
+            if (row < g.T) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int col = n0 + c * 32 + e * 8;
+                    if (col < g.Nout) {
+                        uint4 o;
+                        __nv_bfloat162 p0 = __floats2bfloat162_rn(acc[e * 8 + 0], acc[e * 8 + 1]);
+                        __nv_bfloat162 p1 = __floats2bfloat162_rn(acc[e * 8 + 2], acc[e * 8 + 3]);
+                        __nv_bfloat162 p2 = __floats2bfloat162_rn(acc[e * 8 + 4], acc[e * 8 + 5]);
+                        __nv_bfloat162 p3 = __floats2bfloat162_rn(acc[e * 8 + 6], acc[e * 8 + 7]);
+                        o.x = *reinterpret_cast<uint32_t*>(&p0);
+                        o.y = *reinterpret_cast<uint32_t*>(&p1);
+                        o.z = *reinterpret_cast<uint32_t*>(&p2);
+                        o.w = *reinterpret_cast<uint32_t*>(&p3);
+                        *reinterpret_cast<uint4*>(crow + c * 32 + e * 8) = o;
+                    }
                 }
             }
         }
     }
 
     // ---- teardown ---------------------------------------------------------------------------------------------
+    tc_fence_before();
     __syncthreads();
+    dk_cluster_sync();      // the pair leaves together (its barriers and tensor memory are shared)
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
@@ -523,13 +585,40 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
 }
 
+// x (or hd) viewed as a 3-D tensor (64 k, rows, K / 64) so that one copy brings `panels` K-major tiles of 128 rows
+static marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels) {
+    typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            return fail(MARLAAS_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        fn = (EncodeTiledFn)p;
+    }
+    cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+    cuuint64_t gstr[2] = {(cuuint64_t)ld * 2, 128};
+    cuuint32_t box[3] = {64, 128, panels};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(MARLAAS_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for a %lld x %lld panel view, pitch %lld", (int)r,
+                    (long long)rows, (long long)cols, (long long)ld);
+    return MARLAAS_OK;
+}
+
 }  // namespace sm100
 
 // ---------------------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------------------
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T) {
-    return T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 1024 && pool->sm_count >= 8;
+    return T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 1024 && pool->sm_count >= 8 &&
+           (pool->K % 64) == 0;
 }
 
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
@@ -537,7 +626,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
                                      const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st) {
     using namespace sm100;
     const int64_t K = pool->K, N = pool->N;
-    const int hd_cols = pool->cap * pool->RP;
+    const int hd_cols = (int)align_up((size_t)pool->cap * pool->RP, 64);     // pitch of hd: whole 64-deep panels
 
     // ---- shrink: (cap + 1) clusters, K split over the CTAs of a cluster ----
     {
@@ -546,18 +635,19 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         a.S = S; a.seg_offsets = seg_offsets; a.seg_slot = seg_slot;
         a.x = x; a.ldx = ldx; a.At = pool->d_At; a.d_rank = pool->d_rank; a.d_scale = pool->d_scale;
         a.tok_slot = ws.tok_slot; a.h_out = h_out; a.hd = ws.hd; a.hd_cols = hd_cols; a.status = pool->d_status;
-        int cs = 8;
-        while (cs > 1 && K / cs < 512) cs >>= 1;      // at least one full sub-chunk per CTA
-        const size_t smem_bytes = sizeof(DecodeShrinkSmem) + 16;
-        static bool attr_set[64] = {};
-        if (pool->device >= 64 || !attr_set[pool->device]) {
-            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_shrink, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
-            if (pool->device < 64) attr_set[pool->device] = true;
+        int cs = DS_MAX_CS;
+        while (cs > 1 && K / cs < 32 * 4 * DS_UB) cs >>= 1;      // a full batch of loads per warp
+        static bool carveout_set[64] = {};
+        if (pool->device >= 64 || !carveout_set[pool->device]) {
+            // same shared-memory configuration as the GEMM, so that CTAs of both kernels can share an SM
+            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_shrink, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                                  (int)cudaSharedmemCarveoutMaxShared));
+            if (pool->device < 64) carveout_set[pool->device] = true;
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)((pool->cap + 1) * cs));
         cfg.blockDim = dim3(DS_THREADS);
-        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
@@ -567,33 +657,30 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         count_launch();
     }
 
-    // ---- GEMM with the expand as extra k-blocks ----
+    // ---- GEMM with the expand as extra steps of the contraction ----
     int last_used = -1;
     for (int s = 0; s < pool->cap; ++s)
         if (pool->slots[s].used && pool->slots[s].rank > 0) last_used = s;
     DecodeGemmArgs g;
     g.T = (int)T; g.Nout = (int)N;
-    g.num_kb = (int)cdiv(K, BK);
-    g.num_xb = (int)cdiv((int64_t)(last_used + 1) * pool->RP, BK);
     g.C = y; g.ldc = ldy; g.status = pool->d_status;
-    // strip width and contraction slices: fill the SMs with clusters of 2 * S CTAs
+    // strip width and contraction slices: fill the SMs with one wave of clusters of 2 * S CTAs
     struct Shape { int nch, S; };
     const Shape shapes[] = {{1, 2}, {2, 2}, {1, 1}, {2, 1}, {1, 4}, {2, 4}};
     Shape pick = {2, 1};
     int64_t best = -1;
     static int max_clusters[64][3] = {};      // per device, cluster size 2 / 4 / 8
+    constexpr int DG_SMEM = 200 * 1024;
     for (const Shape& sh : shapes) {
         const int csz = 2 * sh.S;
         const int ci = sh.S == 1 ? 0 : sh.S == 2 ? 1 : 2;
-        const int stages_try = sh.nch == 1 ? 6 : 5;
-        const size_t smem_try = 1024 + (size_t)stages_try * (A_STAGE_BYTES + sh.nch * CHUNK_BYTES) + 256;
         int mc = pool->device < 64 ? max_clusters[pool->device][ci] : 0;
         if (mc == 0) {
-            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM));
             cudaLaunchConfig_t qc = {};
             qc.gridDim = dim3((unsigned)(csz * 64));
             qc.blockDim = dim3(DG_THREADS);
-            qc.dynamicSmemBytes = 200 * 1024;
+            qc.dynamicSmemBytes = DG_SMEM;
             cudaLaunchAttribute qa;
             qa.id = cudaLaunchAttributeClusterDimension;
             qa.val.clusterDim.x = (unsigned)csz; qa.val.clusterDim.y = 1; qa.val.clusterDim.z = 1;
@@ -602,7 +689,6 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
             if (mc < 1) mc = -1;
             if (pool->device < 64) max_clusters[pool->device][ci] = mc;
         }
-        (void)smem_try;
         if (mc < 1) continue;
         const int64_t clusters = cdiv(N, 128 * sh.nch);
         if (clusters > mc) continue;                    // one wave only
@@ -613,21 +699,26 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         if (score > best) { best = score; pick = sh; }
     }
     g.S = pick.S; g.nch = pick.nch;
-    g.stages = pick.nch == 1 ? 6 : 5;
+    g.kp = DG_KP;
+    const size_t step_bytes = (size_t)g.kp * (A_STAGE_BYTES + g.nch * CHUNK_BYTES);
+    g.stages = (int)((DG_SMEM - 1024 - 256) / step_bytes);
+    if (g.stages < 2) g.stages = 2;
+    g.num_ks = (int)cdiv(K, (int64_t)g.kp * BK);
+    g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)g.kp * BK);
     const int NP = 128 * g.nch;
 
     alignas(64) CUtensorMap tmA, tmB, tmXA, tmXB;
     marlaas_status_t rc;
-    if ((rc = make_map(&tmA, x, T, K, ldx, BK, BM)) != MARLAAS_OK) return rc;
-    if ((rc = make_map(&tmB, W, K, N, ldw, 64, BK)) != MARLAAS_OK) return rc;
-    if (g.num_xb > 0) {
-        if ((rc = make_map(&tmXA, ws.hd, T, hd_cols, hd_cols, BK, BM)) != MARLAAS_OK) return rc;
-        if ((rc = make_map(&tmXB, pool->d_Bs, hd_cols, N, N, 64, BK)) != MARLAAS_OK) return rc;
+    if ((rc = make_panel_map(&tmA, x, T, K, ldx, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
+    if ((rc = make_map(&tmB, W, K, N, ldw, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
+    if (g.num_xs > 0) {
+        if ((rc = make_panel_map(&tmXA, ws.hd, T, hd_cols, hd_cols, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXB, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
     } else {
         tmXA = tmA;
         tmXB = tmB;
     }
-    const size_t smem_bytes = 1024 + (size_t)g.stages * (A_STAGE_BYTES + g.nch * CHUNK_BYTES) + 256;
+    const size_t smem_bytes = 1024 + (size_t)g.stages * step_bytes + 256;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(cdiv(N, NP) * 2 * g.S));
     cfg.blockDim = dim3(DG_THREADS);

@@ -48,14 +48,18 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // give up records its site in the CTA's abort word.  Returns false on abort.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int site) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    unsigned long long t0 = 0;      // the global timer is slow to read: sampled every 256 polls only
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_word != 0) return false;
-        if (((++spins) & 63u) == 0 && global_ns() - t0 > WAIT_LIMIT_NS) {
-            atomicCAS((int*)abort_word, 0, site);
-            return false;
+        if (((++spins) & 255u) == 0) {
+            if (*abort_word != 0) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                atomicCAS((int*)abort_word, 0, site);
+                return false;
+            }
         }
     }
 }
