@@ -496,6 +496,10 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     // tensor-memory lane on both sides, [column group][lane] 16-byte slots), and the finishing warp adds them to
     // its own accumulator in ascending pair order.  The mailboxes reuse the pipeline stages.
     const int qper = 4 / g.S;
+    auto slice_steps = [&](uint32_t p) -> int {
+        return (int)((int64_t)(p + 1) * g.num_ks / g.S) - (int)((int64_t)p * g.num_ks / g.S) +
+               (int)((int64_t)(p + 1) * g.num_xs / g.S) - (int)((int64_t)p * g.num_xs / g.S);
+    };
     const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     const int q = warp & 3;
     const uint32_t own = (uint32_t)(q % g.S);
@@ -504,7 +508,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         __syncthreads();
         dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
         tc_fence_after();
-        if (warp >= 2 && epi_ok && own != pairi) {
+        if (warp >= 2 && epi_ok && own != pairi && slice_steps(pairi) > 0) {
             const uint32_t si = pairi < own ? pairi : pairi - 1;
             const uint32_t dst = dk_map_to_cta(sA, 2 * own + half) + (si * (uint32_t)qper + (uint32_t)(q / g.S)) * box_bytes +
                                  (uint32_t)lane * 16u;
@@ -535,6 +539,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] = 0.f;
             for (uint32_t src = 0; src < (uint32_t)g.S; ++src) {      // ascending pair order
+                if (slice_steps(src) == 0) continue;                  // a slice without steps never wrote its accumulator
                 if (src == pairi) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(v[e]);
@@ -692,7 +697,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         if (mc < 1) continue;
         const int64_t clusters = cdiv(N, 128 * sh.nch);
         if (clusters > mc) continue;                    // one wave only
-        if (cdiv(K, BK) < sh.S) continue;
+        if (cdiv(K, (int64_t)DG_KP * BK) < sh.S) continue;     // every slice needs at least one step
         const int64_t ctas = clusters * csz;
         // more CTAs streaming is better; among equals prefer fewer slices and wider strips (less re-read of x)
         const int64_t score = ctas * 16 - sh.S * 2 + sh.nch;

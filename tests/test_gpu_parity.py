@@ -85,6 +85,24 @@ def test_finely_interleaved_tenants_with_backward():
     _check_case(w, w.projections[0])
 
 
+@pytest.mark.parametrize("K,N", [(64, 64), (128, 320), (256, 320), (320, 1024)])
+def test_decode_shallow_contraction_repeated_calls(K, N):
+    # few 64-deep blocks of K: the decode GEMM may not cut the contraction into more slices than it has steps, and a
+    # second call on other activations must not see anything the first one left in tensor memory
+    w = wl.small_random_case(33 + K, 96, K, N, [16, 8, 32, 4], n_segments=9)
+    w.seg_offsets, w.seg_slot = wl.per_token_table(wl.uniform_token_slots(33 + K, 96, 4))
+    p = w.projections[0]
+    dc = DeviceCase(w, p, capacity=6)
+    ts = w.tok_slot()
+    r, s, A, Bm = oracle.adapters_of(p)
+    for rep in range(3):
+        xs = np.roll(p.x_bits, 7 * rep, axis=0)
+        ref, _ = oracle.forward(wl.bf16_bits_to_f32(xs), p.W, r, s, A, Bm, ts)
+        y = dc.forward(x=dev_bf16(xs))
+        assert_close(to_np(y), ref, f"decode K={K} N={N} call {rep}")
+    B.marlaas_check_status(dc.pool)
+
+
 def test_cfg2_decode_full_size():
     w = wl.make_workload(2)
     _check_case(w, w.projections[0])
