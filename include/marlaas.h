@@ -126,6 +126,28 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
                                       const marlaas_segments_t* seg, float* h_save, void* workspace,
                                       size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
+/* The same forward pass for callers that cannot allocate device memory (no counterpart in the paper: an
+ * addition for deployments, not part of the method).  Some hosts of this layer may not call cudaMalloc at all:
+ * a serving loop whose memory pool was sized and frozen at start-up, a plug-in that is handed nothing but its
+ * input and output buffers, a latency-critical path that cannot afford the device-wide synchronisation an
+ * allocation implies or its failure under a full memory budget.  For them the per-call scratch comes from an
+ * array built into the library (marlaas_lora_static_workspace_limit() bytes, 4 MiB, resident on every GPU that
+ * loads the library until the process exits) instead of a caller workspace; x, W, y, the pool storage and h_save
+ * are still the caller's.  The call allocates and frees nothing on the device.
+ *  - Batches whose scratch (marlaas_lora_workspace_bytes) exceeds the limit are rejected with
+ *    MARLAAS_ERR_WORKSPACE_TOO_SMALL before anything is launched: 256 tokens on a pool of 32 slots of rank
+ *    up to 64 fit.
+ *  - The first call on each device looks up the array's device address; make that call before starting any
+ *    stream capture on that device.
+ *  - All calls on a device share the one array and it keeps the previous call's contents (nothing in it has to
+ *    start at zero: each call writes what it later reads).  Two calls whose kernels overlap on the GPU -- different
+ *    streams, or different pools on different streams -- race on it; keep such calls on one stream. */
+size_t marlaas_lora_static_workspace_limit(void);
+marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx,
+                                                const void* W, int64_t ldw, void* y, int64_t ldy,
+                                                const marlaas_segments_t* seg, float* h_save, uint32_t flags,
+                                                void* cuda_stream);
+
 /* Backward for the policy-training stage: dx[T][d_in] bf16 (NULL = skip) and per-slot fp32 adapter gradients.
  * dA_slots / dB_slots: HOST arrays of `capacity` device pointers (either table, or any entry, may be NULL =
  * skip); dA_t is [d_in][r_t], dB_t is [r_t][d_out], row-major, at the slot's true rank.  Without

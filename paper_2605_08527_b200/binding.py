@@ -38,6 +38,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
+    "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws",
 ]
 
 
@@ -86,6 +87,10 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_lora_workspace_bytes.argtypes = [vp, i64]
     L.marlaas_lora_forward.restype = i32
     L.marlaas_lora_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, P(marlaas_segments_t), vp, vp, sz, u32, vp]
+    L.marlaas_lora_static_workspace_limit.restype = sz
+    L.marlaas_lora_static_workspace_limit.argtypes = []
+    L.marlaas_lora_forward_static_ws.restype = i32
+    L.marlaas_lora_forward_static_ws.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, P(marlaas_segments_t), vp, u32, vp]
     L.marlaas_lora_backward.restype = i32
     L.marlaas_lora_backward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, vp,
                                         P(marlaas_segments_t), vp, vp, sz, u32, vp]
@@ -242,6 +247,26 @@ def marlaas_lora_forward(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, se
     _check(load_library().marlaas_lora_forward(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(y), ldy,
                                                ctypes.byref(seg.c), _dptr(h_save), _dptr(ws), ws.numel(),
                                                flags | seg.flags, _stream(stream)))
+    return y
+
+
+def marlaas_lora_static_workspace_limit() -> int:
+    return int(load_library().marlaas_lora_static_workspace_limit())
+
+
+def marlaas_lora_forward_static_ws(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, seg: Segments,
+                                   y: torch.Tensor, h_save: Optional[torch.Tensor] = None, flags: int = 0,
+                                   stream=None) -> torch.Tensor:
+    """Forward for callers that may not allocate on the device: the scratch is the library's built-in array, and
+    this wrapper allocates nothing either (y is the caller's).  Raises for batches beyond the array's size."""
+    T = x.shape[0]
+    ldx, ldw, ldy = _mat(x, pool.d_in, "x"), _mat(W, pool.d_out, "W"), _mat(y, pool.d_out, "y")
+    assert W.shape[0] == pool.d_in and y.shape[0] == T
+    if h_save is not None:
+        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and tuple(h_save.shape) == (T, pool.rank_stride)
+    _check(load_library().marlaas_lora_forward_static_ws(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(y), ldy,
+                                                         ctypes.byref(seg.c), _dptr(h_save), flags | seg.flags,
+                                                         _stream(stream)))
     return y
 
 
