@@ -114,6 +114,7 @@ static marlaas_status_t make_plan(const marlaas_pool* pool, int64_t T, const mar
 // (decode-shaped) batches through the per-token gather kernel, which spreads over more SMs.
 static marlaas_status_t shrink(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
                                const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+    if (T >= 512 && shrink_split_sm100_eligible(pool, T, D)) return launch_shrink_split_sm100(pool, T, src, ld, D, store, ws, out, st);
     if (T >= 512) return launch_shrink_sm100(pool, T, src, ld, D, store, ws, out, st);
     return launch_shrink_hd(pool, T, src, ld, D, store, ws, out, st);
 }

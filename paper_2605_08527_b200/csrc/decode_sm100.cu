@@ -591,7 +591,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 }
 
 // x (or hd) viewed as a 3-D tensor (64 k, rows, K / 64) so that one copy brings `panels` K-major tiles of 128 rows
-static marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels) {
+marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels) {
     typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);

@@ -1,0 +1,412 @@
+// Segmented shrink with the contraction split over a cluster (sm_100a).  Same outputs as shrink_sm100.cu
+// (h = x A_t or g = dy B_t^T per token, fp32, plus the bf16 block-diagonal expand operand hd), for batches with too
+// few 128-token tiles to occupy the SMs one tile per CTA: a cluster of C CTAs owns one tile, each CTA streams 1/C of
+// the contraction dimension through the same TMA / tcgen05 pipeline, and every CTA's epilogue sends, for each token,
+// only the columns of the token's own tenant (at most RP floats) to the cluster's first CTA, which adds the C
+// partial vectors in rank order and writes the results.  No atomics: the sum order is fixed.
+#include "sm100_ptx.cuh"
+
+namespace marlaas {
+namespace sm100 {
+
+constexpr int SS_THREADS = 192;
+constexpr int SS_GROUP_UNITS = 16;                           // units per pass: N = 256 accumulator columns
+constexpr uint32_t SS_B_STAGE_BYTES = SS_GROUP_UNITS * UNIT_BYTES;
+constexpr uint32_t SS_STAGE_BYTES = A_STAGE_BYTES + SS_B_STAGE_BYTES;
+constexpr int SS_MAX_C = 8;
+constexpr int SS_MAX_STAGES = 12;
+
+struct ShrinkSplitArgs {
+    int T, D;
+    int num_kb;
+    int RP, cap;
+    int C;
+    uint32_t stage_area;          // bytes of shared memory for the pipeline stages
+    const int32_t* tok_slot;
+    const int32_t* tok_uoff;
+    const int32_t* tile_nunits;
+    const int32_t* tile_units;
+    int umax;
+    const int32_t* d_rank;
+    const float* d_scale;
+    float* out;       // [T][RP], zero-filled before the launch
+    bf16* hd;         // [T][hd_cols]
+    int hd_cols;
+    int32_t* status;
+};
+
+__device__ __forceinline__ void ss_tc_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t ss_cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t ss_cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t ss_map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void ss_cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void ss_st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// Adapter rows are fetched in runs: consecutive units of the tile's list that are also consecutive in the store (a
+// tenant's own units always are, and so are neighbouring slots) move with one TMA instruction of 16 * 2^i rows, since
+// the issuing thread pays about a hundred cycles per instruction whatever its size.
+struct StoreMaps {
+    CUtensorMap m[5];     // boxes of 16, 32, 64, 128, 256 rows x 64 k
+};
+
+// Cuts a group's unit list into runs; run i covers 2^lg units starting at list position pos, store row `row`.
+struct UnitRun { int row; short pos; short lg; };
+__device__ __forceinline__ int ss_plan_runs(const int32_t* units, int nug, UnitRun* runs) {
+    int u = 0, n = 0;
+    while (u < nug) {
+        const int r0 = units[u];
+        int run = 1;
+        while (u + run < nug && units[u + run] == r0 + 16 * run) ++run;
+        int lg = 31 - __clz(run);                 // largest power of two <= run, at most 16 units
+        if (lg > 4) lg = 4;
+        runs[n].row = r0; runs[n].pos = (short)u; runs[n].lg = (short)lg;
+        ++n;
+        u += 1 << lg;
+    }
+    return n;
+}
+
+// Shared memory: [stages x (A tile 16 KB + unit slabs 32 KB)] [gather buffer C x 128 rows x RP floats] [barriers]
+// (the gather buffer is used in the cluster's first CTA only; every CTA reserves it so that the layout is uniform).
+__global__ void __launch_bounds__(SS_THREADS, 1)
+k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_constant__ CUtensorMap tmSrc2,
+                     const __grid_constant__ CUtensorMap tmSrc4,
+                     const __grid_constant__ StoreMaps tmStore,
+                     const ShrinkSplitArgs g) {
+    constexpr uint32_t TMEM_COLS = 512;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ UnitRun s_runs[SS_GROUP_UNITS];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t crank = ss_cluster_ctarank();
+    const int m = (int)ss_cluster_id_x();                    // the cluster's 128-token tile
+    const int nun = g.tile_nunits[m >> 1];
+    const int32_t* units = g.tile_units + (size_t)(m >> 1) * g.umax;
+    // Pipeline steps are kp 64-deep panels: the two issuing threads pay a fixed price per step (barrier wait, commit,
+    // TMA issue), which at one panel per step, not HBM, set the pace.  Narrow groups take 4 panels, wide ones 2.
+    const int wide = max(1, min(SS_GROUP_UNITS, nun));
+    int kp = wide <= 4 ? 4 : 2;
+    while (kp > 1 && 2u * (uint32_t)kp * (A_STAGE_BYTES + (uint32_t)wide * UNIT_BYTES) > g.stage_area) kp >>= 1;   // two stages at least
+    const CUtensorMap* tmSrc = kp == 4 ? &tmSrc4 : kp == 2 ? &tmSrc2 : &tmSrc1;
+    const int num_steps = (g.num_kb + kp - 1) / kp;
+    const int kb0 = (int)((int64_t)crank * num_steps / g.C), kb1 = (int)((int64_t)(crank + 1) * num_steps / g.C);   // steps
+
+    // A stage holds the 128 x 64 tile of x and as many 16-row unit slabs as the tile's widest group needs: tiles with
+    // few tenants get more, smaller stages, i.e. more bytes in flight.
+    const uint32_t b_panel_bytes = (uint32_t)wide * UNIT_BYTES;         // one panel of all units of a group
+    const uint32_t a_stage_bytes = (uint32_t)kp * A_STAGE_BYTES, b_stage_bytes = (uint32_t)kp * b_panel_bytes;
+    const uint32_t stage_bytes = a_stage_bytes + b_stage_bytes;
+    const int STAGES = min(SS_MAX_STAGES, (int)(g.stage_area / stage_bytes));
+    const uint32_t sA = smem_u32(smem);
+    const uint32_t sB = sA + STAGES * a_stage_bytes;
+    const uint32_t sG = sA + g.stage_area;
+    const uint32_t gather_bytes = (uint32_t)g.C * 128u * (uint32_t)g.RP * 4u;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + g.stage_area + gather_bytes);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * SS_MAX_STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * SS_MAX_STAGES;
+    const uint32_t bar_tempty = bar_tfull + 16;
+    const uint32_t bar_drain = bar_tempty + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SS_MAX_STAGES + 5);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_tfull + 8 * b, 1);
+            mbar_init(bar_tempty + 8 * b, 4);
+        }
+        mbar_init(bar_drain, 1);
+        *abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        prefetch_tmap(tmSrc);
+        for (int i = 0; i < 5; ++i) prefetch_tmap(&tmStore.m[i]);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // per-row routing (epilogue threads): the row's units within the tile's list
+    const int q = warp & 3;
+    const int rl = q * 32 + lane;                            // row within the tile
+    const int row = m * BM + rl;
+    int uo = -1, nu = 0;
+    float sc = 0.f;
+    if (warp >= 2 && row < g.T && nun > 0) {
+        const int t = g.tok_slot[row];
+        const int r = (t >= 0 && t < g.cap) ? g.d_rank[t] : 0;
+        if (r > 0) {
+            uo = g.tok_uoff[row];
+            nu = (r + 15) >> 4;
+            sc = g.d_scale[t];
+        }
+    }
+
+    if (warp == 0) {
+        if (lane == 0) {   // ---- TMA producer: this CTA's slice of the contraction, once per unit group
+            uint32_t it = 0, s = 0, ph = 0;
+            bool ok = true;
+            for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS) {
+                const int nug = min(SS_GROUP_UNITS, nun - g0);
+                const int nruns = ss_plan_runs(units + g0, nug, s_runs);
+                for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 51))) break;
+                    const uint32_t full = bar_full + 8 * s;
+                    mbar_expect_tx(full, a_stage_bytes + kp * nug * UNIT_BYTES);
+                    tma_load_3d(sA + s * a_stage_bytes, tmSrc, full, 0, m * BM, kb * kp);
+                    for (int p = 0; p < kp; ++p)
+                        for (int i = 0; i < nruns; ++i)
+                            tma_load_2d(sB + s * b_stage_bytes + p * b_panel_bytes + s_runs[i].pos * UNIT_BYTES,
+                                        &tmStore.m[s_runs[i].lg], full, (kb * kp + p) * BK, s_runs[i].row);
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+                }
+            }
+            if (!ok) {
+                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                for (uint32_t j = 0; j < back; ++j) {
+                    const uint32_t jt = it - 1 - j;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * (jt % (uint32_t)STAGES), (jt / (uint32_t)STAGES) & 1) &&
+                           global_ns() - t0 < WAIT_LIMIT_NS) {
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {   // ---- MMA issuer
+            uint32_t s = 0, ph = 0, lt = 0;
+            bool ok = true;
+            for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS, ++lt) {
+                const int nug = min(SS_GROUP_UNITS, nun - g0);
+                const uint32_t idesc = make_idesc(nug * 16, 0);
+                const uint32_t b = lt & 1, aph = (lt >> 1) & 1;
+                if (!(ok = mbar_wait(bar_tempty + 8 * b, aph ^ 1, abort_word, 53))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + b * 256;
+                uint32_t acc = 0;
+                for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                    if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 54))) break;
+                    tc_fence_after();
+                    const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
+                    for (int p = 0; p < kp; ++p) {
+#pragma unroll
+                        for (int j = 0; j < BK / 16; ++j) {
+                            tc_mma_bf16(d_tmem, desc_k_major(a0 + p * A_STAGE_BYTES + j * 32),
+                                        desc_k_major(b0 + p * b_panel_bytes + j * 32), idesc, acc);
+                            acc = 1;
+                        }
+                    }
+                    tc_commit(bar_empty + 8 * s);
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+                }
+                if (ok) tc_commit(bar_tfull + 8 * b);
+            }
+            if (!ok) {
+                tc_commit(bar_drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bar_drain, 0) && global_ns() - t0 < WAIT_LIMIT_NS) {
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue: this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
+        const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)g.RP) * 4u;
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS, ++lt) {
+            const int nug = min(SS_GROUP_UNITS, nun - g0);
+            const uint32_t b = lt & 1, aph = (lt >> 1) & 1;
+            ok = mbar_wait(bar_tfull + 8 * b, aph, abort_word, 56);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int u = 0; u < nug; ++u) {
+                uint32_t v[16];
+                ss_tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + b * 256 + u * 16, v);
+                tc_wait_ld();
+                const int gu = g0 + u;
+                if (uo >= 0 && gu >= uo && gu < uo + nu) {
+                    const uint32_t a = gdst + (uint32_t)(gu - uo) * 64u;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        ss_st_cluster_v4(a + e * 16, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
+        }
+    }
+
+    // ---- every CTA's partial vectors are in CTA 0: add them in rank order and write the results ----------------
+    tc_fence_before();
+    __syncthreads();
+    ss_cluster_sync();
+    if (crank == 0 && warp >= 2 && row < g.T && *abort_word == 0) {
+        const float* gbuf = reinterpret_cast<const float*>(smem + g.stage_area);
+        bf16* hrow = g.hd + (size_t)row * g.hd_cols;
+        for (int gu = 0; gu < nun; ++gu) {
+            uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
+            if (uo >= 0 && gu >= uo && gu < uo + nu) {
+                float v[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0.f;
+                for (int c = 0; c < g.C; ++c) {      // fixed order
+                    const float4* p = reinterpret_cast<const float4*>(gbuf + ((size_t)c * 128 + rl) * g.RP + (gu - uo) * 16);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 t4 = p[e];
+                        v[4 * e] += t4.x; v[4 * e + 1] += t4.y; v[4 * e + 2] += t4.z; v[4 * e + 3] += t4.w;
+                    }
+                }
+                __nv_bfloat162 pk[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) pk[e] = __floats2bfloat162_rn(sc * v[2 * e], sc * v[2 * e + 1]);
+                o0 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[0]), *reinterpret_cast<uint32_t*>(&pk[1]),
+                                *reinterpret_cast<uint32_t*>(&pk[2]), *reinterpret_cast<uint32_t*>(&pk[3]));
+                o1 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[4]), *reinterpret_cast<uint32_t*>(&pk[5]),
+                                *reinterpret_cast<uint32_t*>(&pk[6]), *reinterpret_cast<uint32_t*>(&pk[7]));
+                float4* dst = reinterpret_cast<float4*>(g.out + (size_t)row * g.RP + (gu - uo) * 16);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+            }
+            uint4* hdst = reinterpret_cast<uint4*>(hrow + gu * 16);
+            hdst[0] = o0;
+            hdst[1] = o1;
+        }
+    }
+
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+    if (threadIdx.x == 0 && *abort_word != 0) {
+        if (atomicCAS(g.status, 0, DEV_TIMEOUT) == 0) g.status[1] = *abort_word * 1000000 + (int)blockIdx.x;
+    }
+}
+
+}  // namespace sm100
+
+// Cluster width for T tokens: as many CTAs per tile as keep the whole grid resident in one wave (0 = this kernel
+// does not apply: more tiles than SMs, where the persistent one-CTA-per-tile kernel is the better fit).
+static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, size_t* smem_out, uint32_t* area_out) {
+    using namespace sm100;
+    if (tiles > pool->sm_count) return 0;
+    static int max_active[64][SS_MAX_C + 1] = {};
+    for (int C = SS_MAX_C; C >= 1; --C) {
+        if ((int64_t)C * tiles > pool->sm_count || (C > 1 && num_kb < 16 * C)) continue;
+        const size_t gather = (size_t)C * 128 * pool->RP * 4;
+        const size_t avail = 222 * 1024 - 1024 - 256;
+        if (gather + 2 * SS_STAGE_BYTES > avail) continue;
+        const size_t area = (avail - gather) / 1024 * 1024;
+        const size_t smem = 1024 + area + gather + 256;
+        int mc = pool->device < 64 ? max_active[pool->device][C] : 0;
+        if (mc == 0) {
+            if (cudaFuncSetAttribute(k_shrink_split_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024) != cudaSuccess) return 0;
+            cudaLaunchConfig_t qc = {};
+            qc.gridDim = dim3((unsigned)(C * 64));
+            qc.blockDim = dim3(SS_THREADS);
+            qc.dynamicSmemBytes = 200 * 1024;
+            cudaLaunchAttribute qa;
+            qa.id = cudaLaunchAttributeClusterDimension;
+            qa.val.clusterDim.x = (unsigned)C; qa.val.clusterDim.y = 1; qa.val.clusterDim.z = 1;
+            qc.attrs = &qa; qc.numAttrs = 1;
+            if (cudaOccupancyMaxActiveClusters(&mc, k_shrink_split_sm100, &qc) != cudaSuccess || mc < 1) mc = -1;
+            cudaGetLastError();
+            if (pool->device < 64) max_active[pool->device][C] = mc;
+        }
+        if (mc < tiles) continue;
+        *smem_out = smem;
+        *area_out = (uint32_t)area;
+        return C;
+    }
+    return 0;
+}
+
+bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D) {
+    size_t smem; uint32_t area;
+    return T > 0 && (D % 64) == 0 && split_width(pool, cdiv(T, sm100::BM), cdiv(D, sm100::BK), &smem, &area) > 0;
+}
+
+marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
+                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+    using namespace sm100;
+    if (T <= 0) return MARLAAS_OK;
+    const int64_t tiles = cdiv(T, BM);
+    size_t smem_bytes = 0;
+    uint32_t area = 0;
+    const int C = split_width(pool, tiles, cdiv(D, BK), &smem_bytes, &area);
+    if (C <= 0) return fail(MARLAAS_ERR_INVALID_ARG, "shrink_split: %lld tiles do not fit one wave", (long long)tiles);
+    ShrinkSplitArgs g;
+    g.T = (int)T; g.D = (int)D;
+    g.num_kb = (int)cdiv(D, BK);
+    g.RP = pool->RP; g.cap = pool->cap;
+    g.C = C; g.stage_area = area;
+    g.tok_slot = ws.tok_slot; g.tok_uoff = ws.tok_uoff;
+    g.tile_nunits = ws.tile_nunits; g.tile_units = ws.tile_units; g.umax = ws.umax;
+    g.d_rank = pool->d_rank; g.d_scale = pool->d_scale;
+    g.out = out; g.hd = ws.hd; g.hd_cols = ws.umax * 16;
+    g.status = pool->d_status;
+    alignas(64) CUtensorMap tmSrc1, tmSrc2, tmSrc4;
+    alignas(64) StoreMaps maps;
+    marlaas_status_t rc;
+    if ((rc = make_panel_map(&tmSrc1, src, T, D, ld, 1)) != MARLAAS_OK) return rc;
+    if ((rc = make_panel_map(&tmSrc2, src, T, D, ld, 2)) != MARLAAS_OK) return rc;
+    if ((rc = make_panel_map(&tmSrc4, src, T, D, ld, 4)) != MARLAAS_OK) return rc;
+    for (int i = 0; i < 5; ++i)
+        if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, D, BK, 16u << i)) != MARLAAS_OK) return rc;
+    MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * C));
+    cfg.blockDim = dim3(SS_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_shrink_split_sm100, tmSrc1, tmSrc2, tmSrc4, maps, g));
+    count_launch();
+    return MARLAAS_OK;
+}
+
+}  // namespace marlaas

@@ -127,5 +127,16 @@ __host__ __device__ constexpr uint32_t make_idesc(int bn, int b_mn) {
 marlaas_status_t make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols,
                           uint32_t box_rows);
 
+// The same matrix viewed as a 3-D tensor (64 k, rows, cols / 64): one copy brings `panels` consecutive K-major
+// [128 rows][64 k] tiles.  cols must be a multiple of 64.
+marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels);
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
 }  // namespace sm100
 }  // namespace marlaas
