@@ -462,10 +462,11 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tc_fence_after();
                 const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
                 for (int q = 0; q < g.kp; ++q) {
+                    // descriptors of successive 16-deep slices differ only in the start-address field (16-byte units)
+                    const uint64_t da0 = desc_k_major(a0 + q * A_STAGE_BYTES), db0 = desc_mn_major(b0 + q * CHUNK_BYTES, b_chunk_bytes);
 #pragma unroll
                     for (int j = 0; j < BK / 16; ++j) {
-                        dg_mma_pair(tmem_base, desc_k_major(a0 + q * A_STAGE_BYTES + j * 32),
-                                    desc_mn_major(b0 + q * CHUNK_BYTES + j * UNIT_BYTES, b_chunk_bytes), idesc, acc);
+                        dg_mma_pair(tmem_base, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(j * (UNIT_BYTES >> 4)), idesc, acc);
                         acc = 1;
                     }
                 }

@@ -19,6 +19,7 @@ namespace sm100 {
 
 constexpr int GRAD_THREADS = 192;
 constexpr int GRAD_STAGES = 4;
+constexpr int GRAD_QN = 4;               // depth of the CTA's work-item queue
 constexpr uint32_t GB_STAGE_BYTES = 4 * CHUNK_BYTES;   // up to 256 columns of split r-vectors
 
 __device__ __forceinline__ void tc_ld_32x16g(uint32_t taddr, uint32_t (&v)[16]) {
@@ -95,6 +96,8 @@ __global__ void __launch_bounds__(256) k_grad_lists(int nblk, int cap, int max_c
             blk_base[nblk] = total;
             gflag[0] = total > max_copies ? 1 : 0;
             gflag[1] = total;
+            gflag[2] = 0;      // work-item counters of the two reduction launches (dB, dA)
+            gflag[3] = 0;
         }
     }
     // this tenant's copies, ascending block order
@@ -174,6 +177,7 @@ struct GradArgs {
     const int32_t* ten_blks;
     const int32_t* ten_pos;
     const int32_t* gflag;
+    int32_t* counter;      // next work item (zeroed by the plan kernel before every pair of launches)
     float* const* out_ptrs;
     int transpose_out, accumulate;
     int32_t* status;
@@ -195,8 +199,11 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;
     const uint32_t bar_tempty = bar_tfull + 16;
     const uint32_t bar_drain = bar_tempty + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+    const uint32_t bar_qfull = bar_drain + 8, bar_qempty = bar_qfull + 8 * GRAD_QN;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 2 * GRAD_QN);
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    __shared__ int s_cnt[256], s_order[256];
+    __shared__ volatile int s_q[GRAD_QN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_items = g.num_c_tiles * g.cap;
@@ -212,6 +219,10 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
             mbar_init(bar_tempty + 8 * b, 4);
         }
         mbar_init(bar_drain, 1);
+        for (int i = 0; i < GRAD_QN; ++i) {
+            mbar_init(bar_qfull + 8 * i, 1);
+            mbar_init(bar_qempty + 8 * i, 5);     // the MMA thread and the four epilogue warps
+        }
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -224,24 +235,41 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // Work items are handed out dynamically, heaviest tenants first (an item's cost is its tenant's copy count), so that
+    // skewed batches still finish together; which CTA computes an item does not change its value.
+    for (int t = threadIdx.x; t < g.cap; t += GRAD_THREADS) s_cnt[t] = (g.out_ptrs[t] != nullptr && g.d_rank[t] > 0) ? g.ten_nblk[t] : -1;
     tc_fence_before();
+    __syncthreads();
+    for (int t = threadIdx.x; t < g.cap; t += GRAD_THREADS) {
+        const int c = s_cnt[t];
+        int rk = 0;
+        for (int u = 0; u < g.cap; ++u) rk += (s_cnt[u] > c) || (s_cnt[u] == c && u < t);
+        s_order[rk] = t;
+    }
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     // an item does tensor work only if its slot has an output, a rank and at least one copy
     auto item_blocks = [&](int item, int& t, int& c0) -> int {
-        t = item % g.cap;
-        c0 = (item / g.cap) * 128;
-        if (g.out_ptrs[t] == nullptr || g.d_rank[t] <= 0) return -1;
-        return g.ten_nblk[t];
+        t = s_order[item / g.num_c_tiles];
+        c0 = (item % g.num_c_tiles) * 128;
+        return s_cnt[t];      // -1: no output or no rank
     };
 
     if (warp == 0) {
         if (lane == 0) {   // ---- TMA producer
-            uint32_t it = 0;
+            uint32_t it = 0, qi = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            while (ok) {
+                const uint32_t qs = qi % GRAD_QN, qph = (qi / GRAD_QN) & 1;
+                if (!(ok = mbar_wait(bar_qempty + 8 * qs, qph ^ 1, abort_word, 27))) break;
+                int item = atomicAdd(g.counter, 1);
+                if (item >= num_items) item = -1;
+                s_q[qs] = item;
+                mbar_arrive(bar_qfull + 8 * qs);
+                ++qi;
+                if (item < 0) break;
                 int t, c0;
                 const int nb = item_blocks(item, t, c0);
                 if (nb <= 0) continue;
@@ -276,7 +304,14 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
             const uint32_t idesc = make_idesc(g.HW, 1) | (1u << 15);
             uint32_t it = 0, lt = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+            uint32_t qi = 0;
+            while (ok) {
+                const uint32_t qs = qi % GRAD_QN, qph = (qi / GRAD_QN) & 1;
+                if (!(ok = mbar_wait(bar_qfull + 8 * qs, qph, abort_word, 28))) break;
+                const int item = s_q[qs];
+                mbar_arrive(bar_qempty + 8 * qs);
+                ++qi;
+                if (item < 0) break;
                 int t, c0;
                 const int nb = item_blocks(item, t, c0);
                 if (nb <= 0) continue;
@@ -290,10 +325,11 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 24))) break;
                     tc_fence_after();
                     const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * GB_STAGE_BYTES;
+                    // descriptors of successive 16-token slices differ only in the start-address field (16-byte units)
+                    const uint64_t da0 = desc_mn_major(a0, CHUNK_BYTES), db0 = desc_mn_major(b0, CHUNK_BYTES);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        tc_mma_bf16(d_tmem, desc_mn_major(a0 + j * UNIT_BYTES, CHUNK_BYTES),
-                                    desc_mn_major(b0 + j * UNIT_BYTES, CHUNK_BYTES), idesc, acc);
+                        tc_mma_bf16(d_tmem, da0 + (uint64_t)(j * (UNIT_BYTES >> 4)), db0 + (uint64_t)(j * (UNIT_BYTES >> 4)), idesc, acc);
                         acc = 1;
                     }
                     tc_commit(bar_empty + 8 * s);
@@ -314,7 +350,17 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
         const int q = warp & 3;
         uint32_t lt = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        uint32_t qi = 0;
+        while (ok) {
+            const uint32_t qs = qi % GRAD_QN, qph = (qi / GRAD_QN) & 1;
+            ok = mbar_wait(bar_qfull + 8 * qs, qph, abort_word, 29);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const int item = s_q[qs];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_qempty + 8 * qs);
+            ++qi;
+            if (item < 0) break;
             int t, c0;
             const int nb = item_blocks(item, t, c0);
             if (nb < 0) continue;
@@ -407,6 +453,7 @@ marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t 
     g.ten_blks = ws.ten_blks;
     g.ten_pos = ws.ten_pos;
     g.gflag = ws.gflag;
+    g.counter = ws.gflag + (transpose_out ? 3 : 2);
     g.out_ptrs = out_ptrs;
     g.transpose_out = transpose_out ? 1 : 0;
     g.accumulate = accumulate ? 1 : 0;

@@ -226,10 +226,11 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_co
                     tc_fence_after();
                     const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
                     for (int p = 0; p < kp; ++p) {
+                        // descriptors of successive 16-deep slices differ only in the start-address field (16-byte units)
+                        const uint64_t da0 = desc_k_major(a0 + p * A_STAGE_BYTES), db0 = desc_k_major(b0 + p * b_panel_bytes);
 #pragma unroll
                         for (int j = 0; j < BK / 16; ++j) {
-                            tc_mma_bf16(d_tmem, desc_k_major(a0 + p * A_STAGE_BYTES + j * 32),
-                                        desc_k_major(b0 + p * b_panel_bytes + j * 32), idesc, acc);
+                            tc_mma_bf16(d_tmem, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(2 * j), idesc, acc);
                             acc = 1;
                         }
                     }
