@@ -290,9 +290,15 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     }
     if (want_dA || want_dB) {
         const bool tc_grad = tc_path && grad_sm100_eligible(pool, T);
+        // The tensor-core reduction needs one copy of a 64-token block per tenant present in it; there are at most
+        // (blocks + segments) of them, so when that bound fits the workspace the CUDA-core fallback cannot be needed
+        // and neither it, nor the sort it consumes, nor the device copies of the pointer tables are issued.
+        const int64_t nblk = cdiv(T, 64);
+        const bool fits = tc_grad && nblk + (int64_t)seg->num_segments <= (int64_t)ws.max_copies;
+        const bool inline_tables = fits && pool->cap <= 64;
         const int32_t* run_flag = tc_grad ? ws.gflag : nullptr;   // the CUDA-core kernels run only if the flag is set
         if (tc_grad && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
-        if ((rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
+        if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
         if (want_dB) {
             const float* h = h_saved;
             if (!h && T > 0) {
@@ -301,16 +307,18 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
                 if (rc != MARLAAS_OK) return rc;
                 h = ws.h;
             }
-            MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, false, acc, ws, st)) != MARLAAS_OK) return rc;
-            if ((rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
-                                         false, acc, st, run_flag)) != MARLAAS_OK) return rc;
+            if (!inline_tables)
+                MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, dB_slots, false, acc, ws, st)) != MARLAAS_OK) return rc;
+            if (!fits && (rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
+                                                  false, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }
         if (want_dA) {
-            MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, true, acc, ws, st)) != MARLAAS_OK) return rc;
-            if ((rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
-                                         true, acc, st, run_flag)) != MARLAAS_OK) return rc;
+            if (!inline_tables)
+                MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, dA_slots, true, acc, ws, st)) != MARLAAS_OK) return rc;
+            if (!fits && (rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
+                                                  true, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }
     }
     return finish(pool, flags, st);

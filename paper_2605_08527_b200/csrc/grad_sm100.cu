@@ -19,6 +19,7 @@ namespace sm100 {
 
 constexpr int GRAD_THREADS = 192;
 constexpr int GRAD_STAGES = 4;
+constexpr int GRAD_INLINE_SLOTS = 64;
 constexpr int GRAD_QN = 4;               // depth of the CTA's work-item queue
 constexpr uint32_t GB_STAGE_BYTES = 4 * CHUNK_BYTES;   // up to 256 columns of split r-vectors
 
@@ -178,9 +179,10 @@ struct GradArgs {
     const int32_t* ten_pos;
     const int32_t* gflag;
     int32_t* counter;      // next work item (zeroed by the plan kernel before every pair of launches)
-    float* const* out_ptrs;
+    float* const* out_ptrs;   // per-slot outputs in device memory, or nullptr: the table is inl[] below
     int transpose_out, accumulate;
     int32_t* status;
+    float* inl[GRAD_INLINE_SLOTS];   // small pools: the pointer table travels with the launch (no host-to-device copy)
 };
 
 __global__ void __launch_bounds__(GRAD_THREADS, 1)
@@ -237,7 +239,7 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
     }
     // Work items are handed out dynamically, heaviest tenants first (an item's cost is its tenant's copy count), so that
     // skewed batches still finish together; which CTA computes an item does not change its value.
-    for (int t = threadIdx.x; t < g.cap; t += GRAD_THREADS) s_cnt[t] = (g.out_ptrs[t] != nullptr && g.d_rank[t] > 0) ? g.ten_nblk[t] : -1;
+    for (int t = threadIdx.x; t < g.cap; t += GRAD_THREADS) s_cnt[t] = ((g.out_ptrs ? g.out_ptrs[t] : g.inl[t]) != nullptr && g.d_rank[t] > 0) ? g.ten_nblk[t] : -1;
     tc_fence_before();
     __syncthreads();
     for (int t = threadIdx.x; t < g.cap; t += GRAD_THREADS) {
@@ -364,7 +366,7 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
             int t, c0;
             const int nb = item_blocks(item, t, c0);
             if (nb < 0) continue;
-            float* out = g.out_ptrs[t];
+            float* out = g.out_ptrs ? g.out_ptrs[t] : g.inl[t];
             const int r = g.d_rank[t];
             const int c = c0 + q * 32 + lane;
             if (nb == 0) {   // tenant without tokens: exact zeros unless accumulating
@@ -433,7 +435,8 @@ marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Wor
 }
 
 marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
-                                   const float* hg, float* const* out_ptrs, bool transpose_out, bool accumulate,
+                                   const float* hg, float* const* out_ptrs, float* const* host_ptrs, bool transpose_out,
+                                   bool accumulate,
                                    const Workspace& ws, cudaStream_t st) {
     using namespace sm100;
     const int nblk = (int)cdiv(T, 64);
@@ -455,6 +458,10 @@ marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t 
     g.gflag = ws.gflag;
     g.counter = ws.gflag + (transpose_out ? 3 : 2);
     g.out_ptrs = out_ptrs;
+    if (host_ptrs && pool->cap <= GRAD_INLINE_SLOTS) {
+        g.out_ptrs = nullptr;
+        for (int t = 0; t < GRAD_INLINE_SLOTS; ++t) g.inl[t] = t < pool->cap ? host_ptrs[t] : nullptr;
+    }
     g.transpose_out = transpose_out ? 1 : 0;
     g.accumulate = accumulate ? 1 : 0;
     g.status = pool->d_status;

@@ -194,7 +194,8 @@ marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const b
 bool grad_sm100_eligible(const marlaas_pool* pool, int64_t T);
 marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Workspace& ws, cudaStream_t st);
 marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
-                                   const float* hg, float* const* out_ptrs, bool transpose_out, bool accumulate,
-                                   const Workspace& ws, cudaStream_t st);
+                                   const float* hg, float* const* out_ptrs, float* const* host_ptrs, bool transpose_out,
+                                   bool accumulate, const Workspace& ws, cudaStream_t st);
+// host_ptrs: the same table in host memory; pools of at most 64 slots pass it with the launch and never read out_ptrs
 
 }  // namespace marlaas
