@@ -10,18 +10,18 @@ namespace marlaas {
 namespace sm100 {
 
 constexpr int SS_THREADS = 192;
-constexpr int SS_GROUP_UNITS = 16;                           // units per pass: N = 256 accumulator columns
-constexpr uint32_t SS_B_STAGE_BYTES = SS_GROUP_UNITS * UNIT_BYTES;
-constexpr uint32_t SS_STAGE_BYTES = A_STAGE_BYTES + SS_B_STAGE_BYTES;
+constexpr int SS_SUB_UNITS = 8;                              // units per work item: N = 128 accumulator columns
+constexpr int SS_KP = 2;                                     // 64-deep panels per pipeline step
+constexpr uint32_t SS_STEP_BYTES = SS_KP * (A_STAGE_BYTES + SS_SUB_UNITS * UNIT_BYTES);   // 64 KB
 constexpr int SS_MAX_C = 8;
-constexpr int SS_MAX_STAGES = 12;
+constexpr int SS_MAX_STAGES = 4;
+constexpr int SS_MAX_TILES = 160;
 
 struct ShrinkSplitArgs {
     int T, D;
-    int num_kb;
+    int num_kb, num_m_tiles;
     int RP, cap;
-    int C;
-    uint32_t stage_area;          // bytes of shared memory for the pipeline stages
+    int C, stages;
     const int32_t* tok_slot;
     const int32_t* tok_uoff;
     const int32_t* tile_nunits;
@@ -71,7 +71,7 @@ __device__ __forceinline__ void ss_st_cluster_v4(uint32_t addr, uint32_t a, uint
 // tenant's own units always are, and so are neighbouring slots) move with one TMA instruction of 16 * 2^i rows, since
 // the issuing thread pays about a hundred cycles per instruction whatever its size.
 struct StoreMaps {
-    CUtensorMap m[5];     // boxes of 16, 32, 64, 128, 256 rows x 64 k
+    CUtensorMap m[4];     // boxes of 16, 32, 64, 128 rows x 64 k
 };
 
 // Cuts a group's unit list into runs; run i covers 2^lg units starting at list position pos, store row `row`.
@@ -82,8 +82,8 @@ __device__ __forceinline__ int ss_plan_runs(const int32_t* units, int nug, UnitR
         const int r0 = units[u];
         int run = 1;
         while (u + run < nug && units[u + run] == r0 + 16 * run) ++run;
-        int lg = 31 - __clz(run);                 // largest power of two <= run, at most 16 units
-        if (lg > 4) lg = 4;
+        int lg = 31 - __clz(run);                 // largest power of two <= run, at most 8 units
+        if (lg > 3) lg = 3;
         runs[n].row = r0; runs[n].pos = (short)u; runs[n].lg = (short)lg;
         ++n;
         u += 1 << lg;
@@ -91,48 +91,39 @@ __device__ __forceinline__ int ss_plan_runs(const int32_t* units, int nug, UnitR
     return n;
 }
 
-// Shared memory: [stages x (A tile 16 KB + unit slabs 32 KB)] [gather buffer C x 128 rows x RP floats] [barriers]
-// (the gather buffer is used in the cluster's first CTA only; every CTA reserves it so that the layout is uniform).
+// Work items: a 128-token tile's unit list is cut into sub-groups of at most SS_SUB_UNITS units, and one item =
+// (tile, sub-group).  Items, not tiles, are what costs alike (the tile of x plus a bounded slab of adapter rows per
+// 64 k), so a tile that mixes many tenants is spread over several clusters instead of holding everyone up.  The
+// clusters walk the item list with a fixed stride; every CTA derives the same list from the per-tile unit counts.
+//
+// Shared memory: [stages x kp x (A panel 16 KB + unit slab 16 KB)] [gather buffer C x 128 rows x 128 floats]
+// [barriers] (the gather buffer is used in the cluster's first CTA only; every CTA reserves it).
 __global__ void __launch_bounds__(SS_THREADS, 1)
-k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_constant__ CUtensorMap tmSrc2,
-                     const __grid_constant__ CUtensorMap tmSrc4,
-                     const __grid_constant__ StoreMaps tmStore,
+k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ StoreMaps tmStore,
                      const ShrinkSplitArgs g) {
-    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t TMEM_COLS = 128;
+    constexpr int KP = SS_KP;
+    constexpr uint32_t A_STEP = KP * A_STAGE_BYTES, B_PANEL = SS_SUB_UNITS * UNIT_BYTES, B_STEP = KP * B_PANEL;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ UnitRun s_runs[SS_GROUP_UNITS];
+    __shared__ UnitRun s_runs[SS_SUB_UNITS];
+    __shared__ int s_first[SS_MAX_TILES + 1];        // first item of every tile (exclusive scan of the sub-group counts)
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t crank = ss_cluster_ctarank();
-    const int m = (int)ss_cluster_id_x();                    // the cluster's 128-token tile
-    const int nun = g.tile_nunits[m >> 1];
-    const int32_t* units = g.tile_units + (size_t)(m >> 1) * g.umax;
-    // Pipeline steps are kp 64-deep panels: the two issuing threads pay a fixed price per step (barrier wait, commit,
-    // TMA issue), which at one panel per step, not HBM, set the pace.  Narrow groups take 4 panels, wide ones 2.
-    const int wide = max(1, min(SS_GROUP_UNITS, nun));
-    int kp = wide <= 4 ? 4 : 2;
-    while (kp > 1 && 2u * (uint32_t)kp * (A_STAGE_BYTES + (uint32_t)wide * UNIT_BYTES) > g.stage_area) kp >>= 1;   // two stages at least
-    const CUtensorMap* tmSrc = kp == 4 ? &tmSrc4 : kp == 2 ? &tmSrc2 : &tmSrc1;
-    const int num_steps = (g.num_kb + kp - 1) / kp;
-    const int kb0 = (int)((int64_t)crank * num_steps / g.C), kb1 = (int)((int64_t)(crank + 1) * num_steps / g.C);   // steps
+    const int cid = (int)ss_cluster_id_x(), ncl = (int)(gridDim.x / g.C);
 
-    // A stage holds the 128 x 64 tile of x and as many 16-row unit slabs as the tile's widest group needs: tiles with
-    // few tenants get more, smaller stages, i.e. more bytes in flight.
-    const uint32_t b_panel_bytes = (uint32_t)wide * UNIT_BYTES;         // one panel of all units of a group
-    const uint32_t a_stage_bytes = (uint32_t)kp * A_STAGE_BYTES, b_stage_bytes = (uint32_t)kp * b_panel_bytes;
-    const uint32_t stage_bytes = a_stage_bytes + b_stage_bytes;
-    const int STAGES = min(SS_MAX_STAGES, (int)(g.stage_area / stage_bytes));
+    const int STAGES = g.stages;
     const uint32_t sA = smem_u32(smem);
-    const uint32_t sB = sA + STAGES * a_stage_bytes;
-    const uint32_t sG = sA + g.stage_area;
+    const uint32_t sB = sA + STAGES * A_STEP;
+    const uint32_t stage_area = (uint32_t)STAGES * (A_STEP + B_STEP);
+    const uint32_t sG = sA + stage_area;
     const uint32_t gather_bytes = (uint32_t)g.C * 128u * (uint32_t)g.RP * 4u;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + g.stage_area + gather_bytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_area + gather_bytes);
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * SS_MAX_STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * SS_MAX_STAGES;
-    const uint32_t bar_tempty = bar_tfull + 16;
-    const uint32_t bar_drain = bar_tempty + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SS_MAX_STAGES + 5);
+    const uint32_t bar_drain = bar_tfull + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SS_MAX_STAGES + 2);
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (threadIdx.x == 0) {
@@ -140,17 +131,17 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_co
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_tfull + 8 * b, 1);
-            mbar_init(bar_tempty + 8 * b, 4);
-        }
+        mbar_init(bar_tfull, 1);
         mbar_init(bar_drain, 1);
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        prefetch_tmap(tmSrc);
-        for (int i = 0; i < 5; ++i) prefetch_tmap(&tmStore.m[i]);
+        prefetch_tmap(&tmSrc);
+        for (int i = 0; i < 4; ++i) prefetch_tmap(&tmStore.m[i]);
     }
+    // items per tile, then their exclusive scan (one warp, five tiles per lane)
+    for (int m = threadIdx.x; m < SS_MAX_TILES; m += SS_THREADS)
+        s_first[m] = m < g.num_m_tiles ? (g.tile_nunits[m >> 1] + SS_SUB_UNITS - 1) / SS_SUB_UNITS : 0;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(TMEM_COLS)
@@ -159,163 +150,192 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
+    if (warp == 2) {
+        constexpr int PER = SS_MAX_TILES / 32;
+        int c[PER], sum = 0;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) { c[i] = s_first[lane * PER + i]; sum += c[i]; }
+        int inc = sum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        int run = inc - sum;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) { s_first[lane * PER + i] = run; run += c[i]; }
+        if (lane == 31) s_first[SS_MAX_TILES] = inc;
+    }
+    __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const int num_items = s_first[SS_MAX_TILES];
+    const int num_steps = (g.num_kb + KP - 1) / KP;
+    const int ks0 = (int)((int64_t)crank * num_steps / g.C), ks1 = (int)((int64_t)(crank + 1) * num_steps / g.C);
 
-    // per-row routing (epilogue threads): the row's units within the tile's list
-    const int q = warp & 3;
-    const int rl = q * 32 + lane;                            // row within the tile
-    const int row = m * BM + rl;
-    int uo = -1, nu = 0;
-    float sc = 0.f;
-    if (warp >= 2 && row < g.T && nun > 0) {
-        const int t = g.tok_slot[row];
-        const int r = (t >= 0 && t < g.cap) ? g.d_rank[t] : 0;
-        if (r > 0) {
-            uo = g.tok_uoff[row];
-            nu = (r + 15) >> 4;
-            sc = g.d_scale[t];
+    // role-local pipeline state lives across items
+    uint32_t p_s = 0, p_ph = 0, p_it = 0;     // producer
+    uint32_t m_s = 0, m_ph = 0;               // MMA issuer
+    uint32_t done = 0;                        // items finished by this cluster (parity of bar_tfull)
+    bool ok = true;
+
+    for (int item = cid; item < num_items; item += ncl, ++done) {
+        // item -> (tile, sub-group): the last tile whose first item is <= item
+        int lo = 0, hi = g.num_m_tiles - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_first[mid] <= item) lo = mid; else hi = mid - 1;
         }
-    }
+        const int m = lo, u0 = (item - s_first[lo]) * SS_SUB_UNITS;
+        const int nun = g.tile_nunits[m >> 1];
+        const int nug = min(SS_SUB_UNITS, nun - u0);
+        const int32_t* units = g.tile_units + (size_t)(m >> 1) * g.umax + u0;
 
-    if (warp == 0) {
-        if (lane == 0) {   // ---- TMA producer: this CTA's slice of the contraction, once per unit group
-            uint32_t it = 0, s = 0, ph = 0;
-            bool ok = true;
-            for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS) {
-                const int nug = min(SS_GROUP_UNITS, nun - g0);
-                const int nruns = ss_plan_runs(units + g0, nug, s_runs);
-                for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 51))) break;
-                    const uint32_t full = bar_full + 8 * s;
-                    mbar_expect_tx(full, a_stage_bytes + kp * nug * UNIT_BYTES);
-                    tma_load_3d(sA + s * a_stage_bytes, tmSrc, full, 0, m * BM, kb * kp);
-                    for (int p = 0; p < kp; ++p)
+        // per-row routing (epilogue threads): the row's units within the tile's list
+        const int q = warp & 3;
+        const int rl = q * 32 + lane;
+        const int row = m * BM + rl;
+        int uo = -1, nu = 0;
+        float sc = 0.f;
+        if (warp >= 2 && row < g.T) {
+            const int t = g.tok_slot[row];
+            const int r = (t >= 0 && t < g.cap) ? g.d_rank[t] : 0;
+            if (r > 0) {
+                uo = g.tok_uoff[row];
+                nu = (r + 15) >> 4;
+                sc = g.d_scale[t];
+            }
+        }
+
+        if (warp == 0) {
+            if (lane == 0 && ok) {   // ---- TMA producer: this CTA's slice of the contraction
+                const int nruns = ss_plan_runs(units, nug, s_runs);
+                for (int ks = ks0; ks < ks1 && ok; ++ks, ++p_it) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * p_s, p_ph ^ 1, abort_word, 51))) break;
+                    const uint32_t full = bar_full + 8 * p_s;
+                    mbar_expect_tx(full, A_STEP + KP * nug * UNIT_BYTES);
+                    tma_load_3d(sA + p_s * A_STEP, &tmSrc, full, 0, m * BM, ks * KP);
+                    for (int p = 0; p < KP; ++p)
                         for (int i = 0; i < nruns; ++i)
-                            tma_load_2d(sB + s * b_stage_bytes + p * b_panel_bytes + s_runs[i].pos * UNIT_BYTES,
-                                        &tmStore.m[s_runs[i].lg], full, (kb * kp + p) * BK, s_runs[i].row);
-                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+                            tma_load_2d(sB + p_s * B_STEP + p * B_PANEL + s_runs[i].pos * UNIT_BYTES, &tmStore.m[s_runs[i].lg],
+                                        full, (ks * KP + p) * BK, s_runs[i].row);
+                    if (++p_s == (uint32_t)STAGES) { p_s = 0; p_ph ^= 1; }
                 }
             }
-            if (!ok) {
-                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
-                for (uint32_t j = 0; j < back; ++j) {
-                    const uint32_t jt = it - 1 - j;
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_full + 8 * (jt % (uint32_t)STAGES), (jt / (uint32_t)STAGES) & 1) &&
-                           global_ns() - t0 < WAIT_LIMIT_NS) {
-                    }
-                }
-            }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        if (lane == 0) {   // ---- MMA issuer
-            uint32_t s = 0, ph = 0, lt = 0;
-            bool ok = true;
-            for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS, ++lt) {
-                const int nug = min(SS_GROUP_UNITS, nun - g0);
+            __syncwarp();
+        } else if (warp == 1) {
+            if (lane == 0 && ok) {   // ---- MMA issuer
                 const uint32_t idesc = make_idesc(nug * 16, 0);
-                const uint32_t b = lt & 1, aph = (lt >> 1) & 1;
-                if (!(ok = mbar_wait(bar_tempty + 8 * b, aph ^ 1, abort_word, 53))) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + b * 256;
                 uint32_t acc = 0;
-                for (int kb = kb0; kb < kb1 && ok; ++kb) {
-                    if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 54))) break;
+                for (int ks = ks0; ks < ks1 && ok; ++ks) {
+                    if (!(ok = mbar_wait(bar_full + 8 * m_s, m_ph, abort_word, 54))) break;
                     tc_fence_after();
-                    const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
-                    for (int p = 0; p < kp; ++p) {
-                        // descriptors of successive 16-deep slices differ only in the start-address field (16-byte units)
-                        const uint64_t da0 = desc_k_major(a0 + p * A_STAGE_BYTES), db0 = desc_k_major(b0 + p * b_panel_bytes);
+                    const uint32_t a0 = sA + m_s * A_STEP, b0 = sB + m_s * B_STEP;
+#pragma unroll
+                    for (int p = 0; p < KP; ++p) {
+                        const uint64_t da0 = desc_k_major(a0 + p * A_STAGE_BYTES), db0 = desc_k_major(b0 + p * B_PANEL);
 #pragma unroll
                         for (int j = 0; j < BK / 16; ++j) {
-                            tc_mma_bf16(d_tmem, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(2 * j), idesc, acc);
+                            tc_mma_bf16(tmem_base, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(2 * j), idesc, acc);
                             acc = 1;
                         }
                     }
-                    tc_commit(bar_empty + 8 * s);
-                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+                    tc_commit(bar_empty + 8 * m_s);
+                    if (++m_s == (uint32_t)STAGES) { m_s = 0; m_ph ^= 1; }
                 }
-                if (ok) tc_commit(bar_tfull + 8 * b);
+                if (ok) tc_commit(bar_tfull);
             }
-            if (!ok) {
-                tc_commit(bar_drain);
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bar_drain, 0) && global_ns() - t0 < WAIT_LIMIT_NS) {
-                }
-            }
-        }
-        __syncwarp();
-    } else {
-        // ---- epilogue: this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
-        const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)g.RP) * 4u;
-        uint32_t lt = 0;
-        bool ok = true;
-        for (int g0 = 0; g0 < nun && ok; g0 += SS_GROUP_UNITS, ++lt) {
-            const int nug = min(SS_GROUP_UNITS, nun - g0);
-            const uint32_t b = lt & 1, aph = (lt >> 1) & 1;
-            ok = mbar_wait(bar_tfull + 8 * b, aph, abort_word, 56);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll 1
-            for (int u = 0; u < nug; ++u) {
-                uint32_t v[16];
-                ss_tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + b * 256 + u * 16, v);
-                tc_wait_ld();
-                const int gu = g0 + u;
-                if (uo >= 0 && gu >= uo && gu < uo + nu) {
-                    const uint32_t a = gdst + (uint32_t)(gu - uo) * 64u;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        ss_st_cluster_v4(a + e * 16, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-                }
-            }
-            tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * b);
-        }
-    }
-
-    // ---- every CTA's partial vectors are in CTA 0: add them in rank order and write the results ----------------
-    tc_fence_before();
-    __syncthreads();
-    ss_cluster_sync();
-    if (crank == 0 && warp >= 2 && row < g.T && *abort_word == 0) {
-        const float* gbuf = reinterpret_cast<const float*>(smem + g.stage_area);
-        bf16* hrow = g.hd + (size_t)row * g.hd_cols;
-        for (int gu = 0; gu < nun; ++gu) {
-            uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
-            if (uo >= 0 && gu >= uo && gu < uo + nu) {
-                float v[16];
+        } else {
+            // ---- epilogue: this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
+            bool eok = mbar_wait(bar_tfull, done & 1, abort_word, 56);
+            eok = __all_sync(0xffffffffu, eok);
+            ok = eok;
+            if (eok) {
+                tc_fence_after();
+                const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)g.RP) * 4u;
+                const bool empty_slice = ks0 >= ks1;      // no step: the accumulator was never written
+#pragma unroll 1
+                for (int u = 0; u < nug; ++u) {
+                    uint32_t v[16];
+                    ss_tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + u * 16, v);
+                    tc_wait_ld();
+                    const int gu = u0 + u;
+                    if (uo >= 0 && gu >= uo && gu < uo + nu) {
+                        const uint32_t a = gdst + (uint32_t)(gu - uo) * 64u;
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = 0.f;
-                for (int c = 0; c < g.C; ++c) {      // fixed order
-                    const float4* p = reinterpret_cast<const float4*>(gbuf + ((size_t)c * 128 + rl) * g.RP + (gu - uo) * 16);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float4 t4 = p[e];
-                        v[4 * e] += t4.x; v[4 * e + 1] += t4.y; v[4 * e + 2] += t4.z; v[4 * e + 3] += t4.w;
+                        for (int e = 0; e < 4; ++e) {
+                            if (empty_slice) ss_st_cluster_v4(a + e * 16, 0u, 0u, 0u, 0u);
+                            else ss_st_cluster_v4(a + e * 16, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                        }
                     }
                 }
-                __nv_bfloat162 pk[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) pk[e] = __floats2bfloat162_rn(sc * v[2 * e], sc * v[2 * e + 1]);
-                o0 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[0]), *reinterpret_cast<uint32_t*>(&pk[1]),
-                                *reinterpret_cast<uint32_t*>(&pk[2]), *reinterpret_cast<uint32_t*>(&pk[3]));
-                o1 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[4]), *reinterpret_cast<uint32_t*>(&pk[5]),
-                                *reinterpret_cast<uint32_t*>(&pk[6]), *reinterpret_cast<uint32_t*>(&pk[7]));
-                float4* dst = reinterpret_cast<float4*>(g.out + (size_t)row * g.RP + (gu - uo) * 16);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
             }
-            uint4* hdst = reinterpret_cast<uint4*>(hrow + gu * 16);
-            hdst[0] = o0;
-            hdst[1] = o1;
         }
+
+        // ---- every CTA's partial vectors are in CTA 0: add them in rank order and write the results ------------
+        tc_fence_before();
+        __syncthreads();
+        ss_cluster_sync();
+        tc_fence_after();
+        if (crank == 0 && warp >= 2 && row < g.T && ok) {
+            const float* gbuf = reinterpret_cast<const float*>(smem + stage_area);
+            bf16* hrow = g.hd + (size_t)row * g.hd_cols;
+            for (int u = 0; u < nug; ++u) {
+                const int gu = u0 + u;
+                uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
+                if (uo >= 0 && gu >= uo && gu < uo + nu) {
+                    float v[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = 0.f;
+                    for (int c = 0; c < g.C; ++c) {      // fixed order
+                        const float4* p = reinterpret_cast<const float4*>(gbuf + ((size_t)c * 128 + rl) * g.RP + (gu - uo) * 16);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float4 t4 = p[e];
+                            v[4 * e] += t4.x; v[4 * e + 1] += t4.y; v[4 * e + 2] += t4.z; v[4 * e + 3] += t4.w;
+                        }
+                    }
+                    __nv_bfloat162 pk[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) pk[e] = __floats2bfloat162_rn(sc * v[2 * e], sc * v[2 * e + 1]);
+                    o0 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[0]), *reinterpret_cast<uint32_t*>(&pk[1]),
+                                    *reinterpret_cast<uint32_t*>(&pk[2]), *reinterpret_cast<uint32_t*>(&pk[3]));
+                    o1 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[4]), *reinterpret_cast<uint32_t*>(&pk[5]),
+                                    *reinterpret_cast<uint32_t*>(&pk[6]), *reinterpret_cast<uint32_t*>(&pk[7]));
+                    float4* dst = reinterpret_cast<float4*>(g.out + (size_t)row * g.RP + (gu - uo) * 16);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                }
+                uint4* hdst = reinterpret_cast<uint4*>(hrow + gu * 16);
+                hdst[0] = o0;
+                hdst[1] = o1;
+            }
+        }
+        // the gather buffer and the accumulator are free for the cluster's next item
+        tc_fence_before();
+        ss_cluster_sync();
+        tc_fence_after();
     }
 
+    // ---- teardown ---------------------------------------------------------------------------------------------
+    if (threadIdx.x == 0 && *abort_word != 0) {
+        // let the copies already issued land (bounded) before shared memory is released
+        const uint32_t back = p_it < (uint32_t)STAGES ? p_it : (uint32_t)STAGES;
+        for (uint32_t j = 0; j < back; ++j) {
+            const uint32_t jt = p_it - 1 - j;
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bar_full + 8 * (jt % (uint32_t)STAGES), (jt / (uint32_t)STAGES) & 1) &&
+                   global_ns() - t0 < WAIT_LIMIT_NS) {
+            }
+        }
+    }
+    if (warp == 1 && lane == 0 && *abort_word != 0) {
+        tc_commit(bar_drain);
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(bar_drain, 0) && global_ns() - t0 < WAIT_LIMIT_NS) {
+        }
+    }
+    tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
@@ -327,19 +347,21 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc1, const __grid_co
 
 }  // namespace sm100
 
-// Cluster width for T tokens: as many CTAs per tile as keep the whole grid resident in one wave (0 = this kernel
-// does not apply: more tiles than SMs, where the persistent one-CTA-per-tile kernel is the better fit).
-static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, size_t* smem_out, uint32_t* area_out) {
+// Cluster width for T tokens: as many CTAs per tile as keep one cluster per tile resident in a single wave (0 = this
+// kernel does not apply: more tiles than SMs, where the persistent one-CTA-per-tile kernel is the better fit).
+static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, size_t* smem_out, int* stages_out,
+                       int* clusters_out) {
     using namespace sm100;
-    if (tiles > pool->sm_count) return 0;
+    if (tiles > pool->sm_count || tiles > SS_MAX_TILES) return 0;
     static int max_active[64][SS_MAX_C + 1] = {};
     for (int C = SS_MAX_C; C >= 1; --C) {
         if ((int64_t)C * tiles > pool->sm_count || (C > 1 && num_kb < 16 * C)) continue;
         const size_t gather = (size_t)C * 128 * pool->RP * 4;
         const size_t avail = 222 * 1024 - 1024 - 256;
-        if (gather + 2 * SS_STAGE_BYTES > avail) continue;
-        const size_t area = (avail - gather) / 1024 * 1024;
-        const size_t smem = 1024 + area + gather + 256;
+        if (gather + 2 * SS_STEP_BYTES > avail) continue;
+        int stages = (int)((avail - gather) / SS_STEP_BYTES);
+        if (stages > SS_MAX_STAGES) stages = SS_MAX_STAGES;
+        const size_t smem = 1024 + (size_t)stages * SS_STEP_BYTES + gather + 256;
         int mc = pool->device < 64 ? max_active[pool->device][C] : 0;
         if (mc == 0) {
             if (cudaFuncSetAttribute(k_shrink_split_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024) != cudaSuccess) return 0;
@@ -357,15 +379,16 @@ static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, 
         }
         if (mc < tiles) continue;
         *smem_out = smem;
-        *area_out = (uint32_t)area;
+        *stages_out = stages;
+        *clusters_out = mc < pool->sm_count / C ? mc : pool->sm_count / C;     // all resident clusters walk the item list
         return C;
     }
     return 0;
 }
 
 bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D) {
-    size_t smem; uint32_t area;
-    return T > 0 && (D % 64) == 0 && split_width(pool, cdiv(T, sm100::BM), cdiv(D, sm100::BK), &smem, &area) > 0;
+    size_t smem; int stages, clusters;
+    return T > 0 && (D % 64) == 0 && split_width(pool, cdiv(T, sm100::BM), cdiv(D, sm100::BK), &smem, &stages, &clusters) > 0;
 }
 
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
@@ -374,30 +397,29 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     if (T <= 0) return MARLAAS_OK;
     const int64_t tiles = cdiv(T, BM);
     size_t smem_bytes = 0;
-    uint32_t area = 0;
-    const int C = split_width(pool, tiles, cdiv(D, BK), &smem_bytes, &area);
+    int stages = 0, clusters = 0;
+    const int C = split_width(pool, tiles, cdiv(D, BK), &smem_bytes, &stages, &clusters);
     if (C <= 0) return fail(MARLAAS_ERR_INVALID_ARG, "shrink_split: %lld tiles do not fit one wave", (long long)tiles);
     ShrinkSplitArgs g;
     g.T = (int)T; g.D = (int)D;
     g.num_kb = (int)cdiv(D, BK);
+    g.num_m_tiles = (int)tiles;
     g.RP = pool->RP; g.cap = pool->cap;
-    g.C = C; g.stage_area = area;
+    g.C = C; g.stages = stages;
     g.tok_slot = ws.tok_slot; g.tok_uoff = ws.tok_uoff;
     g.tile_nunits = ws.tile_nunits; g.tile_units = ws.tile_units; g.umax = ws.umax;
     g.d_rank = pool->d_rank; g.d_scale = pool->d_scale;
     g.out = out; g.hd = ws.hd; g.hd_cols = ws.umax * 16;
     g.status = pool->d_status;
-    alignas(64) CUtensorMap tmSrc1, tmSrc2, tmSrc4;
+    alignas(64) CUtensorMap tmSrc;
     alignas(64) StoreMaps maps;
     marlaas_status_t rc;
-    if ((rc = make_panel_map(&tmSrc1, src, T, D, ld, 1)) != MARLAAS_OK) return rc;
-    if ((rc = make_panel_map(&tmSrc2, src, T, D, ld, 2)) != MARLAAS_OK) return rc;
-    if ((rc = make_panel_map(&tmSrc4, src, T, D, ld, 4)) != MARLAAS_OK) return rc;
-    for (int i = 0; i < 5; ++i)
+    if ((rc = make_panel_map(&tmSrc, src, T, D, ld, SS_KP)) != MARLAAS_OK) return rc;
+    for (int i = 0; i < 4; ++i)
         if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, D, BK, 16u << i)) != MARLAAS_OK) return rc;
     MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(tiles * C));
+    cfg.gridDim = dim3((unsigned)(clusters * C));
     cfg.blockDim = dim3(SS_THREADS);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
@@ -405,7 +427,7 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_shrink_split_sm100, tmSrc1, tmSrc2, tmSrc4, maps, g));
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_shrink_split_sm100, tmSrc, maps, g));
     count_launch();
     return MARLAAS_OK;
 }
