@@ -1,0 +1,71 @@
+"""GPU parity at the full configured sizes, through the same calls bench.py times (forward with h_save, backward with
+the saved h).  The oracle is too slow for every output row at these sizes, so y and dx are checked on sampled token
+rows (each row of the oracle is computed on its own, from the definition), while the adapter gradients, which sum
+over every token of a tenant, are checked in full.  Index outputs are compared bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_08527_b200 import binding as B
+from paper_2605_08527_b200 import workloads as wl
+
+from helpers import DeviceCase, assert_close, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_rows(T, n, seed):
+    edge = [0, 1, 63, 64, 127, 128, 255, 256, 257, T // 2, T - 257, T - 256, T - 129, T - 128, T - 2, T - 1]
+    rnd = (wl.hash_u64(seed, wl.TID_PERTURB, np.arange(n, dtype=np.uint64)) % np.uint64(T)).astype(np.int64)
+    rows = sorted({int(r) for r in edge if 0 <= r < T} | {int(r) for r in rnd})
+    return np.array(rows, dtype=np.int64)
+
+
+def _check_full(w, p, n_rows=40):
+    ts = w.tok_slot()
+    r, s, A, Bm = oracle.adapters_of(p)
+    dc = DeviceCase(w, p)
+    T, Tb = w.T, w.T_bwd
+    hs = torch.empty((T, dc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+    y = dc.forward(h_save=hs)
+    rows = _sample_rows(T, n_rows, 7 + len(p.name))
+    ry, rh = oracle.forward(p.x[rows], p.W, r, s, A, Bm, ts[rows])
+    assert_close(to_np(y[torch.from_numpy(rows).cuda()]), ry, f"{w.name}/{p.name} y (sampled rows)")
+    hr = np.zeros((len(rows), dc.pool.rank_stride), np.float32)
+    hr[:, :rh.shape[1]] = rh
+    assert_close(to_np(hs[torch.from_numpy(rows).cuda()]), hr, f"{w.name}/{p.name} h_save (sampled rows)", atol=1e-3, rtol=1e-3)
+    if Tb:
+        seg = dc.seg if Tb == T else dc.seg_prefix(Tb)
+        dx, dA, dB = dc.backward(seg=seg, T=Tb, h_saved=hs[:Tb])
+        rb = rows[rows < Tb]
+        rdx, _ = oracle.backward_dx(p.dy[rb], p.W, r, s, A, Bm, ts[rb])
+        assert_close(to_np(dx[torch.from_numpy(rb).cuda()]), rdx, f"{w.name}/{p.name} dx (sampled rows)")
+        rdA, rdB = oracle.backward_dAdB(p.x[:Tb], p.dy[:Tb], r, s, A, Bm, ts[:Tb])
+        for t, a in enumerate(p.adapters):
+            if a.rank > 0:
+                assert_close(to_np(dA[t]), rdA[t], f"{w.name}/{p.name} dA[{t}]")
+                assert_close(to_np(dB[t]), rdB[t], f"{w.name}/{p.name} dB[{t}]")
+    exp = oracle.build_index(T, w.seg_offsets, w.seg_slot, dc.capacity)
+    got = B.marlaas_lora_build_index(dc.pool, T, dc.seg)
+    for g_, e, nm in zip(got, exp, ("tok_slot", "slot_count", "slot_offset", "perm")):
+        assert np.array_equal(g_.cpu().numpy(), e), (w.name, nm)
+    B.marlaas_check_status(dc.pool)
+
+
+def test_cfg3_training_shaped_full_size():
+    w = wl.make_workload(3)
+    _check_full(w, w.projections[0])
+
+
+def test_cfg4_heterogeneous_full_size():
+    w = wl.make_workload(4)
+    _check_full(w, w.projections[0])
+
+
+def test_cfg5_decoder_layer_full_size():
+    w = wl.make_workload(5)
+    for p in w.projections:
+        _check_full(w, p, n_rows=24)
+        torch.cuda.empty_cache()
