@@ -35,7 +35,10 @@ NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed ncu captures
 # (profiles/); None where the kernel has changed since its counters were taken.
-TRAFFIC = {}
+TRAFFIC = {
+    "cfg3": 1.60e9,    # k_gemm2_sm100, mean of the forward (1.30 GB) and dx (1.90 GB) launches: profiles/gemm2_sm100_cfg3_ncu_full.txt
+    "cfg2": 46.5e6,    # k_decode_shrink (6.3 MB) + k_decode_gemm (40.2 MB) of one call: profiles/decode_cfg2_ncu_full.txt
+}
 CFG_OF = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
 CFG_DESC = {
     "cfg1": "tiny: W 512x512, 4 tenants r=8, 256 tokens, fwd+bwd",
@@ -182,7 +185,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg3", choices=sorted(CFG_OF))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -399,6 +402,7 @@ def main():
                     "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)",
                     "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms, "flops_per_launch": flops_per_launch,
                     "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
+                    "frac_of_measured_sustained": ach / peaks["bf16_tflops_sustained"],
                     "whole_step_tflops": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12,
                     "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
 
