@@ -397,14 +397,21 @@ def main():
                     "frac_of_nominal_8TBs": ach / NOMINAL["hbm_gbs"]}
     else:
         ach = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12 if gemm_n else 0.0
-        roofline = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["bf16_tflops"], "traffic": TRAFFIC.get(args.workload), "peak_source": f"of {peak_src} (burst)",
+        # The GEMM launches are timed inside the step loop.  When that loop ran power-capped (SM clock well under its
+        # maximum with sw_power_cap active) the matching denominator is the sustained cuBLAS figure, otherwise the burst one.
+        capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and "sw_power_cap" in clocks.get("reasons", [])
+                      and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
+        peak_t = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+        roofline = {"bound": "tensor", "achieved": ach, "peak": peak_t, "unit": "TFLOP/s",
+                    "frac": ach / peak_t, "traffic": TRAFFIC.get(args.workload),
+                    "peak_source": f"of {peak_src} ({'sustained: the timed loop ran power-capped' if capped else 'burst'})",
+                    "frac_of_measured_burst": ach / peaks["bf16_tflops"],
                     "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)",
                     "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms, "flops_per_launch": flops_per_launch,
                     "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
                     "frac_of_measured_sustained": ach / peaks["bf16_tflops_sustained"],
                     "whole_step_tflops": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12,
-                    "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+                    "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peak_t}
 
     # ---- end to end: host inputs -> device -> layer -> host outputs, all inside the timed region ------------
     e2e = None

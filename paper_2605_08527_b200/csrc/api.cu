@@ -113,8 +113,10 @@ static marlaas_status_t make_plan(const marlaas_pool* pool, int64_t T, const mar
 // Shrink for the tensor-core path: batches with several 128-token tiles go through the tcgen05 kernel, small
 // (decode-shaped) batches through the per-token gather kernel, which spreads over more SMs.
 static marlaas_status_t shrink(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                               const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
-    if (T >= 512 && shrink_split_sm100_eligible(pool, T, D)) return launch_shrink_split_sm100(pool, T, src, ld, D, store, ws, out, st);
+                               const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                               bool out_is_zero = false) {
+    if (T >= 512 && shrink_split_sm100_eligible(pool, T, D))
+        return launch_shrink_split_sm100(pool, T, src, ld, D, store, ws, out, st, out_is_zero);
     if (T >= 512) return launch_shrink_sm100(pool, T, src, ld, D, store, ws, out, st);
     return launch_shrink_hd(pool, T, src, ld, D, store, ws, out, st);
 }
@@ -200,8 +202,12 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         return finish(pool, flags, st);
     }
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH)) {
+        // h is cleared before the plan so that plan -> shrink -> GEMM are consecutive kernels (each is launched as a
+        // programmatic dependent of the one before and overlaps its tail)
+        const bool pre_zero = T >= 512 && shrink_split_sm100_eligible(pool, T, pool->K);
+        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(h, 0, sizeof(float) * (size_t)T * pool->RP, st));
         if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
-        if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st)) != MARLAAS_OK) return rc;
+        if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st, pre_zero)) != MARLAAS_OK) return rc;
         GemmOperands o;
         o.M = T; o.Nout = pool->N; o.Kc = pool->K;
         o.A = (const bf16*)x; o.lda = ldx;
@@ -259,14 +265,16 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     const bool acc = (flags & MARLAAS_FLAG_ACCUMULATE) != 0;
 
     const bool tc_path = !(flags & MARLAAS_FLAG_CUDA_CORE_PATH);
+    const bool pre_zero = tc_path && T >= 512 && (dx || want_dA) && shrink_split_sm100_eligible(pool, T, pool->N);
     if (tc_path && T > 0) {
+        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.g, 0, sizeof(float) * (size_t)T * pool->RP, st));   // see forward
         if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
     } else {
         if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
     if (T > 0 && (dx || want_dA)) {
         if (tc_path) {
-            if ((rc = shrink(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st)) != MARLAAS_OK) return rc;
+            if ((rc = shrink(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st, pre_zero)) != MARLAAS_OK) return rc;
         } else {
             if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
         }

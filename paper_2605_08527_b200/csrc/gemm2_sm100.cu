@@ -166,7 +166,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // ================= TMA producer (both CTAs) =================
         if (lane == 0) {
             uint32_t it = 0;
-            bool ok = true;
+            bool ok = true, waited = false;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 int m_idx, n_idx;
                 decode_tile2(g, tile, m_idx, n_idx);
@@ -187,6 +187,10 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     } else if (my_n < g.Nout) {
                         tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES, &tmB, full, kb * BK, my_n);
                     }
+                }
+                if (!waited) {      // the plan and hd come from the kernels this one was launched behind
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    waited = true;
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
@@ -224,7 +228,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             constexpr uint32_t idesc_mn = make_idesc_pair(1);
             const uint32_t idesc_main = make_idesc_pair(g.b_mn);
             uint32_t it = 0, lt = 0;
-            bool ok = true;
+            bool ok = true, waited = false;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
                 int m_idx, n_idx;
                 decode_tile2(g, tile, m_idx, n_idx);
@@ -247,6 +251,10 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         acc = 1;
                     }
                     tc_commit_pair(bar_empty + 8 * s);
+                }
+                if (!waited) {
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    waited = true;
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
@@ -321,6 +329,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
 
     // ---- teardown ---------------------------------------------------------------------------------------------
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // never complete before the kernels it was launched behind
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();     // neither CTA leaves while its pair may still signal its barriers or use its operands
@@ -393,8 +402,18 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
     }
     const int tiles = g.num_m_tiles * g.num_n_tiles;
     const int pairs = tiles < mc ? tiles : mc;
-    k_gemm2_sm100<<<2 * pairs, G2_THREADS, smem_bytes, st>>>(tmA, tmB, tmXA, tmXB, g);
-    MARLAAS_LAUNCH_CHECK("k_gemm2_sm100");
+    // launched as a programmatic dependent: its main loop (x and W only) may start while the shrink's last CTAs run
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)pairs);
+    cfg.blockDim = dim3(G2_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_gemm2_sm100, tmA, tmB, tmXA, tmXB, g));
+    count_launch();
     return MARLAAS_OK;
 }
 

@@ -169,7 +169,8 @@ marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const 
 // CTAs; applies when all tiles fit one wave
 bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D);
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
+                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                                           bool out_is_zero = false);
 
 // cuda_core_kernels.cu
 // h/g (fp32, [T][RP]) as launch_rowdot, plus the bf16 block-diagonal operand rows hd for the tensor-core path

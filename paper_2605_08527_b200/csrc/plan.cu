@@ -108,6 +108,8 @@ __global__ void __launch_bounds__(256) k_plan_tiles(int T, int S, const int32_t*
                                                     int32_t* __restrict__ tile_units, int umax, int32_t* status) {
     __shared__ int s_u[4096];
     __shared__ int s_warp[8];
+    // the next kernel of the call may be launched now: it waits (griddepcontrol.wait) before it reads the plan
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = blockIdx.x;
     const int i = m * 256 + tid;

@@ -139,6 +139,10 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         prefetch_tmap(&tmSrc);
         for (int i = 0; i < 4; ++i) prefetch_tmap(&tmStore.m[i]);
     }
+    // Launched as a programmatic dependent of the plan kernel: everything above overlapped its tail; the plan's
+    // outputs are read only from here on.  The base GEMM that follows may be launched in turn.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // items per tile, then their exclusive scan (one warp, five tiles per lane)
     for (int m = threadIdx.x; m < SS_MAX_TILES; m += SS_THREADS)
         s_first[m] = m < g.num_m_tiles ? (g.tile_nunits[m >> 1] + SS_SUB_UNITS - 1) / SS_SUB_UNITS : 0;
@@ -392,7 +396,8 @@ bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D)
 }
 
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                                           bool out_is_zero) {
     using namespace sm100;
     if (T <= 0) return MARLAAS_OK;
     const int64_t tiles = cdiv(T, BM);
@@ -417,16 +422,18 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     if ((rc = make_panel_map(&tmSrc, src, T, D, ld, SS_KP)) != MARLAAS_OK) return rc;
     for (int i = 0; i < 4; ++i)
         if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, D, BK, 16u << i)) != MARLAAS_OK) return rc;
-    MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
+    if (!out_is_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * C));
     cfg.blockDim = dim3(SS_THREADS);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
     MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_shrink_split_sm100, tmSrc, maps, g));
     count_launch();
     return MARLAAS_OK;
