@@ -497,10 +497,12 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     // tensor-memory lane on both sides, [column group][lane] 16-byte slots), and the finishing warp adds them to
     // its own accumulator in ascending pair order.  The mailboxes reuse the pipeline stages.
     const int qper = 4 / g.S;
-    auto slice_steps = [&](uint32_t p) -> int {
-        return (int)((int64_t)(p + 1) * g.num_ks / g.S) - (int)((int64_t)p * g.num_ks / g.S) +
-               (int)((int64_t)(p + 1) * g.num_xs / g.S) - (int)((int64_t)p * g.num_xs / g.S);
-    };
+    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
+    uint32_t live = 0;
+    for (int p = 0; p < g.S; ++p) {
+        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
+        if (n > 0) live |= 1u << p;
+    }
     const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     const int q = warp & 3;
     const uint32_t own = (uint32_t)(q % g.S);
@@ -509,7 +511,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         __syncthreads();
         dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
         tc_fence_after();
-        if (warp >= 2 && epi_ok && own != pairi && slice_steps(pairi) > 0) {
+        if (warp >= 2 && epi_ok && own != pairi && ((live >> pairi) & 1u)) {
             const uint32_t si = pairi < own ? pairi : pairi - 1;
             const uint32_t dst = dk_map_to_cta(sA, 2 * own + half) + (si * (uint32_t)qper + (uint32_t)(q / g.S)) * box_bytes +
                                  (uint32_t)lane * 16u;
@@ -540,7 +542,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] = 0.f;
             for (uint32_t src = 0; src < (uint32_t)g.S; ++src) {      // ascending pair order
-                if (slice_steps(src) == 0) continue;                  // a slice without steps never wrote its accumulator
+                if (!((live >> src) & 1u)) continue;                  // a slice without steps never wrote its accumulator
                 if (src == pairi) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(v[e]);
