@@ -156,6 +156,21 @@ def oracle_step_sample(w, n_tok):
     return total
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time: every multi-GPU number is the maximum over ranks (replicas finish together or not at all)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling: per-rank work is fixed)."""
+    return tokens_per_rank * world / (ms_per_step * 1e-3)
+
+
 def run_reference(args, rank, world):
     """--impl reference: the CPU oracle on the host cores, a bounded sample of the workload per step."""
     if rank != 0:
@@ -359,14 +374,10 @@ def main():
         launches = None
         rep_ms = [a.elapsed_time(b) for a, b in evs]
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = float(np.median(rep_ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(np.median(rep_ms)), dist, dev)
     ms_per_step = total_ms / args.steps
     tokens_per_step = w.T * world
-    value = tokens_per_step / (ms_per_step * 1e-3)
+    value = aggregate_tokens_per_s(w.T, world, ms_per_step)
 
     # ---- dominant kernel, timed live with events on the launching stream ---------------------------------------
     for s in all_projs:
@@ -461,11 +472,7 @@ def main():
             h2d, d2h = e2e_step()
         b.record()
         barrier()
-        e_ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(a.elapsed_time(b), dist, dev)
         e2e = {"value": tokens_per_step / (e_ms / args.e2e_steps * 1e-3), "unit": "tokens/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
                "ms_per_step": e_ms / args.e2e_steps}
