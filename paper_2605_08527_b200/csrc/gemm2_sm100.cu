@@ -165,7 +165,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (warp == 0) {
         // ================= TMA producer (both CTAs) =================
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, ph = 0;     // blocks issued; stage and phase bit of the next block
             bool ok = true, waited = false;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 int m_idx, n_idx;
@@ -176,7 +176,6 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const int nchunk = half_chunks(g, n0, (int)rank);
                 const uint32_t stage_tx = main_bytes(g, m0, n0, 0) + main_bytes(g, m0, n0, 1);
                 for (int kb = 0; kb < g.num_kb && ok; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 31))) break;
                     const uint32_t full = map_to_cta(bar_full + 8 * s, 0);
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
@@ -187,6 +186,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     } else if (my_n < g.Nout) {
                         tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES, &tmB, full, kb * BK, my_n);
                     }
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
                 if (!waited) {      // the plan and hd come from the kernels this one was launched behind
                     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -194,7 +194,6 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 32))) break;
                     const uint32_t full = map_to_cta(bar_full + 8 * s, 0);
                     const int nv = min(4, nun - x0);
@@ -207,6 +206,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES + c * CHUNK_BYTES + u * UNIT_BYTES, &tmXB, full,
                                              my_n + c * 64, row);
                     }
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
             }
             if (!ok && rank == 0) {
@@ -227,8 +227,13 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc_mn = make_idesc_pair(1);
             const uint32_t idesc_main = make_idesc_pair(g.b_mn);
-            uint32_t it = 0, lt = 0;
+            uint32_t lt = 0, s = 0, ph = 0;     // stage and phase bit of the next k-block (running counters: no division)
             bool ok = true, waited = false;
+            // descriptors of a stage's operands differ from stage 0's, and those of successive 16-deep slices from the
+            // first slice's, only in the start-address field (16-byte units): they are stepped, not rebuilt
+            const uint64_t da_base = desc_k_major(sA);
+            const uint64_t db_base = g.b_mn ? desc_mn_major(sB, CHUNK_BYTES) : desc_k_major(sB);
+            const uint64_t db_step = g.b_mn ? (uint64_t)(UNIT_BYTES >> 4) : 2ull;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
                 int m_idx, n_idx;
                 decode_tile2(g, tile, m_idx, n_idx);
@@ -237,28 +242,25 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * G2_BN;
                 uint32_t acc = 0;
-                for (int kb = 0; kb < g.num_kb && ok; ++kb, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int kb = 0; kb < g.num_kb && ok; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 34))) break;
                     tc_fence_after();
-                    const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * G2_B_STAGE_BYTES;
+                    const uint64_t da = da_base + (uint64_t)(s * (A_STAGE_BYTES >> 4));
+                    const uint64_t db = db_base + (uint64_t)(s * (G2_B_STAGE_BYTES >> 4));
 #pragma unroll
                     for (int j = 0; j < BK / 16; ++j) {
-                        const uint64_t da = desc_k_major(a0 + j * 32);
-                        const uint64_t db = g.b_mn ? desc_mn_major(b0 + j * UNIT_BYTES, CHUNK_BYTES)
-                                                   : desc_k_major(b0 + j * 32);
-                        tc_mma_bf16_pair(d_tmem, da, db, idesc_main, acc);
+                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * j), db + (uint64_t)j * db_step, idesc_main, acc);
                         acc = 1;
                     }
                     tc_commit_pair(bar_empty + 8 * s);
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
                 if (!waited) {
                     asm volatile("griddepcontrol.wait;" ::: "memory");
                     waited = true;
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
-                for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int x0 = 0; x0 < nun && ok; x0 += 4) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 35))) break;
                     tc_fence_after();
                     const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * G2_B_STAGE_BYTES;
@@ -269,6 +271,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         acc = 1;
                     }
                     tc_commit_pair(bar_empty + 8 * s);
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
                 if (ok) tc_commit_pair(bar_tfull + 8 * b);
             }
