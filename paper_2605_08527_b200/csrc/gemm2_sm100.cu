@@ -167,6 +167,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (lane == 0) {
             uint32_t it = 0, s = 0, ph = 0;     // blocks issued; stage and phase bit of the next block
             bool ok = true, waited = false;
+            const uint32_t full0 = map_to_cta(bar_full, 0);      // the leader's full barriers (8 bytes apart)
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 int m_idx, n_idx;
                 decode_tile2(g, tile, m_idx, n_idx);
@@ -177,7 +178,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint32_t stage_tx = main_bytes(g, m0, n0, 0) + main_bytes(g, m0, n0, 1);
                 for (int kb = 0; kb < g.num_kb && ok; ++kb, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 31))) break;
-                    const uint32_t full = map_to_cta(bar_full + 8 * s, 0);
+                    const uint32_t full = full0 + 8 * s;
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
                     if (have_rows) tma_load_2d_pair(sA + s * A_STAGE_BYTES, &tmA, full, kb * BK, my_m);
                     if (g.b_mn) {
@@ -195,7 +196,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 32))) break;
-                    const uint32_t full = map_to_cta(bar_full + 8 * s, 0);
+                    const uint32_t full = full0 + 8 * s;
                     const int nv = min(4, nun - x0);
                     if (rank == 0)
                         mbar_expect_tx(bar_full + 8 * s, extra_bytes(g, m0, n0, 0, nv) + extra_bytes(g, m0, n0, 1, nv));
@@ -244,7 +245,6 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 uint32_t acc = 0;
                 for (int kb = 0; kb < g.num_kb && ok; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 34))) break;
-                    tc_fence_after();
                     const uint64_t da = da_base + (uint64_t)(s * (A_STAGE_BYTES >> 4));
                     const uint64_t db = db_base + (uint64_t)(s * (G2_B_STAGE_BYTES >> 4));
 #pragma unroll
