@@ -96,27 +96,39 @@ __device__ __forceinline__ void decode_tile2(const Gemm2Args& g, int tile, int& 
 __device__ __forceinline__ int half_chunks(const Gemm2Args& g, int n0, int r) {
     return max(0, min(2, (g.Nout - (n0 + r * 128) + 63) / 64));
 }
-__device__ __forceinline__ uint32_t main_bytes(const Gemm2Args& g, int m0, int n0, int r) {
+__device__ __forceinline__ uint32_t main_bytes(const Gemm2Args& g, int m0, int n0, int r, uint32_t kp) {
     const uint32_t a = (m0 + r * 128 < g.M) ? A_STAGE_BYTES : 0u;
     const uint32_t b = g.b_mn ? (uint32_t)half_chunks(g, n0, r) * CHUNK_BYTES
                               : ((n0 + r * 128 < g.Nout) ? G2_B_STAGE_BYTES : 0u);
-    return a + b;
+    return kp * (a + b);      // kp 64-deep panels per pipeline step
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0,
+                                                 int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
 }
 __device__ __forceinline__ uint32_t extra_bytes(const Gemm2Args& g, int m0, int n0, int r, int nv) {
     const uint32_t a = (m0 + r * 128 < g.M) ? A_STAGE_BYTES : 0u;
     return a + (uint32_t)(nv * half_chunks(g, n0, r)) * UNIT_BYTES;
 }
 
+// KP = 64-deep panels per pipeline step.  KP = 2 (contraction depth a multiple of 64): x / dy and a K-major W are viewed as
+// 3-D tensors so that ONE TMA instruction brings both panels, and the barrier wait / expect / commit of the two issuing
+// threads is paid once per 128 of depth; KP = 1 is the plain 2-D form for any depth.
+template <int KP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(G2_THREADS, 1)
 k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
               const __grid_constant__ CUtensorMap tmXA, const __grid_constant__ CUtensorMap tmXB, const Gemm2Args g) {
-    constexpr int STAGES = G2_STAGES;
+    constexpr int STAGES = G2_STAGES / KP;
+    constexpr uint32_t A_ST = KP * A_STAGE_BYTES, B_ST = KP * G2_B_STAGE_BYTES;
     constexpr uint32_t TMEM_COLS = 512;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sA = smem_u32(smem);
-    const uint32_t sB = sA + STAGES * A_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * G2_STAGE_BYTES);
+    const uint32_t sB = sA + STAGES * A_ST;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_ST + B_ST));
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;
@@ -175,17 +187,21 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const int my_m = m0 + (int)rank * 128, my_n = n0 + (int)rank * 128;
                 const bool have_rows = my_m < g.M;
                 const int nchunk = half_chunks(g, n0, (int)rank);
-                const uint32_t stage_tx = main_bytes(g, m0, n0, 0) + main_bytes(g, m0, n0, 1);
+                const uint32_t stage_tx = main_bytes(g, m0, n0, 0, KP) + main_bytes(g, m0, n0, 1, KP);
                 for (int kb = 0; kb < g.num_kb && ok; ++kb, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 31))) break;
                     const uint32_t full = full0 + 8 * s;
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
-                    if (have_rows) tma_load_2d_pair(sA + s * A_STAGE_BYTES, &tmA, full, kb * BK, my_m);
-                    if (g.b_mn) {
+                    if (have_rows) {
+                        if (KP == 1) tma_load_2d_pair(sA + s * A_ST, &tmA, full, kb * BK, my_m);
+                        else tma_load_3d_pair(sA + s * A_ST, &tmA, full, 0, my_m, kb * KP);
+                    }
+                    if (g.b_mn) {      // box: 64 columns x (KP * 64) rows of W
                         for (int c = 0; c < nchunk; ++c)
-                            tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES + c * CHUNK_BYTES, &tmB, full, my_n + c * 64, kb * BK);
+                            tma_load_2d_pair(sB + s * B_ST + c * (KP * CHUNK_BYTES), &tmB, full, my_n + c * 64, kb * KP * BK);
                     } else if (my_n < g.Nout) {
-                        tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES, &tmB, full, kb * BK, my_n);
+                        if (KP == 1) tma_load_2d_pair(sB + s * B_ST, &tmB, full, kb * BK, my_n);
+                        else tma_load_3d_pair(sB + s * B_ST, &tmB, full, 0, my_n, kb * KP);
                     }
                     if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
@@ -200,11 +216,11 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const int nv = min(4, nun - x0);
                     if (rank == 0)
                         mbar_expect_tx(bar_full + 8 * s, extra_bytes(g, m0, n0, 0, nv) + extra_bytes(g, m0, n0, 1, nv));
-                    if (have_rows) tma_load_2d_pair(sA + s * A_STAGE_BYTES, &tmXA, full, x0 * 16, my_m);
+                    if (have_rows) tma_load_2d_pair(sA + s * A_ST, &tmXA, full, x0 * 16, my_m);
                     for (int u = 0; u < nv; ++u) {
                         const int row = g.tile_units[(size_t)m_idx * g.umax + x0 + u];
                         for (int c = 0; c < nchunk; ++c)
-                            tma_load_2d_pair(sB + s * G2_B_STAGE_BYTES + c * CHUNK_BYTES + u * UNIT_BYTES, &tmXB, full,
+                            tma_load_2d_pair(sB + s * B_ST + c * CHUNK_BYTES + u * UNIT_BYTES, &tmXB, full,
                                              my_n + c * 64, row);
                     }
                     if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
@@ -233,7 +249,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // descriptors of a stage's operands differ from stage 0's, and those of successive 16-deep slices from the
             // first slice's, only in the start-address field (16-byte units): they are stepped, not rebuilt
             const uint64_t da_base = desc_k_major(sA);
-            const uint64_t db_base = g.b_mn ? desc_mn_major(sB, CHUNK_BYTES) : desc_k_major(sB);
+            const uint64_t db_base = g.b_mn ? desc_mn_major(sB, KP * CHUNK_BYTES) : desc_k_major(sB);
             const uint64_t db_step = g.b_mn ? (uint64_t)(UNIT_BYTES >> 4) : 2ull;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
                 int m_idx, n_idx;
@@ -245,12 +261,18 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 uint32_t acc = 0;
                 for (int kb = 0; kb < g.num_kb && ok; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 34))) break;
-                    const uint64_t da = da_base + (uint64_t)(s * (A_STAGE_BYTES >> 4));
-                    const uint64_t db = db_base + (uint64_t)(s * (G2_B_STAGE_BYTES >> 4));
+                    const uint64_t da = da_base + (uint64_t)(s * (A_ST >> 4));
+                    const uint64_t db = db_base + (uint64_t)(s * (B_ST >> 4));
 #pragma unroll
-                    for (int j = 0; j < BK / 16; ++j) {
-                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(2 * j), db + (uint64_t)j * db_step, idesc_main, acc);
-                        acc = 1;
+                    for (int p = 0; p < KP; ++p) {
+                        // panel p: A tile 16 KB further; B rows 64 further down a chunk (MN-major) or tile 16 KB further (K-major)
+                        const uint64_t dap = da + (uint64_t)(p * (A_STAGE_BYTES >> 4));
+                        const uint64_t dbp = db + (g.b_mn ? (uint64_t)(p * (CHUNK_BYTES >> 4)) : (uint64_t)(p * (G2_B_STAGE_BYTES >> 4)));
+#pragma unroll
+                        for (int j = 0; j < BK / 16; ++j) {
+                            tc_mma_bf16_pair(d_tmem, dap + (uint64_t)(2 * j), dbp + (uint64_t)j * db_step, idesc_main, acc);
+                            acc = 1;
+                        }
                     }
                     tc_commit_pair(bar_empty + 8 * s);
                     if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
@@ -263,7 +285,7 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 for (int x0 = 0; x0 < nun && ok; x0 += 4) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 35))) break;
                     tc_fence_after();
-                    const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * G2_B_STAGE_BYTES;
+                    const uint32_t a0 = sA + s * A_ST, b0 = sB + s * B_ST;
                     const int nv = min(4, nun - x0);
                     for (int u = 0; u < nv; ++u) {
                         tc_mma_bf16_pair(d_tmem, desc_k_major(a0 + u * 32),
@@ -348,16 +370,16 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
 bool gemm2_sm100_eligible(const marlaas_pool* pool, int64_t M) { return M >= 1024 && pool->sm_count >= 2; }
 
-marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st) {
+template <int KP>
+static marlaas_status_t launch_gemm2_t(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st) {
     using namespace sm100;
-    if (o.M <= 0) return MARLAAS_OK;
     Gemm2Args g;
     g.M = (int)o.M;
     g.Nout = (int)o.Nout;
     g.Kc = (int)o.Kc;
     g.num_m_tiles = (int)cdiv(o.M, 256);
     g.num_n_tiles = (int)cdiv(o.Nout, G2_BN);
-    g.num_kb = (int)cdiv(o.Kc, BK);
+    g.num_kb = (int)cdiv(o.Kc, (int64_t)BK * KP);      // pipeline steps
     g.group_m = 8;
     g.b_mn = o.b_mn ? 1 : 0;
     g.tile_nunits = o.tile_nunits;
@@ -369,12 +391,13 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
 
     alignas(64) CUtensorMap tmA, tmB, tmXA, tmXB;
     marlaas_status_t rc;
-    if ((rc = make_map(&tmA, o.A, o.M, o.Kc, o.lda, BK, BM)) != MARLAAS_OK) return rc;
-    if (o.b_mn) {
-        if ((rc = make_map(&tmB, o.B, o.Kc, o.Nout, o.ldb, 64, BK)) != MARLAAS_OK) return rc;
-    } else {
-        if ((rc = make_map(&tmB, o.B, o.Nout, o.Kc, o.ldb, BK, 128)) != MARLAAS_OK) return rc;
-    }
+    if (KP == 1) rc = make_map(&tmA, o.A, o.M, o.Kc, o.lda, BK, BM);
+    else rc = make_panel_map(&tmA, o.A, o.M, o.Kc, o.lda, KP);
+    if (rc != MARLAAS_OK) return rc;
+    if (o.b_mn) rc = make_map(&tmB, o.B, o.Kc, o.Nout, o.ldb, 64, BK * KP);
+    else if (KP == 1) rc = make_map(&tmB, o.B, o.Nout, o.Kc, o.ldb, BK, 128);
+    else rc = make_panel_map(&tmB, o.B, o.Nout, o.Kc, o.ldb, KP);
+    if (rc != MARLAAS_OK) return rc;
     if (o.tile_nunits) {
         if ((rc = make_map(&tmXA, o.XA, o.M, o.xa_cols, o.xa_cols, BK, BM)) != MARLAAS_OK) return rc;
         if ((rc = make_map(&tmXB, o.XB, o.xb_rows, o.Nout, o.Nout, 64, 16)) != MARLAAS_OK) return rc;
@@ -386,7 +409,7 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
     static int max_clusters[64] = {};
     int& mc = max_clusters[pool->device < 64 ? pool->device : 63];
     if (mc == 0 || pool->device >= 64) {
-        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_gemm2_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_gemm2_sm100<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2 * (unsigned)(pool->sm_count / 2));
         cfg.blockDim = dim3(G2_THREADS);
@@ -399,7 +422,7 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
         cfg.attrs = &at;
         cfg.numAttrs = 1;
         int n = 0;
-        MARLAAS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, k_gemm2_sm100, &cfg));
+        MARLAAS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, k_gemm2_sm100<KP>, &cfg));
         if (n < 1) return fail(MARLAAS_ERR_CUDA, "no 2-CTA cluster of the GEMM kernel fits on this device");
         mc = n;
     }
@@ -415,9 +438,15 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_gemm2_sm100, tmA, tmB, tmXA, tmXB, g));
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_gemm2_sm100<KP>, tmA, tmB, tmXA, tmXB, g));
     count_launch();
     return MARLAAS_OK;
+}
+
+marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st) {
+    if (o.M <= 0) return MARLAAS_OK;
+    // two panels per step need the contraction depth in whole 64-deep panels (3-D views of the row-major operands)
+    return (o.Kc % 64) == 0 ? launch_gemm2_t<2>(pool, o, st) : launch_gemm2_t<1>(pool, o, st);
 }
 
 }  // namespace marlaas
