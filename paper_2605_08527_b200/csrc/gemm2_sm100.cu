@@ -380,7 +380,7 @@ static marlaas_status_t launch_gemm2_t(const marlaas_pool* pool, const GemmOpera
     g.num_m_tiles = (int)cdiv(o.M, 256);
     g.num_n_tiles = (int)cdiv(o.Nout, G2_BN);
     g.num_kb = (int)cdiv(o.Kc, (int64_t)BK * KP);      // pipeline steps
-    g.group_m = 8;
+    g.group_m = g.num_m_tiles >= 32 ? 16 : 8;      // row tiles per band (measured: 8-16 best; 32 loses the band's x rows from L2)
     g.b_mn = o.b_mn ? 1 : 0;
     g.tile_nunits = o.tile_nunits;
     g.tile_units = o.tile_units;
