@@ -36,7 +36,7 @@ FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed ncu captures
 # (profiles/); None where the kernel has changed since its counters were taken.
 TRAFFIC = {
-    "cfg3": 1.60e9,    # k_gemm2_sm100, mean of the forward (1.30 GB) and dx (1.90 GB) launches: profiles/gemm2_sm100_cfg3_ncu_full.txt
+    "cfg3": 1.49e9,    # k_gemm2_sm100, mean of the forward (0.94 GB) and dx (2.04 GB) launches: profiles/gemm2_sm100_cfg3_ncu_full.txt
     "cfg2": 46.5e6,    # k_decode_shrink (6.3 MB) + k_decode_gemm (40.2 MB) of one call: profiles/decode_cfg2_ncu_full.txt
 }
 CFG_OF = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
