@@ -12,44 +12,10 @@
 //                    dependent of the shrink: it streams W while the shrink runs and waits for hd only before the
 //                    expand k-blocks.
 #include "sm100_ptx.cuh"
+#include "sm100_cluster.cuh"
 
 namespace marlaas {
 namespace sm100 {
-
-// ---------------------------------------------------------------------------------------------------------------
-// shared helpers
-// ---------------------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t dk_cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t dk_cluster_id_x() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t dk_map_to_cta(uint32_t local_addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void dk_cluster_sync() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void dk_st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void dk_st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ void dk_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void dk_wait_prerequisites() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-__device__ __forceinline__ void dk_report(int32_t* status, int code, int detail) {
-    if (atomicCAS(status, 0, code) == 0) status[1] = detail;
-}
 
 // ---------------------------------------------------------------------------------------------------------------
 // k_decode_shrink
@@ -310,33 +276,6 @@ struct DecodeGemmArgs {
     int32_t* status;
 };
 
-__device__ __forceinline__ void dg_tma_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void dg_tma_pair_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0, int c1,
-                                               int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-__device__ __forceinline__ void dg_commit_pair(uint32_t bar, uint16_t mask) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-                 "h"(mask)
-                 : "memory");
-}
-__device__ __forceinline__ void dg_mma_pair(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
 // Operand staging per pipeline step (kp panels of 64 k):
 //   A  [kp][128 rows][64 k]      one 3-D TMA over x viewed as (64 k, rows, K / 64): K-major tiles, 128-byte swizzle
 //   B  [nch][kp * 64 k][64 n]    one 2-D TMA per 64-column chunk: MN-major, chunks kp * 8 KB apart
@@ -593,8 +532,9 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
 }
 
-// x (or hd) viewed as a 3-D tensor (64 k, rows, K / 64) so that one copy brings `panels` K-major tiles of 128 rows
-marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels) {
+// x (or hd) viewed as a 3-D tensor (64 k, rows, K / 64) so that one copy brings `panels` K-major tiles of box_rows rows
+marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels,
+                                uint32_t box_rows) {
     typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -608,7 +548,7 @@ marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows,
     }
     cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
     cuuint64_t gstr[2] = {(cuuint64_t)ld * 2, 128};
-    cuuint32_t box[3] = {64, 128, panels};
+    cuuint32_t box[3] = {64, box_rows, panels};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

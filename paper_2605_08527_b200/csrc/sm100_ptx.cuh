@@ -128,8 +128,9 @@ marlaas_status_t make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64
                           uint32_t box_rows);
 
 // The same matrix viewed as a 3-D tensor (64 k, rows, cols / 64): one copy brings `panels` consecutive K-major
-// [128 rows][64 k] tiles.  cols must be a multiple of 64.
-marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels);
+// [box_rows rows][64 k] tiles.  cols must be a multiple of 64.
+marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t panels,
+                                uint32_t box_rows = 128);
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
     asm volatile(
