@@ -62,11 +62,7 @@ enum {
     MARLAAS_FLAG_HOST_TABLE = 2u,     /* seg_offsets / seg_slot are HOST arrays: validated on the host, then copied
                                          into the workspace in stream order */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
-    MARLAAS_FLAG_CUDA_CORE_PATH = 8u, /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
-    MARLAAS_FLAG_COOPERATIVE_DECODE = 16u /* forward of at most 256 tokens: run the shrink, the base GEMM and the expand as
-                                             ONE cooperative kernel (all its CTAs must be resident at once and they wait on
-                                             one another, so nothing else may hold the GPU's SMs while the call runs)
-                                             instead of two overlapping kernels.  Ignored when the shape rules it out. */
+    MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
 };
 
 /* Token-to-adapter segment table of one mixed batch: segment s covers tokens

@@ -195,17 +195,9 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         }
         {
             TimedLaunch timed(pool, st);
-            bool launched = false;
-            if (flags & MARLAAS_FLAG_COOPERATIVE_DECODE) {
-                rc = launch_decode_fused_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
-                                               seg->seg_offsets, seg->seg_slot, ws, h, workspace, st, &launched);
-                if (rc != MARLAAS_OK) return rc;
-            }
-            if (!launched) {
-                rc = launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
-                                         seg->seg_offsets, seg->seg_slot, ws, h, st);
-                if (rc != MARLAAS_OK) return rc;
-            }
+            rc = launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
+                                     seg->seg_offsets, seg->seg_slot, ws, h, st);
+            if (rc != MARLAAS_OK) return rc;
         }
         return finish(pool, flags, st);
     }

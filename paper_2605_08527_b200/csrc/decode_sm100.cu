@@ -313,6 +313,14 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int ks0 = (int)((int64_t)pairi * g.num_ks / g.S), ks1 = (int)((int64_t)(pairi + 1) * g.num_ks / g.S);
     const int xs0 = (int)((int64_t)pairi * g.num_xs / g.S), xs1 = (int)((int64_t)(pairi + 1) * g.num_xs / g.S);
 
+    const int qper = 4 / g.S;
+    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
+    uint32_t live = 0;
+    for (int p = 0; p < g.S; ++p) {
+        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
+        if (n > 0) live |= 1u << p;
+    }
+    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -365,8 +373,26 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmB, full0 + 8 * s, my_n + c * 64, ks * g.kp * BK);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
+            // the expand's adapter rows Bs do not depend on the shrink grid: the first steps' B operands are fetched
+            // before the wait for it, their hd tiles after
+            const int npre = (xs1 - xs0) < STAGES ? (xs1 - xs0) : STAGES;
+            {
+                uint32_t b_s = s, b_ph = ph;
+                for (int i = 0; i < npre && ok; ++i) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * b_s, b_ph ^ 1, abort_word, 42))) break;
+                    if (half == 0) mbar_expect_tx(bar_full + 8 * b_s, stage_tx);
+                    for (int c = 0; c < my_chunks; ++c)
+                        dg_tma_pair(sB + b_s * b_stage_bytes + c * b_chunk_bytes, &tmXB, full0 + 8 * b_s, my_n + c * 64,
+                                    (xs0 + i) * g.kp * BK);
+                    if (++b_s == (uint32_t)STAGES) { b_s = 0; b_ph ^= 1; }
+                }
+            }
             if (ok && xs0 < xs1) dk_wait_prerequisites();     // hd comes from the shrink grid
-            for (int xs = xs0; xs < xs1 && ok; ++xs, ++it) {
+            for (int i = 0; i < npre && ok; ++i, ++it) {
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, (xs0 + i) * g.kp);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+            }
+            for (int xs = xs0 + npre; xs < xs1 && ok; ++xs, ++it) {
                 if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 42))) break;
                 if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
                 if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, xs * g.kp);
@@ -435,14 +461,6 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     // quarter send their partial accumulators to a mailbox in the finishing CTA (thread to thread: the same
     // tensor-memory lane on both sides, [column group][lane] 16-byte slots), and the finishing warp adds them to
     // its own accumulator in ascending pair order.  The mailboxes reuse the pipeline stages.
-    const int qper = 4 / g.S;
-    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
-    uint32_t live = 0;
-    for (int p = 0; p < g.S; ++p) {
-        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
-        if (n > 0) live |= 1u << p;
-    }
-    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     const int q = warp & 3;
     const uint32_t own = (uint32_t)(q % g.S);
     if (g.S > 1) {

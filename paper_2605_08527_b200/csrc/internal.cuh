@@ -65,8 +65,6 @@ struct SlotMeta {
 //   Bs : bf16 [capacity*RP][N]   row (slot*RP + j) = row j of B_t      (zero rows for j >= r_t)
 // Both serve as gather sources for the shrink (dot products along a contiguous row) and as tensor-core
 // operands for the extra k-steps of the fused expand (rows = rank index).
-constexpr int MARLAAS_SYNC_SETS = 24;     // counter pairs after the first 64 bytes of the 256-byte status block
-
 struct marlaas_pool {
     int device = 0;
     int64_t K = 0, N = 0;
@@ -80,8 +78,6 @@ struct marlaas_pool {
     marlaas::bf16* d_Bs = nullptr;
     std::vector<marlaas::SlotMeta> slots;
     int sm_count = 0;
-    // single-kernel decode: which workspace owns which grid-wide counter pair of the status block
-    mutable const void* sync_owner[MARLAAS_SYNC_SETS] = {};
     // kernel timing (marlaas_kernel_timing_begin/_end): event pairs around the dominant kernel
     bool timing = false;
     std::vector<cudaEvent_t> timing_events;
@@ -161,12 +157,7 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
 // decode_sm100.cu: the whole forward for batches of at most 256 tokens (two overlapping kernels).
 // S < 0: ws.tok_slot already holds the per-token slots.
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T);
-// Single cooperative kernel for the same batches; *launched = false (nothing issued) when the shape, the shared
-// memory or the resident-cluster limit rules it out.  ws_key identifies the caller's workspace.
-marlaas_status_t launch_decode_fused_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
-                                           int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
-                                           const int32_t* seg_slot, const Workspace& ws, float* h_out, const void* ws_key,
-                                           cudaStream_t st, bool* launched);
+
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
                                      int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
                                      const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);

@@ -85,12 +85,8 @@ def test_finely_interleaved_tenants_with_backward():
     _check_case(w, w.projections[0])
 
 
-DECODE_PATHS = [0, B.MARLAAS_FLAG_COOPERATIVE_DECODE]     # shrink and GEMM as two kernels / single cooperative kernel
-
-
-@pytest.mark.parametrize("path", DECODE_PATHS)
 @pytest.mark.parametrize("K,N", [(64, 64), (128, 320), (256, 320), (320, 1024)])
-def test_decode_shallow_contraction_repeated_calls(K, N, path):
+def test_decode_shallow_contraction_repeated_calls(K, N):
     # few 64-deep blocks of K: the decode GEMM may not cut the contraction into more slices than it has steps, and a
     # second call on other activations must not see anything the first one left in tensor memory
     w = wl.small_random_case(33 + K, 96, K, N, [16, 8, 32, 4], n_segments=9)
@@ -102,32 +98,29 @@ def test_decode_shallow_contraction_repeated_calls(K, N, path):
     for rep in range(3):
         xs = np.roll(p.x_bits, 7 * rep, axis=0)
         ref, _ = oracle.forward(wl.bf16_bits_to_f32(xs), p.W, r, s, A, Bm, ts)
-        y = dc.forward(x=dev_bf16(xs), flags=path)
+        y = dc.forward(x=dev_bf16(xs))
         assert_close(to_np(y), ref, f"decode K={K} N={N} call {rep}")
     B.marlaas_check_status(dc.pool)
 
 
-@pytest.mark.parametrize("path", DECODE_PATHS)
-def test_cfg2_decode_full_size(path):
+def test_cfg2_decode_full_size():
     w = wl.make_workload(2)
-    dc, _ = _check_case(w, w.projections[0], flags=path)
-    # the forward of this batch is two kernels, or one on the cooperative path
+    dc, _ = _check_case(w, w.projections[0])
+    # the forward of this batch is two kernels (shrink, and the GEMM launched as its programmatic dependent)
     n0 = B.marlaas_kernel_launch_count()
-    dc.forward(flags=path)
-    assert B.marlaas_kernel_launch_count() - n0 == (2 if path == 0 else 1)
+    dc.forward()
+    assert B.marlaas_kernel_launch_count() - n0 == 2
 
 
-@pytest.mark.parametrize("path", DECODE_PATHS)
 @pytest.mark.parametrize("T,K,N,ranks,cap", [
-    (256, 256, 512, (32, 8, 17, 0, 32, 5), 8),      # three 16-rank units per cluster; a rank-0 tenant; unused slots
-    (100, 192, 384, (16, 16, 16), 3),               # second half of the token tile empty; one unit per cluster
+    (256, 256, 512, (32, 8, 17, 0, 32, 5), 8),      # mixed ranks over two 16-rank units; a rank-0 tenant; unused slots
+    (100, 192, 384, (16, 16, 16), 3),               # second half of the 256-token tile empty
     (200, 128, 200, (64, 1, 40), 4),                # ragged last strip; four units per tenant
-    (256, 512, 128, (16,) * 12, 12),                # a single strip owns every unit (more than a cluster may take:
-                                                    # falls back to two kernels on either path)
+    (256, 512, 128, (16,) * 12, 12),                # a single 128-column strip
 ])
-def test_decode_unit_distribution_over_clusters(T, K, N, ranks, cap, path):
-    # decode-shaped batches whose adapter units do not map one to one onto the column strips, with base-only tokens
-    # and repeated calls on changing activations (the fused kernel's grid-wide counter must return to zero)
+def test_decode_mixed_ranks_and_base_only_tokens(T, K, N, ranks, cap):
+    # decode-shaped batches with base-only tokens, tenants of several rank units and repeated calls on changing
+    # activations, y and the saved h both checked
     w = wl.small_random_case(400 + T + N, T, K, N, list(ranks), n_segments=9)
     ts = wl.uniform_token_slots(400 + T + N, T, len(ranks)).astype(np.int32)
     ts[::11] = -1
@@ -140,7 +133,7 @@ def test_decode_unit_distribution_over_clusters(T, K, N, ranks, cap, path):
         xs = np.roll(p.x_bits, 5 * rep, axis=0)
         ref, rh = oracle.forward(wl.bf16_bits_to_f32(xs), p.W, r, s, A, Bm, tsl)
         hs = torch.full((T, dc.pool.rank_stride), 7.0, dtype=torch.float32, device="cuda:0")
-        y = dc.forward(x=dev_bf16(xs), flags=path, h_save=hs)
+        y = dc.forward(x=dev_bf16(xs), h_save=hs)
         assert_close(to_np(y), ref, f"decode units T={T} N={N} call {rep}: y")
         hr = np.zeros((T, dc.pool.rank_stride), np.float32)
         hr[:, :rh.shape[1]] = rh
