@@ -47,6 +47,36 @@ CFG_DESC = {
     "cfg4": "heterogeneous tenants: W 5120x5120, 32 tenants r in {8,16,32,64}, 8192 Zipf tokens, fwd+bwd",
     "cfg5": "7B decoder-layer adapter set: 7 projections, 32 tenants r=16, 4096 training + 256 decode tokens",
 }
+SWEEPS = {
+    # batch sizes x tenants of the rollout phases (the paper varies the number of concurrent tasks from 1 to 32)
+    "decode": [f"decode-{T}-{n}" for T in (32, 64, 128, 256, 512, 1024) for n in (1, 8, 32)],
+    "prefill": [f"prefill-{T}-{n}" for T in (8192, 16384, 32768) for n in (1, 8, 32)],
+}
+
+
+def workload_desc(name):
+    if name in CFG_DESC:
+        return CFG_DESC[name]
+    kind, T, n = name.split("-")
+    what = "decode tokens (one per sequence, tenants uniform and unsorted)" if kind == "decode" else \
+        "prompt tokens in whole-prompt lognormal segments"
+    return f"{kind} sweep point: W 4096x4096, {n} tenants r=16, {T} {what}, fwd only"
+
+
+def run_sweep(args):
+    """One bench.py process per sweep point (no CPU baseline, no end-to-end leg); prints their JSON lines."""
+    import subprocess
+    for name in SWEEPS[args.sweep]:
+        cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--steps", str(args.steps), "--warmup",
+               str(args.warmup), "--no-cpu-baseline", "--e2e-steps", "0", "--flags", str(args.flags)]
+        r = subprocess.run(cmd, capture_output=True, text=True)
+        lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+        if r.returncode != 0 or not lines:
+            print(json.dumps({"sweep": args.sweep, "workload": name, "failed": r.stderr.strip().splitlines()[-1:] }))
+            continue
+        d = json.loads(lines[-1])
+        d["sweep"] = args.sweep
+        print(json.dumps(d), flush=True)
 
 
 def measured_peaks():
@@ -176,7 +206,7 @@ def run_reference(args, rank, world):
     if rank != 0:
         return
     import oracle
-    w = wl.make_workload(CFG_OF[args.workload])
+    w = wl.make_named_workload(args.workload)
     n_tok = min(w.T, args.reference_tokens)
     for _ in range(args.warmup):
         oracle_step_sample(w, min(n_tok, 32))
@@ -190,7 +220,7 @@ def run_reference(args, rank, world):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32 storage / f64 accumulate", "data": "synthetic",
-        "config": {"workload": args.workload, "desc": CFG_DESC[args.workload], "sample": sample},
+        "config": {"workload": args.workload, "desc": workload_desc(args.workload), "sample": sample},
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -202,7 +232,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg3", choices=sorted(CFG_OF))
+    ap.add_argument("--workload", default="cfg3",
+                    help="cfg1 .. cfg5, or a forward-only sweep point decode-T-n / prefill-T-n (T tokens, n tenants)")
+    ap.add_argument("--sweep", choices=["decode", "prefill"],
+                    help="run a grid of sweep points, one bench.py process and one JSON line each")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--reference-tokens", type=int, default=1024)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2048)
@@ -213,6 +246,11 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+    if args.sweep:
+        if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+            raise SystemExit("bench.py --sweep runs on one GPU")
+        run_sweep(args)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -235,7 +273,7 @@ def main():
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
 
-    w = wl.make_workload(CFG_OF[args.workload])
+    w = wl.make_named_workload(args.workload)
     work = algorithmic_work(w)
     ts_np = w.tok_slot()
 
@@ -397,7 +435,10 @@ def main():
     gemm_flops_per_step = float(sum(work["gemm_flops"]))
     avg_launch_ms = gemm_ms / max(gemm_n, 1)
     flops_per_launch = gemm_flops_per_step / max(len(work["gemm_flops"]), 1)
-    if not Tb:
+    # forward-only batches below the machine balance (flops per byte of the measured peaks) are bound by the one pass
+    # over W; everything else by the tensor cores
+    hbm_bound = (not Tb) and work["fwd_flops"] / work["fwd_bytes"] < peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if hbm_bound:
         ach = work["fwd_bytes"] / (ms_per_step * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": ach / peaks["hbm_gbs"], "traffic": TRAFFIC.get(args.workload), "peak_source": f"of {peak_src}",
@@ -417,7 +458,7 @@ def main():
                     "frac": ach / peak_t, "traffic": TRAFFIC.get(args.workload),
                     "peak_source": f"of {peak_src} ({'sustained: the timed loop ran power-capped' if capped else 'burst'})",
                     "frac_of_measured_burst": ach / peaks["bf16_tflops"],
-                    "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)",
+                    "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)" if Tb else "base GEMM with fused LoRA expand (forward launches)",
                     "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms, "flops_per_launch": flops_per_launch,
                     "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
                     "frac_of_measured_sustained": ach / peaks["bf16_tflops_sustained"],
@@ -495,7 +536,7 @@ def main():
             "metric": METRIC if Tb else "multi-LoRA layer tokens/s (fwd)", "value": value, "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "desc": CFG_DESC[args.workload], "tokens_per_step_per_gpu": w.T,
+            "config": {"workload": args.workload, "desc": workload_desc(args.workload), "tokens_per_step_per_gpu": w.T,
                        "backward_tokens": Tb, "segments": int(len(w.seg_slot)), "l2": l2_note,
                        "timed_as": "one CUDA graph of K steps, median of %d replays" % reps if graph is not None else "K direct steps",
                        "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},

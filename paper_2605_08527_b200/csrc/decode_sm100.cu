@@ -1,5 +1,6 @@
-// Decode-shaped forward (at most 256 tokens, one per sequence, tenants unsorted): the call is bound by the one pass
-// over W from HBM, so the work is cut to keep every SM streaming and the launch count to two overlapping kernels.
+// Decode-shaped forward (up to four 256-token tiles, typically one token per sequence, tenants unsorted): the call is
+// bound by the one pass over W from HBM (or, from about 300 tokens, by the tensor cores on a grid of few tiles), so the
+// work is cut to keep every SM busy and the launch count to two overlapping kernels.
 //
 //   k_decode_shrink  (CUDA cores + warp-level MMA)  per tenant: h_i = x_i A_t for the tenant's tokens, gathered from
 //                    the pooled store; a cluster of CTAs splits K and sums its partial products through distributed
@@ -21,15 +22,17 @@ namespace sm100 {
 // k_decode_shrink
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int DS_THREADS = 128;
-constexpr int DS_MAX_T = 256;          // tokens per call
+constexpr int DS_MAX_T = 1024;         // tokens per call
+constexpr int DS_ROUNDS = DS_MAX_T / DS_THREADS;
 constexpr int DS_PASS = 16;            // tokens per pass (one m16 MMA tile)
 constexpr int DS_MAX_CS = 8;
-constexpr int DS_TABLE_SMEM = 1024;    // the segment table is staged in shared memory when S + 1 <= this
+constexpr int DS_TABLE_SMEM = 1032;    // the segment table is staged in shared memory when S + 1 <= this
 constexpr int DS_UB = 4;               // 32-deep k-blocks whose loads are in flight together per warp
 
 struct DecodeShrinkArgs {
     int T, K, RP, cap;
     int S;                              // segments; < 0: tok_slot already holds the per-token slots
+    int G;                              // clusters per tenant: cluster (t, i) takes the 16-token passes i, i + G, ...
     const int32_t* seg_offsets;
     const int32_t* seg_slot;
     const bf16* x;
@@ -48,11 +51,14 @@ struct __align__(16) DecodeShrinkSmem {
     float wpart[4][256];                // per-warp [16 tokens][16 ranks] partial products
     float part[DS_MAX_CS][256];         // per-CTA partials, gathered in cluster rank 0
     int32_t slot[DS_MAX_T];
-    int32_t list[DS_MAX_T];
-    int32_t off_tab[DS_TABLE_SMEM];
+    union {
+        int32_t off_tab[DS_TABLE_SMEM];  // the staged table is dead once every token has its slot:
+        int32_t list[DS_MAX_T];          // the cluster's token list takes its place
+    };
     int32_t slot_tab[DS_TABLE_SMEM];
-    int32_t cnt[8];
+    int32_t cnt[DS_ROUNDS * 4];
 };
+static_assert(DS_TABLE_SMEM >= DS_MAX_T, "the token list reuses the table's space");
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -84,8 +90,9 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     const int crank = (int)dk_cluster_ctarank();
     int cs;
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(cs));
-    const int t = (int)dk_cluster_id_x();           // tenant slot served by this cluster; == cap: no adapter
-    const bool first = (t == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
+    const int t = (int)dk_cluster_id_x() / g.G;     // tenant slot served by this cluster; == cap: no adapter
+    const int gi = (int)dk_cluster_id_x() % g.G;    // which of the tenant's 16-token passes
+    const bool first = (dk_cluster_id_x() == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
     const int r_t = t < g.cap ? g.d_rank[t] : 0;
     const float sc = t < g.cap ? g.d_scale[t] : 0.f;
 
@@ -132,10 +139,10 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
         }
 
     // ---- this cluster's tokens, ascending --------------------------------------------------------------------
-    unsigned bal[2];
-    bool mine[2];
+    unsigned bal[DS_ROUNDS];
+    bool mine[DS_ROUNDS];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int r = 0; r < DS_ROUNDS; ++r) {
         const int i = r * DS_THREADS + tid;
         bool m = false;
         if (i < g.T) {
@@ -149,9 +156,9 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     __syncthreads();
     int n_t = 0;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) n_t += sm.cnt[e];
+    for (int e = 0; e < DS_ROUNDS * 4; ++e) n_t += sm.cnt[e];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int r = 0; r < DS_ROUNDS; ++r) {
         if (mine[r]) {
             int off = __popc(bal[r] & ((1u << lane) - 1u));
             for (int e = 0; e < r * 4 + warp; ++e) off += sm.cnt[e];
@@ -159,7 +166,7 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
         }
     }
     __syncthreads();
-    if (n_t == 0) return;        // uniform over the cluster
+    if (gi * DS_PASS >= n_t) return;     // nothing for this cluster (uniform over it)
 
     const int own0 = r_t > 0 ? t * g.RP : 0, own1 = r_t > 0 ? own0 + g.RP : 0;   // hd columns written by the MMA part
     const int ngroups = (r_t + 15) >> 4;
@@ -174,6 +181,7 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
 
     // zero the other tenants' columns of this cluster's hd rows (and, with no adapter, the h rows): one warp per row
     for (int e = crank * 4 + warp; e < n_t; e += cs * 4) {
+        if ((e / DS_PASS) % g.G != gi) continue;     // another cluster's pass
         const int tok = sm.list[e];
         bf16* row = g.hd + (size_t)tok * g.hd_cols;
         for (int c = lane * 8; c < g.hd_cols; c += 256)
@@ -183,7 +191,7 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     }
     if (r_t == 0) return;        // uniform over the cluster
 
-    for (int p0 = 0; p0 < n_t; p0 += DS_PASS) {
+    for (int p0 = gi * DS_PASS; p0 < n_t; p0 += DS_PASS * g.G) {
         const int np = min(DS_PASS, n_t - p0);
         const bf16* xr0 = gq < np ? g.x + (size_t)sm.list[p0 + gq] * g.ldx : nullptr;
         const bf16* xr1 = gq + 8 < np ? g.x + (size_t)sm.list[p0 + gq + 8] * g.ldx : nullptr;
@@ -265,6 +273,7 @@ constexpr int DG_KP = 2;               // 64-deep panels per pipeline step
 
 struct DecodeGemmArgs {
     int T, Nout;
+    int nstrips;         // column strips; cluster c works on strip c mod nstrips of 256-row tile c / nstrips
     int num_ks;          // pipeline steps (kp * 64 deep) over K
     int num_xs;          // pipeline steps over the expand rows (cap*RP, or up to the last slot in use)
     int S;               // contraction slices = CTA pairs per cluster
@@ -306,8 +315,9 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const uint32_t pairi = crank >> 1;          // which slice of the contraction
     const uint32_t leader = crank & ~1u;
     const int NP = 128 * g.nch;                 // columns of the cluster's strip
-    const int n0 = (int)dk_cluster_id_x() * NP;
-    const int my_m = (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
+    const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
+    const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
+    const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
     const uint32_t tmem_cols = (uint32_t)NP;    // 128 or 256
 
     const int ks0 = (int)((int64_t)pairi * g.num_ks / g.S), ks1 = (int)((int64_t)(pairi + 1) * g.num_ks / g.S);
@@ -352,7 +362,7 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     // bytes the two CTAs of the pair stage per step (rows and columns outside the tensors are skipped entirely;
     // partly outside boxes are filled with zeros and count in full)
-    auto a_bytes = [&](int r) -> uint32_t { return (r * 128 < g.T) ? a_stage_bytes : 0u; };
+    auto a_bytes = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? a_stage_bytes : 0u; };
     auto b_chunks = [&](int r) -> int { return max(0, min(g.nch, (g.Nout - (n0 + r * 64 * g.nch) + 63) / 64)); };
     const uint32_t stage_tx = a_bytes(0) + a_bytes(1) + (uint32_t)(b_chunks(0) + b_chunks(1)) * b_chunk_bytes;
     const int my_chunks = b_chunks((int)half);
@@ -583,8 +593,10 @@ marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows,
 // host side
 // ---------------------------------------------------------------------------------------------------------------
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T) {
-    return T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 1024 && pool->sm_count >= 8 &&
-           (pool->K % 64) == 0;
+    if (!(T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 1024 && pool->sm_count >= 8 && (pool->K % 64) == 0))
+        return false;
+    // beyond one 256-token tile only while all (token tile, 256-column strip) pairs make a single wave of CTA pairs
+    return T <= 256 || cdiv(T, 256) * cdiv(pool->N, 256) <= pool->sm_count / 2;
 }
 
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
@@ -603,6 +615,10 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         a.tok_slot = ws.tok_slot; a.h_out = h_out; a.hd = ws.hd; a.hd_cols = hd_cols; a.status = pool->d_status;
         int cs = DS_MAX_CS;
         while (cs > 1 && K / cs < 32 * 4 * DS_UB) cs >>= 1;      // a full batch of loads per warp
+        // with few tenants a tenant has many 16-token passes: several clusters share them, as many as keep the grid
+        // within two CTAs per SM
+        const int passes = (int)cdiv(T, DS_PASS);
+        a.G = std::max(1, std::min(passes, (2 * pool->sm_count) / ((pool->cap + 1) * cs)));
         static bool carveout_set[64] = {};
         if (pool->device >= 64 || !carveout_set[pool->device]) {
             // same shared-memory configuration as the GEMM, so that CTAs of both kernels can share an SM
@@ -611,7 +627,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
             if (pool->device < 64) carveout_set[pool->device] = true;
         }
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)((pool->cap + 1) * cs));
+        cfg.gridDim = dim3((unsigned)((pool->cap + 1) * a.G * cs));
         cfg.blockDim = dim3(DS_THREADS);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
@@ -635,6 +651,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
     const Shape shapes[] = {{1, 2}, {2, 2}, {1, 1}, {2, 1}, {1, 4}, {2, 4}};
     Shape pick = {2, 1};
     int64_t best = -1;
+    const int64_t mtiles = cdiv(T, 256);
     static int max_clusters[64][3] = {};      // per device, cluster size 2 / 4 / 8
     constexpr int DG_SMEM = 200 * 1024;
     for (const Shape& sh : shapes) {
@@ -656,20 +673,20 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
             if (pool->device < 64) max_clusters[pool->device][ci] = mc;
         }
         if (mc < 1) continue;
-        const int64_t clusters = cdiv(N, 128 * sh.nch);
+        const int64_t clusters = cdiv(N, 128 * sh.nch) * mtiles;
         if (clusters > mc) continue;                    // one wave only
         if (cdiv(K, (int64_t)DG_KP * BK) < sh.S) continue;     // every slice needs at least one step
         const int64_t ctas = clusters * csz;
         // more CTAs streaming is better; among equals prefer fewer slices and wider strips (less re-read of x)
-        const int64_t score = ctas * 16 - sh.S * 2 + sh.nch;
+        const int64_t score = ctas * 16 + sh.nch * 4 - sh.S * 2;
         if (score > best) { best = score; pick = sh; }
     }
     g.S = pick.S; g.nch = pick.nch;
     g.kp = DG_KP;
     const size_t step_bytes = (size_t)g.kp * (A_STAGE_BYTES + g.nch * CHUNK_BYTES);
-    // leave room for two shrink CTAs (22 KB static + 1 KB system reservation each) on the same SM: the shrink then
+    // leave room for two shrink CTAs (25 KB static + 1 KB system reservation each) on the same SM: the shrink then
     // overlaps the GEMM's main loop instead of delaying its start (measured: 23 us per call against 29 us)
-    g.stages = (int)((DG_SMEM - 1024 - 256 - 2 * 24 * 1024) / step_bytes);
+    g.stages = (int)((DG_SMEM - 1024 - 256 - 2 * 26 * 1024) / step_bytes);
     if (g.stages < 2) g.stages = 2;
     g.num_ks = (int)cdiv(K, (int64_t)g.kp * BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)g.kp * BK);
@@ -688,7 +705,8 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
     }
     const size_t smem_bytes = 1024 + (size_t)g.stages * step_bytes + 256;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(cdiv(N, NP) * 2 * g.S));
+    g.nstrips = (int)cdiv(N, NP);
+    cfg.gridDim = dim3((unsigned)(g.nstrips * mtiles * 2 * g.S));
     cfg.blockDim = dim3(DG_THREADS);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;

@@ -154,7 +154,7 @@ marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands&
 bool gemm2_sm100_eligible(const marlaas_pool* pool, int64_t M);
 marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
 
-// decode_sm100.cu: the whole forward for batches of at most 256 tokens (two overlapping kernels).
+// decode_sm100.cu: the whole forward for batches of at most 1024 tokens (two overlapping kernels).
 // S < 0: ws.tok_slot already holds the per-token slots.
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T);
 

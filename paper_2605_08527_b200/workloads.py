@@ -316,6 +316,36 @@ def make_workload(cfg: int, scale_down: int = 1, seed: Optional[int] = None) -> 
     raise ValueError(f"unknown config {cfg}")
 
 
+SWEEP_NAME = r"^(decode|prefill)-(\d+)-(\d+)$"
+
+
+def make_named_workload(name: str) -> Workload:
+    """``cfgN`` gives make_workload(N).  Two forward-only families for sweeps over the rollout phases, both on a
+    4096 x 4096 base weight with rank-16 adapters of scale 2:
+
+    ``decode-T-n``   T decode tokens (one per sequence), tenant of each token uniform over n tenants, unsorted;
+    ``prefill-T-n``  T prompt tokens in whole-prompt segments (lognormal lengths, median 1024, clipped to
+                     [128, 4096]) dealt to n tenants in shuffled order."""
+    import re
+    if name.startswith("cfg") and name[3:].isdigit():
+        return make_workload(int(name[3:]))
+    m = re.match(SWEEP_NAME, name)
+    if not m:
+        raise ValueError(f"unknown workload {name!r}")
+    kind, T, n = m.group(1), int(m.group(2)), int(m.group(3))
+    if T < 1 or n < 1 or n > 4096:
+        raise ValueError(f"workload {name!r}: need T >= 1 and 1 <= tenants <= 4096")
+    seed = BASE_SEED + 100 + (0 if kind == "decode" else 1)
+    K = N = 4096
+    if kind == "decode":
+        offsets, slots = per_token_table(uniform_token_slots(seed, T, n))
+    else:
+        offsets, slots = lognormal_segments(seed, T, n)
+    ranks, alphas = [16] * n, [32.0] * n
+    projs = [_make_projection(seed, "proj", K, N, n, ranks, alphas, T, 0, 0, 0)]
+    return Workload(name, T, 0, offsets, slots, projs, n, 16)
+
+
 def small_random_case(seed: int, T: int, K: int, N: int, ranks, alphas=None, n_segments: int = 6,
                       with_base_only: bool = True, sigma_w: float = 0.02) -> Workload:
     """Small ragged case for tests: random segment boundaries (zero-length segments allowed), tenants may

@@ -117,6 +117,9 @@ def test_cfg2_decode_full_size():
     (100, 192, 384, (16, 16, 16), 3),               # second half of the 256-token tile empty
     (200, 128, 200, (64, 1, 40), 4),                # ragged last strip; four units per tenant
     (256, 512, 128, (16,) * 12, 12),                # a single 128-column strip
+    (300, 128, 384, (16, 8), 2),                    # two 256-token tiles, the second with 44 rows
+    (777, 192, 320, (32,), 1),                      # one tenant: its 16-token passes are shared by several clusters
+    (1024, 256, 512, (16, 16, 16), 3),              # four full token tiles
 ])
 def test_decode_mixed_ranks_and_base_only_tokens(T, K, N, ranks, cap):
     # decode-shaped batches with base-only tokens, tenants of several rank units and repeated calls on changing
