@@ -79,6 +79,83 @@ def run_sweep(args):
         print(json.dumps(d), flush=True)
 
 
+def run_adamw(args, n_tenants):
+    """Times the fused policy update + commit (marlaas_adapter_pool_adamw_commit) for n tenants of rank 16 on a
+    4096 x 4096 projection: one call = one optimizer step of every tenant.  HBM-bound: 30 bytes per adapter element."""
+    import torch
+    from paper_2605_08527_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the layer has no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    K = N = 4096
+    r = 16
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    elems = n_tenants * r * (K + N)
+    state_bytes = elems * 28                    # gradient, master, two moments read; master and moments written
+    R = int(min(16, max(1, -(-3 * l2 // state_bytes))))
+    copies = []
+    for c in range(R):
+        pool = B.AdapterPool(K, N, r, n_tenants, device=dev)
+        st = {"pool": pool, "ids": list(range(1, n_tenants + 1))}
+        gen = torch.Generator(device=dev).manual_seed(1234 + c)
+        for nm, shape in (("dA", (K, r)), ("dB", (r, N)), ("A", (K, r)), ("B", (r, N))):
+            st[nm] = [torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * (0.02 if nm in "AB" else 1.0)
+                      for _ in range(n_tenants)]
+        for nm, like in (("mA", "A"), ("vA", "A"), ("mB", "B"), ("vB", "B")):
+            st[nm] = [torch.zeros_like(t) for t in st[like]]
+        for i, tid in enumerate(st["ids"]):
+            B.marlaas_adapter_pool_register(pool, tid, 0, r, 32.0, st["A"][i].to(torch.bfloat16), st["B"][i].to(torch.bfloat16))
+        copies.append(st)
+
+    def step(i):
+        c = copies[i % R]
+        B.marlaas_adapter_pool_adamw_commit(c["pool"], c["ids"], c["dA"], c["dB"], c["A"], c["B"], c["mA"], c["vA"], c["mB"],
+                                            c["vB"], lr=1e-3, weight_decay=0.01, step=i + 1)
+
+    for i in range(max(args.warmup, R)):
+        step(i)
+    torch.cuda.synchronize()
+    # a call lasts tens of microseconds, less than Python needs to marshal its eight pointer tables: the K steps are
+    # captured once into a CUDA graph (the call takes its pointers by value, so a capture can hold it) and replayed
+    n0 = B.marlaas_kernel_launch_count()
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(args.steps):
+                step(args.warmup + i)
+    torch.cuda.current_stream().wait_stream(side)
+    launches = B.marlaas_kernel_launch_count() - n0
+    graph.replay()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    reps = 20
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in evs:
+        a.record()
+        graph.replay()
+        b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = float(np.median([a.elapsed_time(b) for a, b in evs])) / args.steps
+    peaks, peak_src = measured_peaks()
+    bytes_per_step = elems * 30.0
+    ach = bytes_per_step / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "adapter AdamW updates + commits per second", "value": n_tenants / (ms * 1e-3), "unit": "tenant updates/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "desc": f"AdamW + commit of {n_tenants} tenants, rank 16, on a 4096x4096 projection; "
+                   "one call per step", "timed_as": "one CUDA graph of K steps, median of 20 replays", "l2": f"optimizer state of a step ({state_bytes / 1e6:.0f} MB) rotates over {R} copies"},
+        "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": f"of {peak_src}", "kernel": "k_adamw_commit",
+                     "bytes_per_launch": bytes_per_step / max(launches / args.steps, 1)},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks}))
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -233,7 +310,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg3",
-                    help="cfg1 .. cfg5, or a forward-only sweep point decode-T-n / prefill-T-n (T tokens, n tenants)")
+                    help="cfg1 .. cfg5, a forward-only sweep point decode-T-n / prefill-T-n (T tokens, n tenants), or adamw-n "
+                         "(the fused optimizer step + commit of n tenants)")
     ap.add_argument("--sweep", choices=["decode", "prefill"],
                     help="run a grid of sweep points, one bench.py process and one JSON line each")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -246,6 +324,9 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+    if args.workload.startswith("adamw-") and args.workload[6:].isdigit():
+        run_adamw(args, int(args.workload[6:]))
+        return
     if args.sweep:
         if int(os.environ.get("WORLD_SIZE", "1")) != 1:
             raise SystemExit("bench.py --sweep runs on one GPU")

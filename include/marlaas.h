@@ -108,6 +108,28 @@ marlaas_status_t marlaas_adapter_pool_lookup(const marlaas_pool_t* pool, uint64_
  * device memory; either may be NULL).  Used to check the store's re-layout bit for bit. */
 marlaas_status_t marlaas_adapter_pool_export(marlaas_pool_t* pool, int32_t slot, void* A_out, void* B_out,
                                              void* cuda_stream);
+/* Policy update and commit of the updated parameters for n tenants in one launch (Algorithm 1: "PolicyUpdate",
+ * then the commit of the new adapter version; Methods, Multi-Task Manager: per-task optimizer state and version
+ * counter).  The paper names no optimizer; this is AdamW with decoupled weight decay, in fp32:
+ *     g = grad_scale * grad;  m = beta1 m + (1 - beta1) g;  v = beta2 v + (1 - beta2) g^2
+ *     theta = theta - lr * ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay * theta )
+ * applied to the fp32 master copies A [d_in][rank] and B [rank][d_out] of every listed tenant (moments m*, v* of the
+ * same shapes, all updated in place), after which the bf16 rounding (round to nearest even) of the new masters
+ * replaces the tenant's rows of the pooled store, as marlaas_adapter_pool_register would write them, and the
+ * tenant's version becomes new_versions[i] (or its old version + 1 when new_versions is NULL).
+ * tenant_ids / new_versions and the eight pointer tables are HOST arrays of n entries; the pointers in the tables are
+ * device memory (4-byte aligned, caller-owned, gradients as marlaas_lora_backward wrote them: true rank, dense).
+ * Stream-ordered like register.  Errors, before anything is launched: unknown tenant (MARLAAS_ERR_UNKNOWN_TENANT),
+ * a tenant of rank 0 or listed twice, a NULL pointer, step < 1 (MARLAAS_ERR_INVALID_ARG). */
+typedef struct marlaas_adamw {
+    float lr, beta1, beta2, eps, weight_decay, grad_scale;
+    int64_t step; /* >= 1: the step being taken */
+} marlaas_adamw_t;
+marlaas_status_t marlaas_adapter_pool_adamw_commit(marlaas_pool_t* pool, int32_t n, const uint64_t* tenant_ids,
+                                                   const uint64_t* new_versions, const float* const* dA,
+                                                   const float* const* dB, float* const* A, float* const* B,
+                                                   float* const* m_A, float* const* v_A, float* const* m_B,
+                                                   float* const* v_B, const marlaas_adamw_t* hp, void* cuda_stream);
 /* Row stride (in floats) of the h_save / h_saved arrays: max_rank rounded up to a multiple of 16. */
 int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool);
 

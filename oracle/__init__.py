@@ -9,6 +9,9 @@ Layer definition (frozen shared base weight W, per-tenant adapters A_t, B_t with
 paper's Multi-Task Manager and Multi-LoRA Rollout sections): y_i = x_i W + s_t (x_i A_t) B_t,
 dx_i = dy_i W^T + s_t (dy_i B_t^T) A_t^T, dA_t = s_t sum_i x_i^T (dy_i B_t^T),
 dB_t = s_t sum_i (x_i A_t)^T dy_i, sums over the tokens routed to tenant t.
+
+adamw_step (the policy update that precedes the commit of a new adapter version in Algorithm 1; the paper names no
+optimizer, AdamW is this build's choice) is written out below in float64 numpy.
 """
 from __future__ import annotations
 
@@ -133,3 +136,18 @@ def adapters_of(proj, dtype=np.float32):
     ranks = [a.rank for a in proj.adapters]
     scales = [np.dtype(dtype).type(a.alpha) / np.dtype(dtype).type(a.rank) if a.rank > 0 else 0 for a in proj.adapters]
     return ranks, scales, [a.A for a in proj.adapters], [a.B for a in proj.adapters]
+
+
+def adamw_step(theta, grad, m, v, *, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, grad_scale=1.0, step=1):
+    """One AdamW step (Adam with decoupled weight decay), from its definition, in float64:
+        g = grad_scale * grad;  m' = beta1 m + (1 - beta1) g;  v' = beta2 v + (1 - beta2) g^2
+        theta' = theta - lr * ( (m' / (1 - beta1^step)) / (sqrt(v' / (1 - beta2^step)) + eps) + weight_decay * theta )
+    Returns (theta', m', v')."""
+    theta, m, v = (np.asarray(a, dtype=np.float64) for a in (theta, m, v))
+    g = float(grad_scale) * np.asarray(grad, dtype=np.float64)
+    m1 = beta1 * m + (1.0 - beta1) * g
+    v1 = beta2 * v + (1.0 - beta2) * g * g
+    m_hat = m1 / (1.0 - beta1 ** step)
+    v_hat = v1 / (1.0 - beta2 ** step)
+    theta1 = theta - lr * (m_hat / (np.sqrt(v_hat) + eps) + weight_decay * theta)
+    return theta1, m1, v1

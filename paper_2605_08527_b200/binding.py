@@ -38,7 +38,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
-    "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws",
+    "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
 ]
 
 
@@ -46,6 +46,11 @@ class MarlaasError(RuntimeError):
     def __init__(self, status: int, message: str):
         super().__init__(f"marlaas status {status}: {message}")
         self.status = status
+
+
+class marlaas_adamw_t(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+                ("weight_decay", ctypes.c_float), ("grad_scale", ctypes.c_float), ("step", ctypes.c_int64)]
 
 
 class marlaas_segments_t(ctypes.Structure):
@@ -81,6 +86,8 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_adapter_pool_lookup.argtypes = [vp, u64, P(i32), P(i32), P(f32), P(u64)]
     L.marlaas_adapter_pool_export.restype = i32
     L.marlaas_adapter_pool_export.argtypes = [vp, i32, vp, vp, vp]
+    L.marlaas_adapter_pool_adamw_commit.restype = i32
+    L.marlaas_adapter_pool_adamw_commit.argtypes = [vp, i32, P(u64), P(u64)] + [P(vp)] * 8 + [P(marlaas_adamw_t), vp]
     L.marlaas_adapter_pool_rank_stride.restype = i32
     L.marlaas_adapter_pool_rank_stride.argtypes = [vp]
     L.marlaas_lora_workspace_bytes.restype = sz
@@ -204,6 +211,29 @@ def marlaas_adapter_pool_register(pool: AdapterPool, tenant_id: int, version: in
     _check(load_library().marlaas_adapter_pool_register(pool.handle, tenant_id, version, rank, alpha, _dptr(A), _dptr(B),
                                                         ctypes.byref(slot), _stream(stream)))
     return int(slot.value)
+
+
+def marlaas_adapter_pool_adamw_commit(pool: AdapterPool, tenant_ids: Sequence[int], dA, dB, A, B, m_A, v_A, m_B, v_B, *,
+                                      lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                                      weight_decay: float = 0.0, grad_scale: float = 1.0, step: int = 1,
+                                      new_versions: Optional[Sequence[int]] = None, stream=None) -> None:
+    """AdamW on the fp32 masters of the listed tenants and commit of their bf16 rounding into the pool.  Each of the
+    eight arguments dA .. v_B is a list (one entry per tenant) of contiguous fp32 device tensors, updated in place
+    (A, m_A, v_A: [d_in][rank]; B, m_B, v_B: [rank][d_out])."""
+    n = len(tenant_ids)
+    tables = []
+    for name, lst in (("dA", dA), ("dB", dB), ("A", A), ("B", B), ("m_A", m_A), ("v_A", v_A), ("m_B", m_B), ("v_B", v_B)):
+        assert len(lst) == n, name
+        tab = (ctypes.c_void_p * max(n, 1))()
+        for i, t in enumerate(lst):
+            assert t.dtype == torch.float32 and t.is_contiguous() and t.device == pool.device, name
+            tab[i] = t.data_ptr()
+        tables.append(tab)
+    ids = (ctypes.c_uint64 * max(n, 1))(*tenant_ids)
+    vers = None if new_versions is None else (ctypes.c_uint64 * max(n, 1))(*new_versions)
+    hp = marlaas_adamw_t(lr, beta1, beta2, eps, weight_decay, grad_scale, step)
+    _check(load_library().marlaas_adapter_pool_adamw_commit(pool.handle, n, ids, vers, *tables, ctypes.byref(hp),
+                                                            _stream(stream)))
 
 
 def marlaas_adapter_pool_unregister(pool: AdapterPool, tenant_id: int, stream=None) -> None:

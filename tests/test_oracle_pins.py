@@ -321,3 +321,59 @@ def test_float_accumulation_agrees_with_double_on_cfg1():
         y32[i] += np.float32(s[t]) * ((p.x[i] @ A[t]) @ B[t])
     bound = 1e-5 * (np.abs(p.x) @ np.abs(p.W) + 1.0)
     assert np.all(np.abs(y32 - y) <= bound)
+
+
+# ---- AdamW (policy update before the commit of a new adapter version) ------------------------------------------
+def _rand(shape, seed):
+    return wl.bf16_bits_to_f32(wl.normal_bf16(seed, wl.TID_PERTURB, shape, 1.0)[0]).astype(np.float64)
+
+
+def test_adamw_first_step_closed_form():
+    # from zero moments the bias corrections cancel the (1 - beta) factors exactly: m_hat = g, v_hat = g^2
+    th, g = _rand((7, 5), 901), _rand((7, 5), 902)
+    lr, eps, wd = 0.05, 1e-3, 0.1
+    t1, m1, v1 = oracle.adamw_step(th, g, np.zeros_like(th), np.zeros_like(th), lr=lr, beta1=0.9, beta2=0.99, eps=eps,
+                                   weight_decay=wd, step=1)
+    np.testing.assert_allclose(t1, th - lr * (g / (np.abs(g) + eps) + wd * th), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(m1, 0.1 * g, rtol=1e-12)
+    np.testing.assert_allclose(v1, 0.01 * g * g, rtol=1e-12)
+
+
+def test_adamw_constant_gradient_and_pure_decay_closed_forms():
+    th0, g = _rand((4, 6), 903), _rand((4, 6), 904)
+    lr, eps, n = 0.01, 1e-4, 9
+    # constant gradient, no decay: m_hat = g and v_hat = g^2 at every step, so each step moves by lr g / (|g| + eps)
+    th, m, v = th0, np.zeros_like(th0), np.zeros_like(th0)
+    for t in range(1, n + 1):
+        th, m, v = oracle.adamw_step(th, g, m, v, lr=lr, beta1=0.8, beta2=0.95, eps=eps, step=t)
+    np.testing.assert_allclose(th, th0 - n * lr * g / (np.abs(g) + eps), rtol=1e-10, atol=1e-12)
+    # zero gradient: only the decoupled decay acts, theta_n = theta_0 (1 - lr wd)^n, and the moments stay zero
+    th, m, v = th0, np.zeros_like(th0), np.zeros_like(th0)
+    for t in range(1, n + 1):
+        th, m, v = oracle.adamw_step(th, np.zeros_like(th0), m, v, lr=lr, weight_decay=0.3, step=t)
+    np.testing.assert_allclose(th, th0 * (1 - lr * 0.3) ** n, rtol=1e-12)
+    assert not m.any() and not v.any()
+
+
+def test_adamw_gradient_scale_is_a_scale_of_the_gradient():
+    th, g = _rand((3, 8), 905), _rand((3, 8), 906)
+    a = oracle.adamw_step(th, g, 0 * th, 0 * th, lr=0.02, grad_scale=0.25, step=1)
+    b = oracle.adamw_step(th, 0.25 * g, 0 * th, 0 * th, lr=0.02, step=1)
+    for x, y in zip(a, b):
+        np.testing.assert_allclose(x, y, rtol=1e-14)
+
+
+def test_adamw_agrees_with_the_library_optimizer_over_several_steps():
+    import torch
+    th0 = _rand((6, 9), 907)
+    hp = dict(lr=3e-2, beta1=0.9, beta2=0.98, eps=1e-6, weight_decay=0.05)
+    p = torch.nn.Parameter(torch.from_numpy(th0.copy()))
+    opt = torch.optim.AdamW([p], lr=hp["lr"], betas=(hp["beta1"], hp["beta2"]), eps=hp["eps"],
+                            weight_decay=hp["weight_decay"])
+    th, m, v = th0, np.zeros_like(th0), np.zeros_like(th0)
+    for t in range(1, 7):
+        g = _rand((6, 9), 910 + t)
+        p.grad = torch.from_numpy(g.copy())
+        opt.step()
+        th, m, v = oracle.adamw_step(th, g, m, v, step=t, **hp)
+        np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-11, atol=1e-13)
