@@ -51,6 +51,8 @@ SWEEPS = {
     # batch sizes x tenants of the rollout phases (the paper varies the number of concurrent tasks from 1 to 32)
     "decode": [f"decode-{T}-{n}" for T in (32, 64, 128, 256, 512, 1024) for n in (1, 8, 32)],
     "prefill": [f"prefill-{T}-{n}" for T in (8192, 16384, 32768) for n in (1, 8, 32)],
+    # projections that share their input, fused into one call against one call each, on a decode batch
+    "fused": [f"{k}-{T}-32" for T in (64, 256) for k in ("qkv", "qkvsep", "gateup", "gateupsep")],
 }
 
 
@@ -58,6 +60,10 @@ def workload_desc(name):
     if name in CFG_DESC:
         return CFG_DESC[name]
     kind, T, n = name.split("-")
+    if kind in ("qkv", "qkvsep", "gateup", "gateupsep"):
+        shape = "q, k, v (4096x4096 each)" if kind.startswith("qkv") else "gate, up (4096x11008 each)"
+        how = "one call each" if kind.endswith("sep") else "fused into one projection (block-diagonal B), one call"
+        return f"{shape}, {how}; {n} tenants r=16 per projection, {T} decode tokens, fwd only"
     what = "decode tokens (one per sequence, tenants uniform and unsorted)" if kind == "decode" else \
         "prompt tokens in whole-prompt lognormal segments"
     return f"{kind} sweep point: W 4096x4096, {n} tenants r=16, {T} {what}, fwd only"
@@ -312,7 +318,7 @@ def main():
     ap.add_argument("--workload", default="cfg3",
                     help="cfg1 .. cfg5, a forward-only sweep point decode-T-n / prefill-T-n (T tokens, n tenants), or adamw-n "
                          "(the fused optimizer step + commit of n tenants)")
-    ap.add_argument("--sweep", choices=["decode", "prefill"],
+    ap.add_argument("--sweep", choices=sorted(SWEEPS),
                     help="run a grid of sweep points, one bench.py process and one JSON line each")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--reference-tokens", type=int, default=1024)

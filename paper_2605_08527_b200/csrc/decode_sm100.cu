@@ -593,7 +593,7 @@ marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows,
 // host side
 // ---------------------------------------------------------------------------------------------------------------
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T) {
-    if (!(T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 1024 && pool->sm_count >= 8 && (pool->K % 64) == 0))
+    if (!(T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 2048 && pool->sm_count >= 8 && (pool->K % 64) == 0))
         return false;
     // beyond one 256-token tile only while all (token tile, 256-column strip) pairs make a single wave of CTA pairs
     return T <= 256 || cdiv(T, 256) * cdiv(pool->N, 256) <= pool->sm_count / 2;

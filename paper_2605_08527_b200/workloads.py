@@ -316,7 +316,34 @@ def make_workload(cfg: int, scale_down: int = 1, seed: Optional[int] = None) -> 
     raise ValueError(f"unknown config {cfg}")
 
 
-SWEEP_NAME = r"^(decode|prefill)-(\d+)-(\d+)$"
+def fuse_projections(w: Workload, names: Optional[List[str]] = None) -> Workload:
+    """Several projections that read the same x (q, k, v; gate, up) as ONE adapted projection, so that one layer call
+    serves them all: the base weights side by side ([d_in][sum d_out]), A_t side by side ([d_in][P r]), B_t block
+    diagonal ([P r][sum d_out], block p = B_t of projection p over that projection's output columns, zeros elsewhere).
+    Then y = x W + s (x A) B of the fused projection is the concatenation of the P separate layer outputs; the same
+    holds for dx (their sum), dA (side by side) and the diagonal blocks of dB.  Needs the same rank and alpha on
+    every projection of a tenant (so that one scale s = alpha / r serves all: the fused adapter gets alpha P)."""
+    projs = [p for p in w.projections if names is None or p.name in names]
+    assert projs and all(p.d_in == projs[0].d_in and p.x_bits is projs[0].x_bits for p in projs), "projections must share x"
+    P = len(projs)
+    offs = np.concatenate([[0], np.cumsum([p.d_out for p in projs])]).astype(np.int64)
+    adapters = []
+    for t, a0 in enumerate(projs[0].adapters):
+        parts = [p.adapters[t] for p in projs]
+        assert all(a.rank == a0.rank and a.alpha == a0.alpha and a.tenant_id == a0.tenant_id for a in parts)
+        r = a0.rank
+        A_bits = np.concatenate([a.A_bits for a in parts], axis=1)
+        B_bits = np.zeros((P * r, int(offs[-1])), dtype=np.uint16)
+        for i, a in enumerate(parts):
+            B_bits[i * r:(i + 1) * r, offs[i]:offs[i + 1]] = a.B_bits
+        adapters.append(Adapter(a0.tenant_id, P * r, a0.alpha * P, np.ascontiguousarray(A_bits), B_bits))
+    dy_bits = None if projs[0].dy_bits is None else np.ascontiguousarray(np.concatenate([p.dy_bits for p in projs], axis=1))
+    fused = Projection("+".join(p.name for p in projs), projs[0].d_in, int(offs[-1]),
+                       np.ascontiguousarray(np.concatenate([p.W_bits for p in projs], axis=1)), adapters, projs[0].x_bits, dy_bits)
+    return Workload(w.name + "-fused", w.T, w.T_bwd, w.seg_offsets, w.seg_slot, [fused], w.n_tenants, P * w.max_rank)
+
+
+SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|gateup|gateupsep)-(\d+)-(\d+)$"
 
 
 def make_named_workload(name: str) -> Workload:
@@ -325,7 +352,9 @@ def make_named_workload(name: str) -> Workload:
 
     ``decode-T-n``   T decode tokens (one per sequence), tenant of each token uniform over n tenants, unsorted;
     ``prefill-T-n``  T prompt tokens in whole-prompt segments (lognormal lengths, median 1024, clipped to
-                     [128, 4096]) dealt to n tenants in shuffled order."""
+                     [128, 4096]) dealt to n tenants in shuffled order;
+    ``qkv-T-n`` / ``gateup-T-n``  a decode batch through the fused q+k+v (4096 x 12288) or gate+up (4096 x 22016)
+                     projection, ``qkvsep`` / ``gateupsep`` through the same projections one call each."""
     import re
     if name.startswith("cfg") and name[3:].isdigit():
         return make_workload(int(name[3:]))
@@ -335,6 +364,23 @@ def make_named_workload(name: str) -> Workload:
     kind, T, n = m.group(1), int(m.group(2)), int(m.group(3))
     if T < 1 or n < 1 or n > 4096:
         raise ValueError(f"workload {name!r}: need T >= 1 and 1 <= tenants <= 4096")
+    if kind in ("qkv", "qkvsep", "gateup", "gateupsep"):
+        # projections of a 7B-shaped decoder layer that share their input, on a decode batch: q, k, v 4096 x 4096 or
+        # gate, up 4096 x 11008, rank 16 each; "...sep" runs them as separate projections (one call each), without
+        # the suffix they are fused into one (fuse_projections)
+        seed = BASE_SEED + 102
+        names, N = (("q", "k", "v"), 4096) if kind.startswith("qkv") else (("gate", "up"), 11008)
+        offsets, slots = per_token_table(uniform_token_slots(seed, T, n))
+        ranks, alphas = [16] * n, [32.0] * n
+        projs = [_make_projection(seed, nm, 4096, N, n, ranks, alphas, T, 0, pi, 0) for pi, nm in enumerate(names)]
+        for p in projs[1:]:
+            p.x_bits = projs[0].x_bits
+        w = Workload(name, T, 0, offsets, slots, projs, n, 16)
+        if kind.endswith("sep"):
+            return w
+        f = fuse_projections(w)
+        f.name = name
+        return f
     seed = BASE_SEED + 100 + (0 if kind == "decode" else 1)
     K = N = 4096
     if kind == "decode":
