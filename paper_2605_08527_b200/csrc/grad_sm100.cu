@@ -390,7 +390,25 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
                 tc_ld_32x16g(trow + j0, hi);
                 tc_ld_32x16g(trow + g.RP + j0, lo);
                 tc_wait_ld();
-                if (c < g.C) {
+                if (c < g.C && g.transpose_out && (r & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0) {
+                    // out is [C][r]: the thread's 16 ranks are contiguous, four per store
+                    float4* dst = reinterpret_cast<float4*>(out + (size_t)c * r + j0);
+#pragma unroll
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        if (j0 + 4 * e4 < r) {
+                            float4 v;
+                            v.x = sc * (__uint_as_float(hi[4 * e4]) + __uint_as_float(lo[4 * e4]));
+                            v.y = sc * (__uint_as_float(hi[4 * e4 + 1]) + __uint_as_float(lo[4 * e4 + 1]));
+                            v.z = sc * (__uint_as_float(hi[4 * e4 + 2]) + __uint_as_float(lo[4 * e4 + 2]));
+                            v.w = sc * (__uint_as_float(hi[4 * e4 + 3]) + __uint_as_float(lo[4 * e4 + 3]));
+                            if (g.accumulate) {
+                                const float4 o = dst[e4];
+                                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                            }
+                            dst[e4] = v;
+                        }
+                    }
+                } else if (c < g.C) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const int j = j0 + e;
