@@ -38,6 +38,7 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.ten_pos = (int32_t*)take(sizeof(int32_t) * gb * gc);
     w.gflag = (int32_t*)take(16);
     w.hm = (bf16*)take(sizeof(bf16) * (size_t)w.max_copies * 64 * (size_t)w.HW);
+    w.hm2 = (bf16*)take(sizeof(bf16) * (size_t)w.max_copies * 64 * (size_t)w.HW);
     w.total = o;
     return w;
 }
@@ -279,6 +280,23 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
         }
     }
+    // The adapter-gradient kernels read none of the dx GEMM's output: when they need no further pass over the workspace
+    // the GEMM uses (the saved h is given, the tensor-core reduction is certain to fit) they are issued on a side stream
+    // of the pool, forked here and joined at the end, so that their small planning and copy kernels run beside the
+    // GEMM instead of after it.
+    const bool tc_grad0 = tc_path && (want_dA || want_dB) && grad_sm100_eligible(pool, T);
+    const bool fits0 = tc_grad0 && cdiv(T, 64) + (int64_t)seg->num_segments <= (int64_t)ws.max_copies;
+    const bool overlap = fits0 && T > 0 && dx && (!want_dB || h_saved) && gemm2_sm100_eligible(pool, T) && pool->cap <= 64;
+    if (overlap) {
+        if (!pool->side) {
+            int lo = 0, hi = 0;
+            MARLAAS_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&lo, &hi));
+            MARLAAS_CUDA_TRY(cudaStreamCreateWithPriority(&pool->side, cudaStreamNonBlocking, lo));   // lowest priority
+            MARLAAS_CUDA_TRY(cudaEventCreateWithFlags(&pool->ev_fork, cudaEventDisableTiming));
+            MARLAAS_CUDA_TRY(cudaEventCreateWithFlags(&pool->ev_join, cudaEventDisableTiming));
+        }
+        MARLAAS_CUDA_TRY(cudaEventRecord(pool->ev_fork, st));
+    }
     if (T > 0 && dx && tc_path) {
         GemmOperands o;
         o.M = T; o.Nout = pool->K; o.Kc = pool->N;
@@ -305,6 +323,23 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         const bool fits = tc_grad && nblk + (int64_t)seg->num_segments <= (int64_t)ws.max_copies;
         const bool inline_tables = fits && pool->cap <= 64;
         const int32_t* run_flag = tc_grad ? ws.gflag : nullptr;   // the CUDA-core kernels run only if the flag is set
+        if (overlap) {
+            cudaStream_t gs = pool->side;
+            MARLAAS_CUDA_TRY(cudaStreamWaitEvent(gs, pool->ev_fork, 0));
+            if ((rc = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return rc;
+            // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
+            if (want_dB && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
+                                                   gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return rc;
+            if (want_dA && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
+                                                   gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return rc;
+            if (want_dB && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
+                                                   gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return rc;
+            if (want_dA && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
+                                                   gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return rc;
+            MARLAAS_CUDA_TRY(cudaEventRecord(pool->ev_join, gs));
+            MARLAAS_CUDA_TRY(cudaStreamWaitEvent(st, pool->ev_join, 0));
+            return finish(pool, flags, st);
+        }
         if (tc_grad && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
         if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
         if (want_dB) {
@@ -317,14 +352,14 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             }
             if (!inline_tables)
                 MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, dB_slots, false, acc, ws, st)) != MARLAAS_OK) return rc;
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, dB_slots, false, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
             if (!fits && (rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
                                                   false, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }
         if (want_dA) {
             if (!inline_tables)
                 MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, dA_slots, true, acc, ws, st)) != MARLAAS_OK) return rc;
+            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, dA_slots, true, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
             if (!fits && (rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
                                                   true, acc, st, run_flag)) != MARLAAS_OK) return rc;
         }

@@ -455,12 +455,15 @@ marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Wor
 marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
                                    const float* hg, float* const* out_ptrs, float* const* host_ptrs, bool transpose_out,
                                    bool accumulate,
-                                   const Workspace& ws, cudaStream_t st) {
+                                   const Workspace& ws, cudaStream_t st, bf16* hm, int phases) {
     using namespace sm100;
     const int nblk = (int)cdiv(T, 64);
-    k_pad_split<<<nblk, 256, 0, st>>>((int)T, pool->cap, pool->RP, ws.HW, hg, ws.tok_slot, ws.blk_base, ws.blk_rank,
-                                      ws.gflag, ws.hm);
-    MARLAAS_LAUNCH_CHECK("k_pad_split");
+    if (phases & GRAD_PHASE_COPIES) {
+        k_pad_split<<<nblk, 256, 0, st>>>((int)T, pool->cap, pool->RP, ws.HW, hg, ws.tok_slot, ws.blk_base, ws.blk_rank,
+                                          ws.gflag, hm);
+        MARLAAS_LAUNCH_CHECK("k_pad_split");
+    }
+    if (!(phases & GRAD_PHASE_REDUCE)) return MARLAAS_OK;
     GradArgs g;
     g.C = (int)C;
     g.num_c_tiles = (int)cdiv(C, 128);
@@ -486,7 +489,7 @@ marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t 
     alignas(64) CUtensorMap tmSrc, tmHm;
     marlaas_status_t rc;
     if ((rc = make_map(&tmSrc, src, T, C, ld, 64, 64)) != MARLAAS_OK) return rc;
-    if ((rc = make_map(&tmHm, ws.hm, (int64_t)ws.max_copies * 64, ws.HW, ws.HW, 64, 64)) != MARLAAS_OK) return rc;
+    if ((rc = make_map(&tmHm, hm, (int64_t)ws.max_copies * 64, ws.HW, ws.HW, 64, 64)) != MARLAAS_OK) return rc;
     constexpr size_t smem_bytes = 1024 + (size_t)GRAD_STAGES * (A_STAGE_BYTES + GB_STAGE_BYTES) + 256;
     static bool attr_set[64] = {};
     if (pool->device >= 64 || !attr_set[pool->device]) {

@@ -82,6 +82,9 @@ struct marlaas_pool {
     bool timing = false;
     std::vector<cudaEvent_t> timing_events;
     size_t timing_used = 0;
+    // backward: the adapter-gradient kernels run on a side stream beside the dx GEMM (created on first use)
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 namespace marlaas {
@@ -117,6 +120,7 @@ struct Workspace {
     int32_t* ten_pos;      // [cap][nblk]   the matching copy positions
     int32_t* gflag;        // [4]           [0] = 1 when the copies do not fit (CUDA-core reduction runs instead)
     bf16* hm;              // [max_copies*64][HW]  hi | lo split r-vectors
+    bf16* hm2;             // a second set of copies, so that the dB and dA reductions need not share one
     int32_t max_copies, HW;
     size_t total;
 };
@@ -195,9 +199,11 @@ marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const b
 // grad_sm100.cu: the same reductions on the tensor cores
 bool grad_sm100_eligible(const marlaas_pool* pool, int64_t T);
 marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Workspace& ws, cudaStream_t st);
+// phases: build the masked hi/lo copies of the r-vectors into hm, reduce from hm, or both
+enum { GRAD_PHASE_COPIES = 1, GRAD_PHASE_REDUCE = 2 };
 marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
                                    const float* hg, float* const* out_ptrs, float* const* host_ptrs, bool transpose_out,
-                                   bool accumulate, const Workspace& ws, cudaStream_t st);
+                                   bool accumulate, const Workspace& ws, cudaStream_t st, bf16* hm, int phases = GRAD_PHASE_COPIES | GRAD_PHASE_REDUCE);
 // host_ptrs: the same table in host memory; pools of at most 64 slots pass it with the launch and never read out_ptrs
 
 }  // namespace marlaas

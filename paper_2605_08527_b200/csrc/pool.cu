@@ -179,8 +179,12 @@ marlaas_status_t marlaas_kernel_timing_end(marlaas_pool_t* pool, float* gemm_ms,
 }
 
 marlaas_status_t marlaas_adapter_pool_destroy(marlaas_pool_t* pool) {
-    if (pool)
+    if (pool) {
         for (cudaEvent_t e : pool->timing_events) cudaEventDestroy(e);
+        if (pool->ev_fork) cudaEventDestroy(pool->ev_fork);
+        if (pool->ev_join) cudaEventDestroy(pool->ev_join);
+        if (pool->side) cudaStreamDestroy(pool->side);
+    }
     delete pool;
     return MARLAAS_OK;
 }
