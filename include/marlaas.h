@@ -175,7 +175,11 @@ marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T,
  * skip); dA_t is [d_in][r_t], dB_t is [r_t][d_out], row-major, at the slot's true rank.  Without
  * MARLAAS_FLAG_ACCUMULATE every non-NULL slot is overwritten (tenants with no token in the batch get exact
  * zeros); with it the batch's contribution is added.  The sums over a tenant's tokens run over all of its
- * segments.  h_saved: what forward wrote to h_save for the same batch and adapters, or NULL = recompute. */
+ * segments.  h_saved: what forward wrote to h_save for the same batch and adapters, or NULL = recompute.
+ * Part of the work (the adapter-gradient kernels, when h_saved is given) may be issued on a stream that the pool
+ * owns, forked from cuda_stream after the call's first kernels and joined to it before the call returns (events;
+ * legal inside a stream capture): everything the call writes is ordered on cuda_stream as if issued there.  Calls
+ * on one pool are not to be issued from several host threads at once. */
 marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx,
                                        const void* W, int64_t ldw, const void* dy, int64_t lddy,
                                        void* dx, int64_t lddx, float* const* dA_slots, float* const* dB_slots,
