@@ -18,7 +18,8 @@ namespace marlaas {
 namespace sm100 {
 
 constexpr int GRAD_THREADS = 192;
-constexpr int GRAD_STAGES = 4;
+constexpr int GRAD_STAGES = 4;          // at most: as many steps as fit the shared-memory budget (see the launch)
+constexpr int GRAD_BPS = 2;              // 64-token blocks per pipeline step: one barrier round trip and one commit for both
 constexpr int GRAD_INLINE_SLOTS = 64;
 constexpr int GRAD_QN = 4;               // depth of the CTA's work-item queue
 constexpr uint32_t GB_STAGE_BYTES = 4 * CHUNK_BYTES;   // up to 256 columns of split r-vectors
@@ -181,35 +182,39 @@ struct GradArgs {
     int32_t* counter;      // next work item (zeroed by the plan kernel before every pair of launches)
     float* const* out_ptrs;   // per-slot outputs in device memory, or nullptr: the table is inl[] below
     int transpose_out, accumulate;
+    int stages;            // pipeline steps in flight
     int32_t* status;
     float* inl[GRAD_INLINE_SLOTS];   // small pools: the pointer table travels with the launch (no host-to-device copy)
 };
 
 __global__ void __launch_bounds__(GRAD_THREADS, 1)
 k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ CUtensorMap tmHm, const GradArgs g) {
-    constexpr int STAGES = GRAD_STAGES;
+    constexpr int MAX_STAGES = GRAD_STAGES;
+    const int STAGES = g.stages;
     constexpr uint32_t TMEM_COLS = 512;
     if (g.gflag[0] != 0) return;   // copies did not fit: the CUDA-core reduction handles this call
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sA = smem_u32(smem);
-    const uint32_t sB = sA + STAGES * A_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + GB_STAGE_BYTES));
+    const int hw_chunks = g.HW / 64;
+    const uint32_t B_BLOCK = (uint32_t)hw_chunks * CHUNK_BYTES;      // one block's split r-vectors
+    const uint32_t A_STEP = GRAD_BPS * A_STAGE_BYTES, B_STEP = GRAD_BPS * B_BLOCK;
+    const uint32_t sB = sA + STAGES * A_STEP;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STEP + B_STEP));
     const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_empty = bar_full + 8 * STAGES;
-    const uint32_t bar_tfull = bar_empty + 8 * STAGES;
+    const uint32_t bar_empty = bar_full + 8 * MAX_STAGES;
+    const uint32_t bar_tfull = bar_empty + 8 * MAX_STAGES;
     const uint32_t bar_tempty = bar_tfull + 16;
     const uint32_t bar_drain = bar_tempty + 16;
     const uint32_t bar_qfull = bar_drain + 8, bar_qempty = bar_qfull + 8 * GRAD_QN;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 2 * GRAD_QN);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 5 + 2 * GRAD_QN);
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
     __shared__ int s_cnt[256], s_order[256];
     __shared__ volatile int s_q[GRAD_QN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_items = g.num_c_tiles * g.cap;
-    const int hw_chunks = g.HW / 64;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -261,7 +266,7 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
 
     if (warp == 0) {
         if (lane == 0) {   // ---- TMA producer
-            uint32_t it = 0, qi = 0;
+            uint32_t it = 0, qi = 0, ps = 0, pph = 0;    // steps issued; stage and phase of the next step
             bool ok = true;
             while (ok) {
                 const uint32_t qs = qi % GRAD_QN, qph = (qi / GRAD_QN) & 1;
@@ -276,17 +281,21 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
                 const int nb = item_blocks(item, t, c0);
                 if (nb <= 0) continue;
                 const int a_chunks = min(2, (g.C - c0 + 63) / 64);
-                for (int k = 0; k < nb && ok; ++k, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int k = 0; k < nb && ok; k += GRAD_BPS, ++it) {
+                    const uint32_t s = ps, ph = pph;
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 21))) break;
-                    const int blk = g.ten_blks[(size_t)t * g.nblk + k];
-                    const int pos = g.ten_pos[(size_t)t * g.nblk + k];
+                    if (++ps == (uint32_t)STAGES) { ps = 0; pph ^= 1; }
+                    const int nj = min(GRAD_BPS, nb - k);
                     const uint32_t full = bar_full + 8 * s;
-                    mbar_expect_tx(full, (a_chunks + hw_chunks) * CHUNK_BYTES);
-                    for (int c = 0; c < a_chunks; ++c)
-                        tma_load_2d(sA + s * A_STAGE_BYTES + c * CHUNK_BYTES, &tmSrc, full, c0 + c * 64, blk * 64);
-                    for (int c = 0; c < hw_chunks; ++c)
-                        tma_load_2d(sB + s * GB_STAGE_BYTES + c * CHUNK_BYTES, &tmHm, full, c * 64, pos * 64);
+                    mbar_expect_tx(full, (uint32_t)nj * (a_chunks + hw_chunks) * CHUNK_BYTES);
+                    for (int j = 0; j < nj; ++j) {
+                        const int blk = g.ten_blks[(size_t)t * g.nblk + k + j];
+                        const int pos = g.ten_pos[(size_t)t * g.nblk + k + j];
+                        for (int c = 0; c < a_chunks; ++c)
+                            tma_load_2d(sA + s * A_STEP + j * A_STAGE_BYTES + c * CHUNK_BYTES, &tmSrc, full, c0 + c * 64, blk * 64);
+                        for (int c = 0; c < hw_chunks; ++c)
+                            tma_load_2d(sB + s * B_STEP + j * B_BLOCK + c * CHUNK_BYTES, &tmHm, full, c * 64, pos * 64);
+                    }
                 }
             }
             if (!ok) {
@@ -304,7 +313,7 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
     } else if (warp == 1) {
         if (lane == 0) {   // ---- MMA issuer: A and B both MN-major, M = 128, N = HW
             const uint32_t idesc = make_idesc(g.HW, 1) | (1u << 15);
-            uint32_t it = 0, lt = 0;
+            uint32_t it = 0, lt = 0, ms = 0, mph = 0;
             bool ok = true;
             uint32_t qi = 0;
             while (ok) {
@@ -322,17 +331,21 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + b * 256;
                 uint32_t acc = 0;
-                for (int k = 0; k < nb && ok; ++k, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int k = 0; k < nb && ok; k += GRAD_BPS, ++it) {
+                    const uint32_t s = ms, ph = mph;
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 24))) break;
+                    if (++ms == (uint32_t)STAGES) { ms = 0; mph ^= 1; }
                     tc_fence_after();
-                    const uint32_t a0 = sA + s * A_STAGE_BYTES, b0 = sB + s * GB_STAGE_BYTES;
-                    // descriptors of successive 16-token slices differ only in the start-address field (16-byte units)
-                    const uint64_t da0 = desc_mn_major(a0, CHUNK_BYTES), db0 = desc_mn_major(b0, CHUNK_BYTES);
+                    const int nj = min(GRAD_BPS, nb - k);
+                    for (int jb = 0; jb < nj; ++jb) {
+                        const uint32_t a0 = sA + s * A_STEP + jb * A_STAGE_BYTES, b0 = sB + s * B_STEP + jb * B_BLOCK;
+                        // descriptors of successive 16-token slices differ only in the start-address field (16-byte units)
+                        const uint64_t da0 = desc_mn_major(a0, CHUNK_BYTES), db0 = desc_mn_major(b0, CHUNK_BYTES);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        tc_mma_bf16(d_tmem, da0 + (uint64_t)(j * (UNIT_BYTES >> 4)), db0 + (uint64_t)(j * (UNIT_BYTES >> 4)), idesc, acc);
-                        acc = 1;
+                        for (int j = 0; j < 4; ++j) {
+                            tc_mma_bf16(d_tmem, da0 + (uint64_t)(j * (UNIT_BYTES >> 4)), db0 + (uint64_t)(j * (UNIT_BYTES >> 4)), idesc, acc);
+                            acc = 1;
+                        }
                     }
                     tc_commit(bar_empty + 8 * s);
                 }
@@ -490,7 +503,10 @@ marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t 
     marlaas_status_t rc;
     if ((rc = make_map(&tmSrc, src, T, C, ld, 64, 64)) != MARLAAS_OK) return rc;
     if ((rc = make_map(&tmHm, hm, (int64_t)ws.max_copies * 64, ws.HW, ws.HW, 64, 64)) != MARLAAS_OK) return rc;
-    constexpr size_t smem_bytes = 1024 + (size_t)GRAD_STAGES * (A_STAGE_BYTES + GB_STAGE_BYTES) + 256;
+    // as many steps of GRAD_BPS blocks as fit what four single-block steps of the widest r-vectors take
+    constexpr size_t smem_bytes = 1024 + (size_t)4 * (A_STAGE_BYTES + GB_STAGE_BYTES) + 256;
+    const size_t step_bytes = (size_t)GRAD_BPS * (A_STAGE_BYTES + (size_t)(ws.HW / 64) * CHUNK_BYTES);
+    g.stages = (int)std::min<size_t>(GRAD_STAGES, (smem_bytes - 1024 - 256) / step_bytes);
     static bool attr_set[64] = {};
     if (pool->device >= 64 || !attr_set[pool->device]) {
         MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_grad_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
