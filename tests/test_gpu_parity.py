@@ -348,3 +348,37 @@ def test_malformed_calls_return_status_codes_and_launch_nothing():
     e = B.marlaas_lora_forward(dc.pool, dc.x[:0], dc.W, B.Segments(torch.zeros(1, dtype=torch.int32).cuda(),
                                                                   torch.zeros(0, dtype=torch.int32).cuda()))
     assert e.shape[0] == 0
+
+
+def test_backward_inside_a_stream_capture_replays_to_the_same_bits():
+    # training-shaped batch large enough for the 2-CTA GEMM, saved h given: the adapter-gradient kernels go to the
+    # pool's side stream (fork / join by events), which a capture must be able to hold; the replayed graph has to
+    # reproduce the directly issued call bit for bit, twice
+    w = wl.make_workload(4, scale_down=4)
+    p = w.projections[0]
+    dc = DeviceCase(w, p)
+    hs = torch.empty((w.T, dc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+    dc.forward(h_save=hs)
+    dx0, dA0, dB0 = dc.backward(h_saved=hs)
+    torch.cuda.synchronize()
+    dx = torch.zeros_like(dx0)
+    dA, dB = dc.grads(fill=0.0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            B.marlaas_lora_backward(dc.pool, dc.x, dc.W, dc.dy, dc.seg, dx=dx, dA=dA, dB=dB, h_saved=hs)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        dx.fill_(7.0)
+        for t in dA + dB:
+            if t is not None:
+                t.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dx, dx0)
+        for a, b in zip(dA + dB, dA0 + dB0):
+            if a is not None:
+                assert torch.equal(a, b)
+    B.marlaas_check_status(dc.pool)
