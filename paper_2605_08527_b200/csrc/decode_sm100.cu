@@ -82,7 +82,7 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
 // Operand fragments of the m16n8k16 MMA come straight from global memory with 16-byte loads: within a 32-deep
 // k-block lane (g, t) reads elements 8t .. 8t+7 of its rows, and the same element-to-position permutation is used
 // for the token rows (A fragment) and the adapter rows (B fragment), so every product pairs matching k.
-__global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrinkArgs g) {
+__global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShrinkArgs g) {
     __shared__ DecodeShrinkSmem sm;
     dk_launch_dependents();      // the GEMM may start streaming W now; it waits for this grid before the expand
 
@@ -95,6 +95,27 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     const bool first = (dk_cluster_id_x() == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
     const int r_t = t < g.cap ? g.d_rank[t] : 0;
     const float sc = t < g.cap ? g.d_scale[t] : 0.f;
+
+    // This warp's share of K: the cluster's CTAs split the 32-deep k-blocks, then each CTA's warps do.  The adapter rows
+    // of the tenant's first rank group do not depend on the token list, and a load issued beside the GEMM's stream takes
+    // microseconds to come back: they are requested before anything else.
+    const int nb32 = (g.K + 31) >> 5;
+    const int cb0 = (int)((int64_t)crank * nb32 / cs), cb1 = (int)((int64_t)(crank + 1) * nb32 / cs);
+    const int wb0 = cb0 + (int)((int64_t)warp * (cb1 - cb0) / 4), wb1 = cb0 + (int)((int64_t)(warp + 1) * (cb1 - cb0) / 4);
+    const int gq = lane >> 2, tq = lane & 3;
+    uint4 ba[DS_UB], bb[DS_UB];     // adapter fragments; held_jg / held_b0 say of which rank group and k-block batch
+    int held_jg = 0, held_b0 = wb0;
+    {
+        const bf16* ar0 = g.At + ((size_t)(t < g.cap ? t : 0) * g.RP + gq) * g.K;
+        const bf16* ar1 = ar0 + (size_t)8 * g.K;
+#pragma unroll
+        for (int u = 0; u < DS_UB; ++u) {
+            const int k = (wb0 + u) * 32 + tq * 8;
+            const bool in = t < g.cap && (wb0 + u) < wb1 && k < g.K;
+            ba[u] = in ? ldg_nc_v4(ar0 + k) : make_uint4(0u, 0u, 0u, 0u);
+            bb[u] = in ? ldg_nc_v4(ar1 + k) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
 
     // ---- per-token slot ------------------------------------------------------------------------------------
     if (g.S >= 0) {
@@ -172,11 +193,6 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
     const int ngroups = (r_t + 15) >> 4;
 
     // ---- partial products over this warp's share of K --------------------------------------------------------
-    // 32-deep k-blocks [kb0, kb1) of this warp: the cluster's CTAs split the blocks, then each CTA's warps do
-    const int nb32 = (g.K + 31) >> 5;
-    const int cb0 = (int)((int64_t)crank * nb32 / cs), cb1 = (int)((int64_t)(crank + 1) * nb32 / cs);
-    const int wb0 = cb0 + (int)((int64_t)warp * (cb1 - cb0) / 4), wb1 = cb0 + (int)((int64_t)(warp + 1) * (cb1 - cb0) / 4);
-    const int gq = lane >> 2, tq = lane & 3;
     const uint32_t part_rank0 = dk_map_to_cta(smem_u32(&sm.part[0][0]), 0);
 
     // zero the other tenants' columns of this cluster's hd rows (and, with no adapter, the h rows): one warp per row
@@ -200,7 +216,8 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
             const bf16* ar0 = g.At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
             const bf16* ar1 = ar0 + (size_t)8 * g.K;
             for (int b0 = wb0; b0 < wb1; b0 += DS_UB) {
-                uint4 xa[DS_UB], xb[DS_UB], ba[DS_UB], bb[DS_UB];
+                uint4 xa[DS_UB], xb[DS_UB];
+                const bool held = held_jg == jg && held_b0 == b0;     // the adapter fragments are in registers already
 #pragma unroll
                 for (int u = 0; u < DS_UB; ++u) {
                     const int k = (b0 + u) * 32 + tq * 8;
@@ -208,9 +225,13 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
                     const uint4 z = make_uint4(0u, 0u, 0u, 0u);
                     xa[u] = (in && xr0) ? ldg_nc_v4(xr0 + k) : z;
                     xb[u] = (in && xr1) ? ldg_nc_v4(xr1 + k) : z;
-                    ba[u] = in ? ldg_nc_v4(ar0 + k) : z;
-                    bb[u] = in ? ldg_nc_v4(ar1 + k) : z;
+                    if (!held) {
+                        ba[u] = in ? ldg_nc_v4(ar0 + k) : z;
+                        bb[u] = in ? ldg_nc_v4(ar1 + k) : z;
+                    }
                 }
+                held_jg = jg;
+                held_b0 = b0;
 #pragma unroll
                 for (int u = 0; u < DS_UB; ++u) {
                     mma_bf16_16816(c0, xa[u].x, xb[u].x, xa[u].y, xb[u].y, ba[u].x, ba[u].y);
@@ -220,7 +241,9 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
                 }
             }
             // warp partials -> CTA partial (fixed order) -> cluster rank 0
-            __syncthreads();        // wpart of the previous group has been consumed
+            const bool first_round = p0 == gi * DS_PASS && jg == 0;
+            const bool last_round = p0 + DS_PASS * g.G >= n_t && jg == ngroups - 1;
+            if (!first_round) __syncthreads();      // wpart of the previous group has been consumed
             {
                 float* wp = sm.wpart[warp];
                 wp[gq * 16 + 2 * tq] = c0[0];
@@ -250,7 +273,8 @@ __global__ void __launch_bounds__(DS_THREADS) k_decode_shrink(const DecodeShrink
                     }
                 }
             }
-            dk_cluster_sync();      // rank 0 has read the partials before they are overwritten
+            if (!last_round) dk_cluster_sync();     // rank 0 has read the partials before they are overwritten (its own
+                                                    // shared memory: after the last round the other CTAs may leave)
         }
         // ranks beyond the tenant's true rank (rounded up to 16) stay zero
         if (crank == 0) {
