@@ -47,18 +47,19 @@ struct DecodeShrinkArgs {
     int32_t* status;
 };
 
+// Shared memory: the fixed part below, then (dynamic, sized by the launch) slot[T'], off_tab[max(S + 1, T')] whose
+// space the cluster's token list takes over once every token has its slot, and slot_tab[S]; T' = T rounded up to 32.
+// Keeping this small matters: two of these CTAs share an SM with a GEMM CTA, whose pipeline gets what is left.
 struct __align__(16) DecodeShrinkSmem {
     float wpart[4][256];                // per-warp [16 tokens][16 ranks] partial products
     float part[DS_MAX_CS][256];         // per-CTA partials, gathered in cluster rank 0
-    int32_t slot[DS_MAX_T];
-    union {
-        int32_t off_tab[DS_TABLE_SMEM];  // the staged table is dead once every token has its slot:
-        int32_t list[DS_MAX_T];          // the cluster's token list takes its place
-    };
-    int32_t slot_tab[DS_TABLE_SMEM];
     int32_t cnt[DS_ROUNDS * 4];
 };
-static_assert(DS_TABLE_SMEM >= DS_MAX_T, "the token list reuses the table's space");
+static size_t decode_shrink_dyn_smem(int64_t T, int32_t S) {
+    const size_t Tp = (size_t)((T + 31) / 32 * 32);
+    const bool staged = S >= 0 && S + 1 <= DS_TABLE_SMEM;
+    return 4 * (Tp + std::max<size_t>(staged ? (size_t)S + 1 : 0, Tp) + (staged ? (size_t)S : 0));
+}
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -84,6 +85,13 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
 // for the token rows (A fragment) and the adapter rows (B fragment), so every product pairs matching k.
 __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShrinkArgs g) {
     __shared__ DecodeShrinkSmem sm;
+    extern __shared__ int32_t ds_dyn[];
+    const int Tp = (g.T + 31) / 32 * 32;
+    const bool staged_tab = g.S >= 0 && g.S + 1 <= DS_TABLE_SMEM;
+    int32_t* const s_slot = ds_dyn;
+    int32_t* const s_off = ds_dyn + Tp;             // the segment offsets, later the token list
+    int32_t* const s_list = s_off;
+    int32_t* const s_stab = s_off + max(staged_tab ? g.S + 1 : 0, Tp);
     dk_launch_dependents();      // the GEMM may start streaming W now; it waits for this grid before the expand
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -119,17 +127,17 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
 
     // ---- per-token slot ------------------------------------------------------------------------------------
     if (g.S >= 0) {
-        const bool staged = g.S + 1 <= DS_TABLE_SMEM;
+        const bool staged = staged_tab;
         if (staged) {
             for (int s = tid; s <= g.S; s += DS_THREADS) {
-                sm.off_tab[s] = g.seg_offsets[s];
-                if (s < g.S) sm.slot_tab[s] = g.seg_slot[s];
+                s_off[s] = g.seg_offsets[s];
+                if (s < g.S) s_stab[s] = g.seg_slot[s];
             }
             __syncthreads();
         }
         if (first) {
             for (int s = tid; s < g.S; s += DS_THREADS) {
-                const int a = staged ? sm.off_tab[s] : g.seg_offsets[s], b = staged ? sm.off_tab[s + 1] : g.seg_offsets[s + 1];
+                const int a = staged ? s_off[s] : g.seg_offsets[s], b = staged ? s_off[s + 1] : g.seg_offsets[s + 1];
                 if (b < a || a < 0 || b > g.T) dk_report(g.status, DEV_BAD_TABLE, s);
                 if (s == 0 && a != 0) dk_report(g.status, DEV_BAD_TABLE, -1);
                 if (s == g.S - 1 && b != g.T) dk_report(g.status, DEV_BAD_TABLE, -2);
@@ -140,18 +148,18 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
             int lo = 0, hi = g.S;
             while (lo < hi) {       // first s with seg_offsets[s + 1] > i
                 const int mid = (lo + hi) >> 1;
-                const int v = staged ? sm.off_tab[mid + 1] : g.seg_offsets[mid + 1];
+                const int v = staged ? s_off[mid + 1] : g.seg_offsets[mid + 1];
                 if (v > i) hi = mid; else lo = mid + 1;
             }
-            sm.slot[i] = lo < g.S ? (staged ? sm.slot_tab[lo] : g.seg_slot[lo]) : -1;
+            s_slot[i] = lo < g.S ? (staged ? s_stab[lo] : g.seg_slot[lo]) : -1;
         }
     } else {
-        for (int i = tid; i < g.T; i += DS_THREADS) sm.slot[i] = g.tok_slot[i];
+        for (int i = tid; i < g.T; i += DS_THREADS) s_slot[i] = g.tok_slot[i];
     }
     __syncthreads();
     if (first)
         for (int i = tid; i < g.T; i += DS_THREADS) {
-            int s = sm.slot[i];
+            int s = s_slot[i];
             if (s < -1 || s >= g.cap) {
                 dk_report(g.status, DEV_BAD_INDEX, i);
                 s = -1;
@@ -167,7 +175,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
         const int i = r * DS_THREADS + tid;
         bool m = false;
         if (i < g.T) {
-            const int s = sm.slot[i];
+            const int s = s_slot[i];
             m = (t < g.cap) ? (s == t) : (s < 0 || s >= g.cap);
         }
         mine[r] = m;
@@ -183,7 +191,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
         if (mine[r]) {
             int off = __popc(bal[r] & ((1u << lane) - 1u));
             for (int e = 0; e < r * 4 + warp; ++e) off += sm.cnt[e];
-            sm.list[off] = r * DS_THREADS + tid;
+            s_list[off] = r * DS_THREADS + tid;
         }
     }
     __syncthreads();
@@ -198,7 +206,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     // zero the other tenants' columns of this cluster's hd rows (and, with no adapter, the h rows): one warp per row
     for (int e = crank * 4 + warp; e < n_t; e += cs * 4) {
         if ((e / DS_PASS) % g.G != gi) continue;     // another cluster's pass
-        const int tok = sm.list[e];
+        const int tok = s_list[e];
         bf16* row = g.hd + (size_t)tok * g.hd_cols;
         for (int c = lane * 8; c < g.hd_cols; c += 256)
             if (c < own0 || c >= own1) *reinterpret_cast<uint4*>(row + c) = make_uint4(0u, 0u, 0u, 0u);
@@ -209,8 +217,8 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
 
     for (int p0 = gi * DS_PASS; p0 < n_t; p0 += DS_PASS * g.G) {
         const int np = min(DS_PASS, n_t - p0);
-        const bf16* xr0 = gq < np ? g.x + (size_t)sm.list[p0 + gq] * g.ldx : nullptr;
-        const bf16* xr1 = gq + 8 < np ? g.x + (size_t)sm.list[p0 + gq + 8] * g.ldx : nullptr;
+        const bf16* xr0 = gq < np ? g.x + (size_t)s_list[p0 + gq] * g.ldx : nullptr;
+        const bf16* xr1 = gq + 8 < np ? g.x + (size_t)s_list[p0 + gq + 8] * g.ldx : nullptr;
         for (int jg = 0; jg < ngroups; ++jg) {
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
             const bf16* ar0 = g.At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
@@ -267,7 +275,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
                     if (i < np) {
                         float v = 0.f;
                         for (int s = 0; s < cs; ++s) v += sm.part[s][e];   // fixed order
-                        const int tok = sm.list[p0 + i];
+                        const int tok = s_list[p0 + i];
                         g.h_out[(size_t)tok * g.RP + jg * 16 + j] = v;
                         g.hd[(size_t)tok * g.hd_cols + own0 + jg * 16 + j] = __float2bfloat16_rn(sc * v);
                     }
@@ -281,7 +289,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
             const int rest = g.RP - ngroups * 16;
             for (int e = tid; e < np * rest; e += DS_THREADS) {
                 const int i = e / rest, j = ngroups * 16 + e % rest;
-                const int tok = sm.list[p0 + i];
+                const int tok = s_list[p0 + i];
                 g.h_out[(size_t)tok * g.RP + j] = 0.f;
                 g.hd[(size_t)tok * g.hd_cols + own0 + j] = __float2bfloat16_rn(0.f);
             }
@@ -653,7 +661,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)((pool->cap + 1) * a.G * cs));
         cfg.blockDim = dim3(DS_THREADS);
-        cfg.dynamicSmemBytes = 0;
+        cfg.dynamicSmemBytes = decode_shrink_dyn_smem(T, S);
         cfg.stream = st;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension;
@@ -683,7 +691,7 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
         const int ci = sh.S == 1 ? 0 : sh.S == 2 ? 1 : 2;
         int mc = pool->device < 64 ? max_clusters[pool->device][ci] : 0;
         if (mc == 0) {
-            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, DG_SMEM));
+            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             cudaLaunchConfig_t qc = {};
             qc.gridDim = dim3((unsigned)(csz * 64));
             qc.blockDim = dim3(DG_THREADS);
@@ -709,9 +717,11 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
     g.S = pick.S; g.nch = pick.nch;
     g.kp = DG_KP;
     const size_t step_bytes = (size_t)g.kp * (A_STAGE_BYTES + g.nch * CHUNK_BYTES);
-    // leave room for two shrink CTAs (25 KB static + 1 KB system reservation each) on the same SM: the shrink then
-    // overlaps the GEMM's main loop instead of delaying its start (measured: 23 us per call against 29 us)
-    g.stages = (int)((DG_SMEM - 1024 - 256 - 2 * 26 * 1024) / step_bytes);
+    // leave room for two shrink CTAs (their static and dynamic shared memory + 1 KB system reservation each) on the same
+    // SM: the shrink then overlaps the GEMM's main loop instead of delaying its start (measured: 23 us per call against
+    // 29 us); what is left of the SM's 227 KB goes to the pipeline (4 steps at 256 tokens, 3 at 1024)
+    const size_t shrink_smem = sizeof(DecodeShrinkSmem) + decode_shrink_dyn_smem(T, S) + 1024;
+    g.stages = (int)std::min<size_t>(6, ((size_t)227 * 1024 - 2 * shrink_smem - 1024 - 256 - 1024) / step_bytes);
     if (g.stages < 2) g.stages = 2;
     g.num_ks = (int)cdiv(K, (int64_t)g.kp * BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)g.kp * BK);
