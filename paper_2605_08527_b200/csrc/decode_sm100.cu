@@ -108,8 +108,8 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     // of the tenant's first rank group do not depend on the token list, and a load issued beside the GEMM's stream takes
     // microseconds to come back: they are requested before anything else.
     const int nb32 = (g.K + 31) >> 5;
-    const int cb0 = (int)((int64_t)crank * nb32 / cs), cb1 = (int)((int64_t)(crank + 1) * nb32 / cs);
-    const int wb0 = cb0 + (int)((int64_t)warp * (cb1 - cb0) / 4), wb1 = cb0 + (int)((int64_t)(warp + 1) * (cb1 - cb0) / 4);
+    const int cb0 = crank * nb32 / cs, cb1 = (crank + 1) * nb32 / cs;        // (32-bit: 64-bit division is slow, and these
+    const int wb0 = cb0 + warp * (cb1 - cb0) / 4, wb1 = cb0 + (warp + 1) * (cb1 - cb0) / 4;   // precede the first loads)
     const int gq = lane >> 2, tq = lane & 3;
     uint4 ba[DS_UB], bb[DS_UB];     // adapter fragments; held_jg / held_b0 say of which rank group and k-block batch
     int held_jg = 0, held_b0 = wb0;
@@ -342,27 +342,10 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t crank = dk_cluster_ctarank();
-    const uint32_t half = crank & 1;            // which 128 rows of the 256-row tile
-    const uint32_t pairi = crank >> 1;          // which slice of the contraction
-    const uint32_t leader = crank & ~1u;
     const int NP = 128 * g.nch;                 // columns of the cluster's strip
-    const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
-    const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
-    const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
     const uint32_t tmem_cols = (uint32_t)NP;    // 128 or 256
-
-    const int ks0 = (int)((int64_t)pairi * g.num_ks / g.S), ks1 = (int)((int64_t)(pairi + 1) * g.num_ks / g.S);
-    const int xs0 = (int)((int64_t)pairi * g.num_xs / g.S), xs1 = (int)((int64_t)(pairi + 1) * g.num_xs / g.S);
-
-    const int qper = 4 / g.S;
-    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
-    uint32_t live = 0;
-    for (int p = 0; p < g.S; ++p) {
-        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
-        if (n > 0) live |= 1u << p;
-    }
-    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
+    // set-up first (one thread the barriers, one the descriptor prefetches, one warp the tensor-memory allocation): the
+    // index arithmetic below holds a dozen integer divisions, a microsecond if it came before
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -373,6 +356,8 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x == 64) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
         if (g.num_xs > 0) {
@@ -386,6 +371,25 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
+    const uint32_t crank = dk_cluster_ctarank();
+    const uint32_t half = crank & 1;            // which 128 rows of the 256-row tile
+    const uint32_t pairi = crank >> 1;          // which slice of the contraction
+    const uint32_t leader = crank & ~1u;
+    const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
+    const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
+    const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
+
+    const int ks0 = (int)pairi * g.num_ks / g.S, ks1 = ((int)pairi + 1) * g.num_ks / g.S;
+    const int xs0 = (int)pairi * g.num_xs / g.S, xs1 = ((int)pairi + 1) * g.num_xs / g.S;
+
+    const int qper = 4 / g.S;
+    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
+    uint32_t live = 0;
+    for (int p = 0; p < g.S; ++p) {
+        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
+        if (n > 0) live |= 1u << p;
+    }
+    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     tc_fence_before();
     __syncthreads();
     dk_cluster_sync();      // every CTA's barriers exist before any remote arrive or TMA completion
