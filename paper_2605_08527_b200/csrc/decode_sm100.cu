@@ -391,7 +391,6 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     }
     const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     tc_fence_before();
-    __syncthreads();
     dk_cluster_sync();      // every CTA's barriers exist before any remote arrive or TMA completion
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
@@ -511,7 +510,6 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const uint32_t own = (uint32_t)(q % g.S);
     if (g.S > 1) {
         tc_fence_before();
-        __syncthreads();
         dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
         tc_fence_after();
         if (warp >= 2 && epi_ok && own != pairi && ((live >> pairi) & 1u)) {
@@ -585,7 +583,6 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     // ---- teardown ---------------------------------------------------------------------------------------------
     tc_fence_before();
-    __syncthreads();
     dk_cluster_sync();      // the pair leaves together (its barriers and tensor memory are shared)
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
