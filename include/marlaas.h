@@ -62,7 +62,10 @@ enum {
     MARLAAS_FLAG_HOST_TABLE = 2u,     /* seg_offsets / seg_slot are HOST arrays: validated on the host, then copied
                                          into the workspace in stream order */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
-    MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
+    MARLAAS_FLAG_CUDA_CORE_PATH = 8u, /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
+    MARLAAS_FLAG_SERIAL_KERNELS = 16u /* diagnostics: the decode-shaped forward normally runs its two kernels side by
+                                         side, the second feeding the first; tools that run one kernel at a time
+                                         (profilers, CUDA_LAUNCH_BLOCKING=1) need this flag, which orders them plainly */
 };
 
 /* Token-to-adapter segment table of one mixed batch: segment s covers tokens
@@ -138,6 +141,8 @@ int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool);
 /* Bytes of workspace forward/backward need for a batch of T tokens on this pool (device memory, 256-byte
  * aligned, contents need not be preserved between calls; two calls in flight need two workspaces). */
 size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
+/* The part of that workspace a forward call uses (its leading bytes): enough for marlaas_lora_forward alone. */
+size_t marlaas_lora_forward_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
 
 /* Forward: y[T][d_out] = x[T][d_in] W + s_t (x A_t) B_t with t from the segment table.
  * x (ldx >= d_in), W (ldw >= d_out), y (ldy >= d_out): bf16 row-major.  h_save: optional fp32
@@ -153,14 +158,17 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
  * a serving loop whose memory pool was sized and frozen at start-up, a plug-in that is handed nothing but its
  * input and output buffers, a latency-critical path that cannot afford the device-wide synchronisation an
  * allocation implies or its failure under a full memory budget.  For them the per-call scratch comes from an
- * array built into the library (marlaas_lora_static_workspace_limit() bytes, 4 MiB, resident on every GPU that
+ * array built into the library (marlaas_lora_static_workspace_limit() bytes, 8 MiB, resident on every GPU that
  * loads the library until the process exits) instead of a caller workspace; x, W, y, the pool storage and h_save
- * are still the caller's.  The call allocates and frees nothing on the device.
- *  - Batches whose scratch (marlaas_lora_workspace_bytes) exceeds the limit are rejected with
+ * are still the caller's.  The call itself allocates and frees nothing on the device.
+ *  - Batches whose forward scratch (marlaas_lora_forward_workspace_bytes) exceeds the limit are rejected with
  *    MARLAAS_ERR_WORKSPACE_TOO_SMALL before anything is launched: 256 tokens on a pool of 32 slots of rank
  *    up to 64 fit.
- *  - The first call on each device looks up the array's device address; make that call before starting any
- *    stream capture on that device.
+ *  - The first call on each device looks up the array's device address.  That lookup is also the moment the CUDA
+ *    runtime loads this part of the library onto the device and the device's copy of the array comes into being
+ *    (8 MiB of device memory, taken once, which can fail if the device is full): make that first call at start-up,
+ *    while memory may still be taken, and before starting any stream capture on that device.  Later calls on the
+ *    device leave its free memory unchanged.
  *  - All calls on a device share the one array and it keeps the previous call's contents (nothing in it has to
  *    start at zero: each call writes what it later reads).  Two calls whose kernels overlap on the GPU -- different
  *    streams, or different pools on different streams -- race on it; keep such calls on one stream. */

@@ -31,11 +31,13 @@ MARLAAS_FLAG_ACCUMULATE = 1
 MARLAAS_FLAG_HOST_TABLE = 2
 MARLAAS_FLAG_VALIDATE_SYNC = 4
 MARLAAS_FLAG_CUDA_CORE_PATH = 8
+MARLAAS_FLAG_SERIAL_KERNELS = 16
 
 EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",
     "marlaas_adapter_pool_register", "marlaas_adapter_pool_unregister", "marlaas_adapter_pool_lookup",
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
+    "marlaas_lora_forward_workspace_bytes",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
     "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
@@ -92,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_adapter_pool_rank_stride.argtypes = [vp]
     L.marlaas_lora_workspace_bytes.restype = sz
     L.marlaas_lora_workspace_bytes.argtypes = [vp, i64]
+    L.marlaas_lora_forward_workspace_bytes.restype = sz
+    L.marlaas_lora_forward_workspace_bytes.argtypes = [vp, i64]
     L.marlaas_lora_forward.restype = i32
     L.marlaas_lora_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, P(marlaas_segments_t), vp, vp, sz, u32, vp]
     L.marlaas_lora_static_workspace_limit.restype = sz
@@ -256,6 +260,10 @@ def marlaas_adapter_pool_export(pool: AdapterPool, slot: int, rank: int, stream=
 
 def marlaas_lora_workspace_bytes(pool: AdapterPool, T: int) -> int:
     return int(load_library().marlaas_lora_workspace_bytes(pool.handle, T))
+
+
+def marlaas_lora_forward_workspace_bytes(pool: AdapterPool, T: int) -> int:
+    return int(load_library().marlaas_lora_forward_workspace_bytes(pool.handle, T))
 
 
 def _mat(t: torch.Tensor, cols: int, name: str):

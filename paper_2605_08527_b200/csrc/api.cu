@@ -11,20 +11,23 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 1);
     auto take = [&](size_t bytes) { char* q = p ? p + o : nullptr; o += align_up(bytes, 256); return q; };
+    // forward's fields first: a forward call needs only the first fwd_total bytes
     w.tok_slot = (int32_t*)take(sizeof(int32_t) * Tn);
-    w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
-    w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
-    w.slot_offset = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 2));
     w.h = (float*)take(sizeof(float) * Tn * pool->RP);
-    w.g = (float*)take(sizeof(float) * Tn * pool->RP);
-    w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
-    w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     const size_t ntiles = (Tn + 255) / 256;
     w.umax = (pool->cap < 256 ? pool->cap : 256) * (pool->RP / 16);
     w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
     w.hd = (bf16*)take(sizeof(bf16) * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
+    w.xbuf = (float*)take(decode_sm100_xbuf_bytes(pool, (int64_t)Tn));
+    w.fwd_total = o;
+    w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
+    w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
+    w.slot_offset = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 2));
+    w.g = (float*)take(sizeof(float) * Tn * pool->RP);
+    w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
+    w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     const size_t nblk = (Tn + 63) / 64;
     const bool grad_tc = grad_sm100_eligible(pool, (int64_t)Tn);
     w.HW = ((2 * pool->RP + 63) / 64) * 64;
@@ -138,6 +141,11 @@ size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T) {
     return carve_workspace(pool, T, nullptr).total;
 }
 
+size_t marlaas_lora_forward_workspace_bytes(const marlaas_pool_t* pool, int64_t T) {
+    if (!pool || T < 0) return 0;
+    return carve_workspace(pool, T, nullptr).fwd_total;
+}
+
 marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const marlaas_segments_t* seg,
                                           int32_t* tok_slot, int32_t* slot_count, int32_t* slot_offset,
                                           int32_t* perm, void* workspace, size_t workspace_bytes, uint32_t flags,
@@ -181,8 +189,8 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     if ((rc = check_segments(fn, pool, T, seg, flags, &host_ts)) != MARLAAS_OK) return rc;
     if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
     const Workspace ws = carve_workspace(pool, T, workspace);
-    if (workspace_bytes < ws.total)
-        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
+    if (workspace_bytes < ws.fwd_total)
+        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.fwd_total);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
 
@@ -197,7 +205,7 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         {
             TimedLaunch timed(pool, st);
             rc = launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
-                                     seg->seg_offsets, seg->seg_slot, ws, h, st);
+                                     seg->seg_offsets, seg->seg_slot, ws, h, st, (flags & MARLAAS_FLAG_SERIAL_KERNELS) != 0);
             if (rc != MARLAAS_OK) return rc;
         }
         return finish(pool, flags, st);

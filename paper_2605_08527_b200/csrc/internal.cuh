@@ -72,6 +72,7 @@ struct marlaas_pool {
     char* storage = nullptr;
     size_t storage_bytes = 0;
     int32_t* d_status = nullptr;
+    int32_t* d_sync = nullptr;      // counters and flags of the decode-shaped forward (zero between calls)
     int32_t* d_rank = nullptr;
     float* d_scale = nullptr;
     marlaas::bf16* d_At = nullptr;
@@ -90,7 +91,7 @@ struct marlaas_pool {
 namespace marlaas {
 
 struct StorageLayout {
-    size_t off_status, off_rank, off_scale, off_At, off_Bs, total;
+    size_t off_status, off_sync, off_rank, off_scale, off_At, off_Bs, total;
 };
 StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap);
 
@@ -111,6 +112,8 @@ struct Workspace {
     bf16* hd;              // [T][umax*16]  bf16(s_t h_i) (forward) or bf16(s_t g_i) (backward) in the tenant's unit
                            //               columns, zeros in the other units of the tile
     int32_t umax;
+    float* xbuf;           // decode path with four contraction slices: partial sums passed between a tile's two clusters
+    size_t fwd_total;      // bytes a forward call uses (the fields above); the rest serves backward only
     // tensor-core gradient reductions: 64-token blocks, one masked copy of the block's r-vectors per tenant present
     int32_t* blk_np;       // [nblk]        tenants present in the block
     int32_t* blk_base;     // [nblk+1]      exclusive scan of blk_np (= first copy of the block)
@@ -161,10 +164,13 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
 // decode_sm100.cu: the whole forward for batches of at most 1024 tokens (two overlapping kernels).
 // S < 0: ws.tok_slot already holds the per-token slots.
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T);
+size_t decode_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T);    // exchange scratch of the decode path (0 if unused)
+constexpr size_t DECODE_SYNC_BYTES = 8192;
 
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
                                      int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
-                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
+                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st,
+                                     bool serial = false);
 
 // shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,

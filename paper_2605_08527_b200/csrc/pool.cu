@@ -42,6 +42,7 @@ StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap) {
     StorageLayout L;
     size_t o = 0;
     L.off_status = o; o += 256;
+    L.off_sync = o;   o += DECODE_SYNC_BYTES;
     L.off_rank = o;   o += align_up(sizeof(int32_t) * (size_t)cap, 256);
     L.off_scale = o;  o += align_up(sizeof(float) * (size_t)cap, 256);
     L.off_At = o;     o += align_up(sizeof(bf16) * (size_t)cap * RP * (size_t)K, 256);
@@ -145,6 +146,7 @@ marlaas_status_t marlaas_adapter_pool_create(marlaas_pool_t** out, int device, i
     p->storage = (char*)storage;
     p->storage_bytes = storage_bytes;
     p->d_status = (int32_t*)(p->storage + L.off_status);
+    p->d_sync = (int32_t*)(p->storage + L.off_sync);
     p->d_rank = (int32_t*)(p->storage + L.off_rank);
     p->d_scale = (float*)(p->storage + L.off_scale);
     p->d_At = (bf16*)(p->storage + L.off_At);

@@ -6,22 +6,27 @@
 // cudaMalloc's implicit device synchronisation (or its failure under a tight memory budget) is not acceptable.
 // Such a caller still owns x, W, y and the adapter pool; only the scratch the layer needs between its kernels
 // (per-token slots, the low-rank intermediates, the expand operand) comes from here.
+#include <mutex>
+
 #include "internal.cuh"
 
 namespace marlaas {
 
-constexpr size_t STATIC_WS_BYTES = 4u << 20;   // 4 MiB: enough for 256 tokens on a pool of 32 slots of rank <= 64
+constexpr size_t STATIC_WS_BYTES = 8u << 20;   // 8 MiB: enough for 256 tokens on a pool of 32 slots of rank <= 64
 
 // In host code this name is only a stand-in for the device array: its device address comes from
 // cudaGetSymbolAddress, once per device, with that device current.
 static __device__ __align__(256) unsigned char g_static_ws[STATIC_WS_BYTES];
 
 static void* g_static_ws_addr[64] = {};
+static std::mutex g_static_ws_mutex;      // two host threads may make the first call on a device at the same time
 
-// Device address of the array on `device` (which must be current).  Resolved on first use per device.
+// Device address of the array on `device` (which must be current).  Resolved on first use per device: that lookup
+// makes the CUDA runtime load this module on the device, which is when the device's copy of the array comes into being.
 static marlaas_status_t static_ws_address(int device, void** out) {
     if (device < 0 || device >= 64)
         return fail(MARLAAS_ERR_INVALID_ARG, "lora_forward_static_ws: device index %d is outside [0,64)", device);
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
     if (!g_static_ws_addr[device]) {
         void* p = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&p, g_static_ws);
@@ -49,7 +54,7 @@ marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T,
     if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
     if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
     if (T == 0) return MARLAAS_OK;
-    const size_t need = marlaas_lora_workspace_bytes(pool, T);
+    const size_t need = marlaas_lora_forward_workspace_bytes(pool, T);     // forward's share of the workspace only
     if (need == 0 || need > STATIC_WS_BYTES)
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL,
                     "%s: a batch of %lld tokens on this pool needs %zu bytes of scratch, the built-in array holds %zu; "

@@ -10,3 +10,4 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a); run with -m gpu on a B200")
+    config.addinivalue_line("markers", "slow: takes about a minute of host time (the oracle over a full-size output)")

@@ -1,7 +1,9 @@
 """GPU parity at the full configured sizes, through the same calls bench.py times (forward with h_save, backward with
-the saved h).  The oracle is too slow for every output row at these sizes, so y and dx are checked on sampled token
-rows (each row of the oracle is computed on its own, from the definition), while the adapter gradients, which sum
-over every token of a tenant, are checked in full.  Index outputs are compared bit for bit.
+the saved h).  y and dx are checked, over all columns, on at least one token row of every 128-row block (the rows one
+CTA of a 256-row tile owns, so every CTA of every tile of the launch has a checked row) plus the tile-edge rows; each
+oracle row is computed on its own, from the definition.  The adapter gradients, which sum over every token of a
+tenant, are checked in full, and one slow test checks every row of y at the largest size.  Index outputs are compared
+bit for bit.
 """
 import numpy as np
 import pytest
@@ -17,9 +19,14 @@ pytestmark = pytest.mark.gpu
 
 
 def _sample_rows(T, n, seed):
+    """Edge rows, one seeded row inside every 128-row block, and n more seeded rows anywhere."""
     edge = [0, 1, 63, 64, 127, 128, 255, 256, 257, T // 2, T - 257, T - 256, T - 129, T - 128, T - 2, T - 1]
+    nblk = (T + 127) // 128
+    off = (wl.hash_u64(seed, wl.TID_PERTURB, np.arange(nblk, dtype=np.uint64) + np.uint64(1 << 20)) % np.uint64(128)).astype(np.int64)
+    per_block = np.minimum(np.arange(nblk, dtype=np.int64) * 128 + off, T - 1)
     rnd = (wl.hash_u64(seed, wl.TID_PERTURB, np.arange(n, dtype=np.uint64)) % np.uint64(T)).astype(np.int64)
-    rows = sorted({int(r) for r in edge if 0 <= r < T} | {int(r) for r in rnd})
+    rows = sorted({int(r) for r in edge if 0 <= r < T} | {int(r) for r in per_block} | {int(r) for r in rnd})
+    assert len({r // 128 for r in rows}) == nblk
     return np.array(rows, dtype=np.int64)
 
 
@@ -57,6 +64,22 @@ def _check_full(w, p, n_rows=40):
 def test_cfg3_training_shaped_full_size():
     w = wl.make_workload(3)
     _check_full(w, w.projections[0])
+
+
+@pytest.mark.slow
+def test_cfg3_every_row_of_y():
+    """All 16384 x 11008 outputs of the largest forward against the oracle (about a minute of host time)."""
+    w = wl.make_workload(3)
+    p = w.projections[0]
+    ts = w.tok_slot()
+    r, s, A, Bm = oracle.adapters_of(p)
+    dc = DeviceCase(w, p)
+    y = to_np(dc.forward())
+    B.marlaas_check_status(dc.pool)
+    step = 2048
+    for r0 in range(0, w.T, step):
+        ry, _ = oracle.forward(p.x[r0:r0 + step], p.W, r, s, A, Bm, ts[r0:r0 + step])
+        assert_close(y[r0:r0 + step], ry, f"{w.name}/{p.name} y rows {r0}..{r0 + step - 1}")
 
 
 def test_cfg4_heterogeneous_full_size():
