@@ -62,10 +62,7 @@ enum {
     MARLAAS_FLAG_HOST_TABLE = 2u,     /* seg_offsets / seg_slot are HOST arrays: validated on the host, then copied
                                          into the workspace in stream order */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
-    MARLAAS_FLAG_CUDA_CORE_PATH = 8u, /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
-    MARLAAS_FLAG_SERIAL_KERNELS = 16u /* diagnostics: the decode-shaped forward normally runs its two kernels side by
-                                         side, the second feeding the first; tools that run one kernel at a time
-                                         (profilers, CUDA_LAUNCH_BLOCKING=1) need this flag, which orders them plainly */
+    MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
 };
 
 /* Token-to-adapter segment table of one mixed batch: segment s covers tokens

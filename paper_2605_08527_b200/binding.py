@@ -31,7 +31,6 @@ MARLAAS_FLAG_ACCUMULATE = 1
 MARLAAS_FLAG_HOST_TABLE = 2
 MARLAAS_FLAG_VALIDATE_SYNC = 4
 MARLAAS_FLAG_CUDA_CORE_PATH = 8
-MARLAAS_FLAG_SERIAL_KERNELS = 16
 
 EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",

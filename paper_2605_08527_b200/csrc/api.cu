@@ -20,7 +20,7 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
     w.hd = (bf16*)take(sizeof(bf16) * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
-    w.xbuf = (float*)take(decode_sm100_xbuf_bytes(pool, (int64_t)Tn));
+    w.xbuf = (float*)take(decode_wide_sm100_xbuf_bytes(pool, (int64_t)Tn));
     w.fwd_total = o;
     w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
     w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
@@ -204,8 +204,11 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         }
         {
             TimedLaunch timed(pool, st);
-            rc = launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
-                                     seg->seg_offsets, seg->seg_slot, ws, h, st, (flags & MARLAAS_FLAG_SERIAL_KERNELS) != 0);
+            rc = decode_wide_sm100_eligible(pool, T)
+                     ? launch_decode_wide_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
+                                                seg->seg_offsets, seg->seg_slot, ws, h, st)
+                     : launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
+                                           seg->seg_offsets, seg->seg_slot, ws, h, st);
             if (rc != MARLAAS_OK) return rc;
         }
         return finish(pool, flags, st);

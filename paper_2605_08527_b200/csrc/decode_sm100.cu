@@ -1,63 +1,297 @@
 // Decode-shaped forward (up to four 256-token tiles, typically one token per sequence, tenants unsorted): the call is
-// bound by the one pass over W from HBM, so the work is cut to keep the memory system busy from the first microsecond
-// to the last and the launch count to two kernels that run side by side on disjoint SMs.
+// bound by the one pass over W from HBM (or, from about 300 tokens, by the tensor cores on a grid of few tiles), so the
+// work is cut to keep every SM busy and the launch count to two overlapping kernels.
 //
-//   k_decode_gemm    (tcgen05, TMA)  y^T = [W ; Bs]^T * [x | hd]^T: the base product and the expand as ONE contraction
-//                    over K + cap*RP, with the operand roles swapped against the training GEMM: 256 columns of W are the
-//                    M side of a cta_group::2 MMA (128 per CTA, read as an MN-major A operand straight from the row-major
-//                    weight), the 256 tokens its N side (128 per CTA).  A 64-deep step therefore brings as many bytes of
-//                    W as of x into a CTA (16 KB each), half the activation re-reads of a token-major tile.  A tile's
-//                    contraction is cut into S slices (1, 2 or 4 CTA pairs); the partial accumulators are summed in a
-//                    fixed tree: the two pairs of a 4-CTA cluster exchange token halves through distributed shared
-//                    memory, the two clusters of a tile exchange token quarters through an L2-resident scratch buffer.
-//   k_decode_shrink  (mma.sync, bulk copies)  per tenant and 16-token pass: h_i = x_i A_t from the pooled store.  Runs on
-//                    the SMs the GEMM's clusters leave free (its CTAs take work units from a counter, so any number of
-//                    resident CTAs is correct), writes tok_slot, fp32 h and the dense expand operand
-//                    hd[i][t*RP + j] = bf16(s_t h_i[j]) (zeros in every other tenant's columns), and counts finished units;
-//                    the GEMM's expand steps wait for that count.
-//
-// Launch order: the GEMM first (it triggers its dependents at once), the shrink second as its programmatic dependent.
-// The shrink grid ends with a wait for the GEMM grid and then clears the counters and flags, so a kernel ordered after
-// the pair sees both complete, and a replay of a captured call finds the counters at zero.
+//   k_decode_shrink  (CUDA cores + warp-level MMA)  per tenant: h_i = x_i A_t for the tenant's tokens, gathered from
+//                    the pooled store; a cluster of CTAs splits K and sums its partial products through distributed
+//                    shared memory in a fixed order.  Writes tok_slot, h (fp32) and the dense expand operand
+//                    hd[i][t*RP + j] = bf16(s_t h_i[j]) (zeros in every other tenant's columns).
+//   k_decode_gemm    (tcgen05, TMA)  y = bf16( [x | hd] * [W ; Bs] ): the base product and the expand as one
+//                    contraction over K + cap*RP.  A cluster owns one strip of output columns; its S CTA pairs
+//                    (cta_group::2, 256 rows) each take a slice of the contraction and the partial accumulators are
+//                    summed through distributed shared memory, again in a fixed order.  Launched as a programmatic
+//                    dependent of the shrink: it streams W while the shrink runs and waits for hd only before the
+//                    expand k-blocks.
 #include "sm100_ptx.cuh"
 #include "sm100_cluster.cuh"
-
-#include <algorithm>
 
 namespace marlaas {
 namespace sm100 {
 
-// words of the pool's synchronisation area
-constexpr int SY_TICKET = 0;        // next shrink work unit
-constexpr int SY_DONE = 1;          // finished shrink work units
-constexpr int SY_EXIT = 2;          // shrink CTAs that have reached their end
-constexpr int SY_FLAGS = 16;        // split-K exchange flags, one per (tile, destination cluster, CTA, epilogue warp)
+// ---------------------------------------------------------------------------------------------------------------
+// k_decode_shrink
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int DS_THREADS = 128;
+constexpr int DS_MAX_T = 1024;         // tokens per call
+constexpr int DS_ROUNDS = DS_MAX_T / DS_THREADS;
+constexpr int DS_PASS = 16;            // tokens per pass (one m16 MMA tile)
+constexpr int DS_MAX_CS = 8;
+constexpr int DS_TABLE_SMEM = 1032;    // the segment table is staged in shared memory when S + 1 <= this
+constexpr int DS_UB = 4;               // 32-deep k-blocks whose loads are in flight together per warp
 
-__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+struct DecodeShrinkArgs {
+    int T, K, RP, cap;
+    int S;                              // segments; < 0: tok_slot already holds the per-token slots
+    int G;                              // clusters per tenant: cluster (t, i) takes the 16-token passes i, i + G, ...
+    const int32_t* seg_offsets;
+    const int32_t* seg_slot;
+    const bf16* x;
+    int64_t ldx;
+    const bf16* At;                     // [cap*RP][K]
+    const int32_t* d_rank;
+    const float* d_scale;
+    int32_t* tok_slot;                  // [T]
+    float* h_out;                       // [T][RP]
+    bf16* hd;                           // [T][hd_cols]
+    int hd_cols;
+    int32_t* status;
+};
+
+// Shared memory: the fixed part below, then (dynamic, sized by the launch) slot[T'], off_tab[max(S + 1, T')] whose
+// space the cluster's token list takes over once every token has its slot, and slot_tab[S]; T' = T rounded up to 32.
+// Keeping this small matters: two of these CTAs share an SM with a GEMM CTA, whose pipeline gets what is left.
+struct __align__(16) DecodeShrinkSmem {
+    float wpart[4][256];                // per-warp [16 tokens][16 ranks] partial products
+    float part[DS_MAX_CS][256];         // per-CTA partials, gathered in cluster rank 0
+    int32_t cnt[DS_ROUNDS * 4];
+};
+static size_t decode_shrink_dyn_smem(int64_t T, int32_t S) {
+    const size_t Tp = (size_t)((T + 31) / 32 * 32);
+    const bool staged = S >= 0 && S + 1 <= DS_TABLE_SMEM;
+    return 4 * (Tp + std::max<size_t>(staged ? (size_t)S + 1 : 0, Tp) + (staged ? (size_t)S : 0));
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
     return v;
 }
-__device__ __forceinline__ void st_release_gpu(int32_t* p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Bounded wait for a global word to reach `target` (acquire); gives up like mbar_wait.
-__device__ __forceinline__ bool wait_word_ge(const int32_t* p, int target, volatile int* abort_word, int site) {
-    if (ld_acquire_gpu(p) >= target) return true;
-    unsigned long long t0 = 0;
-    uint32_t spins = 0;
-    while (true) {
-        if (ld_acquire_gpu(p) >= target) return true;
-        __nanosleep(40);
-        if (((++spins) & 63u) == 0) {
-            if (*abort_word != 0) return false;
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
-                atomicCAS((int*)abort_word, 0, site);
-                return false;
+// grid = (cap + 1) clusters of CS CTAs; cluster t < cap serves tenant slot t, cluster cap the tokens routed to no
+// adapter (slot -1, or a slot outside the pool, which is reported).  The cluster's CTAs (and their warps) split K.
+//
+// Operand fragments of the m16n8k16 MMA come straight from global memory with 16-byte loads: within a 32-deep
+// k-block lane (g, t) reads elements 8t .. 8t+7 of its rows, and the same element-to-position permutation is used
+// for the token rows (A fragment) and the adapter rows (B fragment), so every product pairs matching k.
+__global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShrinkArgs g) {
+    __shared__ DecodeShrinkSmem sm;
+    extern __shared__ int32_t ds_dyn[];
+    const int Tp = (g.T + 31) / 32 * 32;
+    const bool staged_tab = g.S >= 0 && g.S + 1 <= DS_TABLE_SMEM;
+    int32_t* const s_slot = ds_dyn;
+    int32_t* const s_off = ds_dyn + Tp;             // the segment offsets, later the token list
+    int32_t* const s_list = s_off;
+    int32_t* const s_stab = s_off + max(staged_tab ? g.S + 1 : 0, Tp);
+    dk_launch_dependents();      // the GEMM may start streaming W now; it waits for this grid before the expand
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int crank = (int)dk_cluster_ctarank();
+    int cs;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(cs));
+    const int t = (int)dk_cluster_id_x() / g.G;     // tenant slot served by this cluster; == cap: no adapter
+    const int gi = (int)dk_cluster_id_x() % g.G;    // which of the tenant's 16-token passes
+    const bool first = (dk_cluster_id_x() == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
+    const int r_t = t < g.cap ? g.d_rank[t] : 0;
+    const float sc = t < g.cap ? g.d_scale[t] : 0.f;
+
+    // This warp's share of K: the cluster's CTAs split the 32-deep k-blocks, then each CTA's warps do.  The adapter rows
+    // of the tenant's first rank group do not depend on the token list, and a load issued beside the GEMM's stream takes
+    // microseconds to come back: they are requested before anything else.
+    const int nb32 = (g.K + 31) >> 5;
+    const int cb0 = crank * nb32 / cs, cb1 = (crank + 1) * nb32 / cs;        // (32-bit: 64-bit division is slow, and these
+    const int wb0 = cb0 + warp * (cb1 - cb0) / 4, wb1 = cb0 + (warp + 1) * (cb1 - cb0) / 4;   // precede the first loads)
+    const int gq = lane >> 2, tq = lane & 3;
+    uint4 ba[DS_UB], bb[DS_UB];     // adapter fragments; held_jg / held_b0 say of which rank group and k-block batch
+    int held_jg = 0, held_b0 = wb0;
+    {
+        const bf16* ar0 = g.At + ((size_t)(t < g.cap ? t : 0) * g.RP + gq) * g.K;
+        const bf16* ar1 = ar0 + (size_t)8 * g.K;
+#pragma unroll
+        for (int u = 0; u < DS_UB; ++u) {
+            const int k = (wb0 + u) * 32 + tq * 8;
+            const bool in = t < g.cap && (wb0 + u) < wb1 && k < g.K;
+            ba[u] = in ? ldg_nc_v4(ar0 + k) : make_uint4(0u, 0u, 0u, 0u);
+            bb[u] = in ? ldg_nc_v4(ar1 + k) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+
+    // ---- per-token slot ------------------------------------------------------------------------------------
+    if (g.S >= 0) {
+        const bool staged = staged_tab;
+        if (staged) {
+            for (int s = tid; s <= g.S; s += DS_THREADS) {
+                s_off[s] = g.seg_offsets[s];
+                if (s < g.S) s_stab[s] = g.seg_slot[s];
+            }
+            __syncthreads();
+        }
+        if (first) {
+            for (int s = tid; s < g.S; s += DS_THREADS) {
+                const int a = staged ? s_off[s] : g.seg_offsets[s], b = staged ? s_off[s + 1] : g.seg_offsets[s + 1];
+                if (b < a || a < 0 || b > g.T) dk_report(g.status, DEV_BAD_TABLE, s);
+                if (s == 0 && a != 0) dk_report(g.status, DEV_BAD_TABLE, -1);
+                if (s == g.S - 1 && b != g.T) dk_report(g.status, DEV_BAD_TABLE, -2);
+            }
+            if (tid == 0 && g.S == 0 && g.T != 0) dk_report(g.status, DEV_BAD_TABLE, -3);
+        }
+        for (int i = tid; i < g.T; i += DS_THREADS) {
+            int lo = 0, hi = g.S;
+            while (lo < hi) {       // first s with seg_offsets[s + 1] > i
+                const int mid = (lo + hi) >> 1;
+                const int v = staged ? s_off[mid + 1] : g.seg_offsets[mid + 1];
+                if (v > i) hi = mid; else lo = mid + 1;
+            }
+            s_slot[i] = lo < g.S ? (staged ? s_stab[lo] : g.seg_slot[lo]) : -1;
+        }
+    } else {
+        for (int i = tid; i < g.T; i += DS_THREADS) s_slot[i] = g.tok_slot[i];
+    }
+    __syncthreads();
+    if (first)
+        for (int i = tid; i < g.T; i += DS_THREADS) {
+            int s = s_slot[i];
+            if (s < -1 || s >= g.cap) {
+                dk_report(g.status, DEV_BAD_INDEX, i);
+                s = -1;
+            }
+            g.tok_slot[i] = s;
+        }
+
+    // ---- this cluster's tokens, ascending --------------------------------------------------------------------
+    unsigned bal[DS_ROUNDS];
+    bool mine[DS_ROUNDS];
+#pragma unroll
+    for (int r = 0; r < DS_ROUNDS; ++r) {
+        const int i = r * DS_THREADS + tid;
+        bool m = false;
+        if (i < g.T) {
+            const int s = s_slot[i];
+            m = (t < g.cap) ? (s == t) : (s < 0 || s >= g.cap);
+        }
+        mine[r] = m;
+        bal[r] = __ballot_sync(0xffffffffu, m);
+        if (lane == 0) sm.cnt[r * 4 + warp] = __popc(bal[r]);
+    }
+    __syncthreads();
+    int n_t = 0;
+#pragma unroll
+    for (int e = 0; e < DS_ROUNDS * 4; ++e) n_t += sm.cnt[e];
+#pragma unroll
+    for (int r = 0; r < DS_ROUNDS; ++r) {
+        if (mine[r]) {
+            int off = __popc(bal[r] & ((1u << lane) - 1u));
+            for (int e = 0; e < r * 4 + warp; ++e) off += sm.cnt[e];
+            s_list[off] = r * DS_THREADS + tid;
+        }
+    }
+    __syncthreads();
+    if (gi * DS_PASS >= n_t) return;     // nothing for this cluster (uniform over it)
+
+    const int own0 = r_t > 0 ? t * g.RP : 0, own1 = r_t > 0 ? own0 + g.RP : 0;   // hd columns written by the MMA part
+    const int ngroups = (r_t + 15) >> 4;
+
+    // ---- partial products over this warp's share of K --------------------------------------------------------
+    const uint32_t part_rank0 = dk_map_to_cta(smem_u32(&sm.part[0][0]), 0);
+
+    // zero the other tenants' columns of this cluster's hd rows (and, with no adapter, the h rows): one warp per row
+    for (int e = crank * 4 + warp; e < n_t; e += cs * 4) {
+        if ((e / DS_PASS) % g.G != gi) continue;     // another cluster's pass
+        const int tok = s_list[e];
+        bf16* row = g.hd + (size_t)tok * g.hd_cols;
+        for (int c = lane * 8; c < g.hd_cols; c += 256)
+            if (c < own0 || c >= own1) *reinterpret_cast<uint4*>(row + c) = make_uint4(0u, 0u, 0u, 0u);
+        if (r_t == 0)
+            for (int j = lane; j < g.RP; j += 32) g.h_out[(size_t)tok * g.RP + j] = 0.f;
+    }
+    if (r_t == 0) return;        // uniform over the cluster
+
+    for (int p0 = gi * DS_PASS; p0 < n_t; p0 += DS_PASS * g.G) {
+        const int np = min(DS_PASS, n_t - p0);
+        const bf16* xr0 = gq < np ? g.x + (size_t)s_list[p0 + gq] * g.ldx : nullptr;
+        const bf16* xr1 = gq + 8 < np ? g.x + (size_t)s_list[p0 + gq + 8] * g.ldx : nullptr;
+        for (int jg = 0; jg < ngroups; ++jg) {
+            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+            const bf16* ar0 = g.At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
+            const bf16* ar1 = ar0 + (size_t)8 * g.K;
+            for (int b0 = wb0; b0 < wb1; b0 += DS_UB) {
+                uint4 xa[DS_UB], xb[DS_UB];
+                const bool held = held_jg == jg && held_b0 == b0;     // the adapter fragments are in registers already
+#pragma unroll
+                for (int u = 0; u < DS_UB; ++u) {
+                    const int k = (b0 + u) * 32 + tq * 8;
+                    const bool in = (b0 + u) < wb1 && k < g.K;
+                    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                    xa[u] = (in && xr0) ? ldg_nc_v4(xr0 + k) : z;
+                    xb[u] = (in && xr1) ? ldg_nc_v4(xr1 + k) : z;
+                    if (!held) {
+                        ba[u] = in ? ldg_nc_v4(ar0 + k) : z;
+                        bb[u] = in ? ldg_nc_v4(ar1 + k) : z;
+                    }
+                }
+                held_jg = jg;
+                held_b0 = b0;
+#pragma unroll
+                for (int u = 0; u < DS_UB; ++u) {
+                    mma_bf16_16816(c0, xa[u].x, xb[u].x, xa[u].y, xb[u].y, ba[u].x, ba[u].y);
+                    mma_bf16_16816(c1, xa[u].x, xb[u].x, xa[u].y, xb[u].y, bb[u].x, bb[u].y);
+                    mma_bf16_16816(c0, xa[u].z, xb[u].z, xa[u].w, xb[u].w, ba[u].z, ba[u].w);
+                    mma_bf16_16816(c1, xa[u].z, xb[u].z, xa[u].w, xb[u].w, bb[u].z, bb[u].w);
+                }
+            }
+            // warp partials -> CTA partial (fixed order) -> cluster rank 0
+            const bool first_round = p0 == gi * DS_PASS && jg == 0;
+            const bool last_round = p0 + DS_PASS * g.G >= n_t && jg == ngroups - 1;
+            if (!first_round) __syncthreads();      // wpart of the previous group has been consumed
+            {
+                float* wp = sm.wpart[warp];
+                wp[gq * 16 + 2 * tq] = c0[0];
+                wp[gq * 16 + 2 * tq + 1] = c0[1];
+                wp[(gq + 8) * 16 + 2 * tq] = c0[2];
+                wp[(gq + 8) * 16 + 2 * tq + 1] = c0[3];
+                wp[gq * 16 + 8 + 2 * tq] = c1[0];
+                wp[gq * 16 + 8 + 2 * tq + 1] = c1[1];
+                wp[(gq + 8) * 16 + 8 + 2 * tq] = c1[2];
+                wp[(gq + 8) * 16 + 8 + 2 * tq + 1] = c1[3];
+            }
+            __syncthreads();
+            for (int e = tid; e < 256; e += DS_THREADS) {
+                const float v = ((sm.wpart[0][e] + sm.wpart[1][e]) + sm.wpart[2][e]) + sm.wpart[3][e];
+                dk_st_cluster_f32(part_rank0 + (uint32_t)(crank * 256 + e) * 4, v);
+            }
+            dk_cluster_sync();
+            if (crank == 0) {
+                for (int e = tid; e < 256; e += DS_THREADS) {
+                    const int i = e >> 4, j = e & 15;
+                    if (i < np) {
+                        float v = 0.f;
+                        for (int s = 0; s < cs; ++s) v += sm.part[s][e];   // fixed order
+                        const int tok = s_list[p0 + i];
+                        g.h_out[(size_t)tok * g.RP + jg * 16 + j] = v;
+                        g.hd[(size_t)tok * g.hd_cols + own0 + jg * 16 + j] = __float2bfloat16_rn(sc * v);
+                    }
+                }
+            }
+            if (!last_round) dk_cluster_sync();     // rank 0 has read the partials before they are overwritten (its own
+                                                    // shared memory: after the last round the other CTAs may leave)
+        }
+        // ranks beyond the tenant's true rank (rounded up to 16) stay zero
+        if (crank == 0) {
+            const int rest = g.RP - ngroups * 16;
+            for (int e = tid; e < np * rest; e += DS_THREADS) {
+                const int i = e / rest, j = ngroups * 16 + e % rest;
+                const int tok = s_list[p0 + i];
+                g.h_out[(size_t)tok * g.RP + j] = 0.f;
+                g.hd[(size_t)tok * g.hd_cols + own0 + j] = __float2bfloat16_rn(0.f);
             }
         }
     }
@@ -66,74 +300,52 @@ __device__ __forceinline__ bool wait_word_ge(const int32_t* p, int target, volat
 // ---------------------------------------------------------------------------------------------------------------
 // k_decode_gemm
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int DG_THREADS = 320;        // warp 0: TMA producer, warp 1: MMA issuer + tensor memory, warps 2..9: epilogue
-constexpr int DG_TN = 256;             // tokens per tile = N of the MMA
-constexpr int DG_TM = 256;             // W columns per tile = M of the MMA (128 per CTA)
-constexpr uint32_t DG_MBOX_BYTES = 64 * 1024;   // one token half of a CTA's accumulator: 128 lanes x 128 columns fp32
+constexpr int DG_THREADS = 192;
+constexpr int DG_KP = 2;               // 64-deep panels per pipeline step
 
 struct DecodeGemmArgs {
     int T, Nout;
-    int nstrips;         // 256-column strips of W; tile = (token tile, strip)
-    int num_ks;          // 64-deep pipeline steps over K
-    int num_xs;          // 64-deep pipeline steps over the expand rows (up to the last slot in use)
-    int S;               // contraction slices per tile: 1 (clusters of one CTA pair), 2 or 4 (clusters of two pairs)
+    int nstrips;         // column strips; cluster c works on strip c mod nstrips of 256-row tile c / nstrips
+    int num_ks;          // pipeline steps (kp * 64 deep) over K
+    int num_xs;          // pipeline steps over the expand rows (cap*RP, or up to the last slot in use)
+    int S;               // contraction slices = CTA pairs per cluster
+    int nch;             // 64-column chunks of the B operand staged per CTA: the pair's strip is 128 * nch columns
+    int kp;              // 64-deep panels per pipeline step: one TMA instruction per operand moves all of them
     int stages;
-    int w3d;             // the W-side operand moves with one 3-D copy per step (N a multiple of 64), else one per chunk
-    int n_units;         // shrink work units that must be finished before hd is read
-    int n_flags;         // exchange flags in use (S = 4)
-    int reset_at_end;    // serial order (shrink grid first): this grid ends last and clears the counters and flags
     bf16* C;
     int64_t ldc;
     int32_t* status;
-    int32_t* sync;
-    float* xbuf;         // S = 4: exchange buffer between the two clusters of a tile
 };
 
-__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t bar_cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
-}
-__device__ __forceinline__ uint4 ld_cg_v4(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-    return v;
-}
-
-// Operand staging per 64-deep pipeline step and CTA:
-//   Wt [2 chunks][64 k][64 n]   the CTA's 128 columns of W (or of the adapter rows Bs): MN-major A operand, 128-byte
-//                               swizzle, chunks 8 KB apart
-//   Xt [128 tokens][64 k]       the CTA's half of the token tile of x (or of hd): K-major B operand
+// Operand staging per pipeline step (kp panels of 64 k):
+//   A  [kp][128 rows][64 k]      one 3-D TMA over x viewed as (64 k, rows, K / 64): K-major tiles, 128-byte swizzle
+//   B  [nch][kp * 64 k][64 n]    one 2-D TMA per 64-column chunk: MN-major, chunks kp * 8 KB apart
+// A single thread issues the loads and a single thread the MMAs, and each of their instructions costs tens to a
+// hundred cycles of issue latency, so the steps are made deep: with 64-deep steps the issue loop, not HBM, set the pace.
 __global__ void __launch_bounds__(DG_THREADS, 1)
-k_decode_gemm(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-              const __grid_constant__ CUtensorMap tmXW, const __grid_constant__ CUtensorMap tmXX, const DecodeGemmArgs g) {
+k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const __grid_constant__ CUtensorMap tmXA, const __grid_constant__ CUtensorMap tmXB, const DecodeGemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int STAGES = g.stages;
-    constexpr uint32_t W_BYTES = 2 * CHUNK_BYTES, X_BYTES = A_STAGE_BYTES, STAGE_BYTES = W_BYTES + X_BYTES;
-    const uint32_t sStage = smem_u32(smem);
-    const uint32_t mbox_off = (uint32_t)STAGES * STAGE_BYTES;
-    const uint32_t sMbox = sStage + mbox_off;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + mbox_off + (g.S > 1 ? DG_MBOX_BYTES : 0u));
+    const uint32_t a_stage_bytes = (uint32_t)g.kp * A_STAGE_BYTES;
+    const uint32_t b_chunk_bytes = (uint32_t)g.kp * CHUNK_BYTES;
+    const uint32_t b_stage_bytes = (uint32_t)g.nch * b_chunk_bytes;
+    const uint32_t sA = smem_u32(smem);
+    const uint32_t sB = sA + STAGES * a_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (a_stage_bytes + b_stage_bytes));
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * STAGES;
     const uint32_t bar_drain = bar_tfull + 8;
-    const uint32_t bar_mbox = bar_drain + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 3);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr uint32_t TMEM_COLS = DG_TN;
+    const int NP = 128 * g.nch;                 // columns of the cluster's strip
+    const uint32_t tmem_cols = (uint32_t)NP;    // 128 or 256
+    // set-up first (one thread the barriers, one the descriptor prefetches, one warp the tensor-memory allocation): the
+    // index arithmetic below holds a dozen integer divisions, a microsecond if it came before
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -141,90 +353,100 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         }
         mbar_init(bar_tfull, 1);
         mbar_init(bar_drain, 1);
-        mbar_init(bar_mbox, DG_THREADS - 64);       // every epilogue thread of the partner CTA arrives once
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (threadIdx.x == 64) {
-        prefetch_tmap(&tmW);
-        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
         if (g.num_xs > 0) {
-            prefetch_tmap(&tmXW);
-            prefetch_tmap(&tmXX);
+            prefetch_tmap(&tmXA);
+            prefetch_tmap(&tmXB);
         }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(TMEM_COLS)
+                     "r"(tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     const uint32_t crank = dk_cluster_ctarank();
-    const uint32_t half = crank & 1;            // which 128 W columns and which 128 tokens this CTA stages
-    const uint32_t pi = crank >> 1;             // pair within the cluster
+    const uint32_t half = crank & 1;            // which 128 rows of the 256-row tile
+    const uint32_t pairi = crank >> 1;          // which slice of the contraction
     const uint32_t leader = crank & ~1u;
-    const int C2 = g.S > 2 ? 2 : 1;             // clusters per tile
-    const int cid = (int)dk_cluster_id_x();
-    const int tile = cid / C2, cs = cid % C2;
-    const int sl = cs * 2 + (int)pi;            // contraction slice of this pair
-    const int n0 = (tile % g.nstrips) * DG_TM;
-    const int m0 = (tile / g.nstrips) * DG_TN;
-    const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
-    const int ks0 = sl * g.num_ks / g.S, ks1 = (sl + 1) * g.num_ks / g.S;
-    const int xs0 = sl * g.num_xs / g.S, xs1 = (sl + 1) * g.num_xs / g.S;
-    const int nbase = ks1 - ks0, nstep = nbase + (xs1 - xs0);
+    const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
+    const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
+    const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
 
-    // Everything above touches no global memory; from here on the kernels ordered before this one are complete.  The
-    // shrink grid (this grid's dependent) may start as soon as every CTA has passed this point.
-    dk_wait_prerequisites();
-    dk_launch_dependents();
+    const int ks0 = (int)pairi * g.num_ks / g.S, ks1 = ((int)pairi + 1) * g.num_ks / g.S;
+    const int xs0 = (int)pairi * g.num_xs / g.S, xs1 = ((int)pairi + 1) * g.num_xs / g.S;
 
+    const int qper = 4 / g.S;
+    // bit p set: slice p has at least one step (computed once: integer division is slow in these short loops)
+    uint32_t live = 0;
+    for (int p = 0; p < g.S; ++p) {
+        const int n = ((p + 1) * g.num_ks / g.S - p * g.num_ks / g.S) + ((p + 1) * g.num_xs / g.S - p * g.num_xs / g.S);
+        if (n > 0) live |= 1u << p;
+    }
+    const uint32_t box_bytes = (uint32_t)NP * 4u * 32u;      // one quarter from one pair
     tc_fence_before();
     dk_cluster_sync();      // every CTA's barriers exist before any remote arrive or TMA completion
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // bytes the two CTAs of the pair stage per step (boxes wholly outside the tensors are skipped; partly outside boxes
-    // are filled with zeros and count in full)
-    auto x_tx = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? X_BYTES : 0u; };
-    auto w_chunks = [&](int r) -> int { return max(0, min(2, (g.Nout - (n0 + r * 128) + 63) / 64)); };
-    auto w_tx = [&](int r) -> uint32_t { const int c = w_chunks(r); return (g.w3d ? (c > 0 ? 2u : 0u) : (uint32_t)c) * CHUNK_BYTES; };
-    const uint32_t stage_tx = x_tx(0) + x_tx(1) + w_tx(0) + w_tx(1);
-    const int my_chunks = w_chunks((int)half);
-    const bool have_rows = my_tok < g.T;
+    // bytes the two CTAs of the pair stage per step (rows and columns outside the tensors are skipped entirely;
+    // partly outside boxes are filled with zeros and count in full)
+    auto a_bytes = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? a_stage_bytes : 0u; };
+    auto b_chunks = [&](int r) -> int { return max(0, min(g.nch, (g.Nout - (n0 + r * 64 * g.nch) + 63) / 64)); };
+    const uint32_t stage_tx = a_bytes(0) + a_bytes(1) + (uint32_t)(b_chunks(0) + b_chunks(1)) * b_chunk_bytes;
+    const int my_chunks = b_chunks((int)half);
+    const bool have_rows = my_m < g.T;
 
     bool epi_ok = true;
     if (warp == 0) {
         // ================= TMA producer (every CTA) =================
         if (lane == 0) {
-            uint32_t it = 0, s = 0, ph = 0;
-            bool ok = true, hd_ready = false;
+            uint32_t it = 0, s = 0, ph = 0;     // steps issued; stage and phase bit of the next step
+            bool ok = true;
             const uint32_t full0 = dk_map_to_cta(bar_full, leader);
-            for (int b = 0; b < nstep && ok; ++b, ++it) {
-                const bool ex = b >= nbase;
-                const int step = ex ? xs0 + (b - nbase) : ks0 + b;
-                const CUtensorMap* mw = ex ? &tmXW : &tmW;
-                const CUtensorMap* mx = ex ? &tmXX : &tmX;
+            for (int ks = ks0; ks < ks1 && ok; ++ks, ++it) {
                 if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 41))) break;
                 if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
-                const uint32_t dw = sStage + s * STAGE_BYTES, dx = dw + W_BYTES;
-                if (g.w3d) {
-                    if (my_chunks > 0) dg_tma_pair_3d(dw, mw, full0 + 8 * s, 0, step * BK, my_n >> 6);
-                } else {
-                    for (int c = 0; c < my_chunks; ++c) dg_tma_pair(dw + c * CHUNK_BYTES, mw, full0 + 8 * s, my_n + c * 64, step * BK);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmA, full0 + 8 * s, 0, my_m, ks * g.kp);
+                for (int c = 0; c < my_chunks; ++c)
+                    dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmB, full0 + 8 * s, my_n + c * 64, ks * g.kp * BK);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+            }
+            // the expand's adapter rows Bs do not depend on the shrink grid: the first steps' B operands are fetched
+            // before the wait for it, their hd tiles after
+            const int npre = (xs1 - xs0) < STAGES ? (xs1 - xs0) : STAGES;
+            {
+                uint32_t b_s = s, b_ph = ph;
+                for (int i = 0; i < npre && ok; ++i) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * b_s, b_ph ^ 1, abort_word, 42))) break;
+                    if (half == 0) mbar_expect_tx(bar_full + 8 * b_s, stage_tx);
+                    for (int c = 0; c < my_chunks; ++c)
+                        dg_tma_pair(sB + b_s * b_stage_bytes + c * b_chunk_bytes, &tmXB, full0 + 8 * b_s, my_n + c * 64,
+                                    (xs0 + i) * g.kp * BK);
+                    if (++b_s == (uint32_t)STAGES) { b_s = 0; b_ph ^= 1; }
                 }
-                if (ex && !hd_ready) {
-                    // the adapter rows above do not depend on the shrink grid; hd does
-                    if (!(ok = wait_word_ge(g.sync + SY_DONE, g.n_units, abort_word, 43))) break;
-                    fence_proxy_async_all();
-                    hd_ready = true;
-                }
-                if (have_rows) dg_tma_pair_3d(dx, mx, full0 + 8 * s, 0, my_tok, step);
+            }
+            if (ok && xs0 < xs1) dk_wait_prerequisites();     // hd comes from the shrink grid
+            for (int i = 0; i < npre && ok; ++i, ++it) {
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, (xs0 + i) * g.kp);
+                if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
+            }
+            for (int xs = xs0 + npre; xs < xs1 && ok; ++xs, ++it) {
+                if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 42))) break;
+                if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, xs * g.kp);
+                for (int c = 0; c < my_chunks; ++c)
+                    dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmXB, full0 + 8 * s, my_n + c * 64, xs * g.kp * BK);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
             if (!ok && half == 0) {
-                // let the copies already issued land (bounded) before shared memory is released
+                // let the copies already issued land (bounded) before shared memory is reused or released
                 const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
                 for (uint32_t j = 0; j < back; ++j) {
                     const uint32_t jt = it - 1 - j;
@@ -239,22 +461,24 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     } else if (warp == 1) {
         // ================= MMA issuer (the pair's leader CTA) =================
         if (lane == 0 && half == 0) {
-            // fp32 accumulate, bf16 x bf16, A MN-major (W columns), B K-major (tokens), M = 256, N = 256
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(DG_TN >> 3) << 17) |
-                                       ((uint32_t)(DG_TM >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(NP >> 3) << 17) |
+                                   ((uint32_t)(256 >> 4) << 24);    // fp32 acc, bf16 x bf16, B MN-major, M = 256, N = NP
             const uint16_t mask = (uint16_t)(3u << leader);
             uint32_t acc = 0, s = 0, ph = 0;
             bool ok = true;
+            const int nstep = (ks1 - ks0) + (xs1 - xs0);
             for (int b = 0; b < nstep && ok; ++b) {
                 if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 44))) break;
                 tc_fence_after();
-                const uint32_t dw = sStage + s * STAGE_BYTES, dx = dw + W_BYTES;
-                // descriptors of successive 16-deep slices differ only in the start-address field (16-byte units)
-                const uint64_t da0 = desc_mn_major(dw, CHUNK_BYTES), db0 = desc_k_major(dx);
+                const uint32_t a0 = sA + s * a_stage_bytes, b0 = sB + s * b_stage_bytes;
+                for (int q = 0; q < g.kp; ++q) {
+                    // descriptors of successive 16-deep slices differ only in the start-address field (16-byte units)
+                    const uint64_t da0 = desc_k_major(a0 + q * A_STAGE_BYTES), db0 = desc_mn_major(b0 + q * CHUNK_BYTES, b_chunk_bytes);
 #pragma unroll
-                for (int j = 0; j < BK / 16; ++j) {
-                    dg_mma_pair(tmem_base, da0 + (uint64_t)(j * (UNIT_BYTES >> 4)), db0 + (uint64_t)(2 * j), idesc, acc);
-                    acc = 1;
+                    for (int j = 0; j < BK / 16; ++j) {
+                        dg_mma_pair(tmem_base, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(j * (UNIT_BYTES >> 4)), idesc, acc);
+                        acc = 1;
+                    }
                 }
                 dg_commit_pair(bar_empty + 8 * s, mask);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
@@ -271,139 +495,86 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         }
         __syncwarp();
     } else {
-        // ================= epilogue warps =================
-        // Thread (q, lane) owns W column n = my_n + 32 q + lane (tensor-memory lane 32 q + lane); the accumulator's
-        // columns are the tile's tokens.  The two warps of a lane quarter split the token columns between them.
-        const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
+        // ================= epilogue warps: wait for the pair's accumulator =================
         epi_ok = mbar_wait(bar_tfull, 0, abort_word, 46);
         epi_ok = __all_sync(0xffffffffu, epi_ok);
         tc_fence_after();
-        const uint32_t tl = tmem_base + ((uint32_t)(q * 32) << 16);
-        uint8_t* stg = smem + ew * 2048;            // the pipeline stages are free: every MMA of the pair has completed
-        const int ncol = my_n + q * 32;             // first W column of this warp
-        // 32 tokens x this warp's 32 columns, fp32 in registers (one column per thread) -> bf16 rows of y
-        auto store_chunk = [&](const float (&v)[32], int tok0) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) reinterpret_cast<bf16*>(stg)[j * 32 + lane] = __float2bfloat16_rn(v[j]);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int tk = i * 8 + (lane >> 2), sg = lane & 3;
-                const uint4 o = *reinterpret_cast<const uint4*>(stg + tk * 64 + sg * 16);
-                const int tok = tok0 + tk, col = ncol + sg * 8;
-                if (tok < g.T && col < g.Nout) *reinterpret_cast<uint4*>(g.C + (size_t)tok * g.ldc + col) = o;
-            }
-            __syncwarp();
-        };
-        if (g.S == 1) {
-            if (epi_ok) {
+    }
+
+    // ---- sum the S slices through distributed shared memory ---------------------------------------------------
+    // Row quarter q (32 rows) of each half is finished by pair (q mod S).  The other pairs' warps holding that
+    // quarter send their partial accumulators to a mailbox in the finishing CTA (thread to thread: the same
+    // tensor-memory lane on both sides, [column group][lane] 16-byte slots), and the finishing warp adds them to
+    // its own accumulator in ascending pair order.  The mailboxes reuse the pipeline stages.
+    const int q = warp & 3;
+    const uint32_t own = (uint32_t)(q % g.S);
+    if (g.S > 1) {
+        tc_fence_before();
+        dk_cluster_sync();      // every pair's MMAs are complete: the pipeline stages may be overwritten
+        tc_fence_after();
+        if (warp >= 2 && epi_ok && own != pairi && ((live >> pairi) & 1u)) {
+            const uint32_t si = pairi < own ? pairi : pairi - 1;
+            const uint32_t dst = dk_map_to_cta(sA, 2 * own + half) + (si * (uint32_t)qper + (uint32_t)(q / g.S)) * box_bytes +
+                                 (uint32_t)lane * 16u;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tc_ld_32x32(tl + ch * 128 + c * 32, v);
-                    tc_wait_ld();
-                    float f[32];
+            for (int c = 0; c < NP / 32; ++c) {
+                uint32_t v[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, v);
+                tc_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]);
-                    store_chunk(f, m0 + ch * 128 + c * 32);
-                }
+                for (int e = 0; e < 8; ++e)
+                    dk_st_cluster_v4(dst + (uint32_t)(c * 8 + e) * 512u, v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
             }
-        } else {
-            // ---- level 1: the cluster's two pairs (slices 2 cs and 2 cs + 1) exchange token halves through
-            // distributed shared memory.  Pair pi keeps tokens [128 pi, 128 pi + 128) and sends the other half to the
-            // CTA of the other pair that stages the same W columns, thread to thread ([column group][lane] 16-byte
-            // slots).  The mailbox is dedicated memory, so nobody waits before sending.
-            const int keep = (int)pi, send = 1 - keep;
-            if (epi_ok) {
-                const uint32_t dst = dk_map_to_cta(sMbox, crank ^ 2u) + (uint32_t)(q * 32 + lane) * 16u;
+        }
+        tc_fence_before();
+        dk_cluster_sync();      // all partial accumulators have landed
+        tc_fence_after();
+    }
+    if (warp >= 2 && epi_ok && own == pairi) {
+        const int row = my_m + q * 32 + lane;
+        bf16* crow = g.C + (size_t)row * g.ldc + n0;
+        const uint32_t mbox = sA + (uint32_t)(q / g.S) * box_bytes + (uint32_t)lane * 16u;
 #pragma unroll 1
-                for (int e = 0; e < 2; ++e) {
-                    uint32_t v[32];
-                    tc_ld_32x32(tl + send * 128 + ch * 64 + e * 32, v);
-                    tc_wait_ld();
+        for (int c = 0; c < NP / 32; ++c) {
+            uint32_t v[32];
+            tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + c * 32, v);
+            tc_wait_ld();
+            float acc[32];
 #pragma unroll
-                    for (int gq = 0; gq < 8; ++gq)
-                        dk_st_cluster_v4(dst + (uint32_t)((ch * 2 + e) * 8 + gq) * 2048u, v[4 * gq], v[4 * gq + 1], v[4 * gq + 2],
-                                         v[4 * gq + 3]);
-                }
-            }
-            mbar_arrive_remote_release(dk_map_to_cta(bar_mbox, crank ^ 2u));      // also on abort: the partner must not wait
-            {
-                bool ok = true;
-                if (!mbar_try_wait_cluster(bar_mbox, 0)) {
-                    unsigned long long t0 = 0;
-                    uint32_t spins = 0;
-                    while (!mbar_try_wait_cluster(bar_mbox, 0)) {
-                        if (((++spins) & 255u) == 0) {
-                            if (*abort_word != 0) { ok = false; break; }
-                            const unsigned long long now = global_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > WAIT_LIMIT_NS) { atomicCAS((int*)abort_word, 0, 47); ok = false; break; }
-                        }
-                    }
-                }
-                epi_ok = __all_sync(0xffffffffu, epi_ok && ok);
-            }
-            if (epi_ok) {
-                const uint32_t mb = sMbox + (uint32_t)(q * 32 + lane) * 16u;
-                // sum of the two slices of this cluster for 32 token columns (fp32 addition commutes, so both pairs
-                // form the same bits whichever of them adds)
-                auto level1 = [&](int e, float (&f)[32]) {
-                    uint32_t v[32];
-                    tc_ld_32x32(tl + keep * 128 + ch * 64 + e * 32, v);
-                    tc_wait_ld();
+            for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+            for (uint32_t src = 0; src < (uint32_t)g.S; ++src) {      // ascending pair order
+                if (!((live >> src) & 1u)) continue;                  // a slice without steps never wrote its accumulator
+                if (src == pairi) {
 #pragma unroll
-                    for (int gq = 0; gq < 8; ++gq) {
+                    for (int e = 0; e < 32; ++e) acc[e] += __uint_as_float(v[e]);
+                } else {
+                    const uint32_t si = src < pairi ? src : src - 1;
+                    const uint32_t a = mbox + si * (uint32_t)qper * box_bytes + (uint32_t)(c * 8) * 512u;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
                         float4 p;
                         asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                      : "=f"(p.x), "=f"(p.y), "=f"(p.z), "=f"(p.w)
-                                     : "r"(mb + (uint32_t)((ch * 2 + e) * 8 + gq) * 2048u));
-                        f[4 * gq] = __uint_as_float(v[4 * gq]) + p.x;
-                        f[4 * gq + 1] = __uint_as_float(v[4 * gq + 1]) + p.y;
-                        f[4 * gq + 2] = __uint_as_float(v[4 * gq + 2]) + p.z;
-                        f[4 * gq + 3] = __uint_as_float(v[4 * gq + 3]) + p.w;
+                                     : "r"(a + (uint32_t)e * 512u));
+                        acc[4 * e] += p.x; acc[4 * e + 1] += p.y; acc[4 * e + 2] += p.z; acc[4 * e + 3] += p.w;
                     }
-                };
-                const int tok_keep = m0 + keep * 128 + ch * 64;
-                if (g.S == 2) {
-#pragma unroll 1
-                    for (int e = 0; e < 2; ++e) {
-                        float f[32];
-                        level1(e, f);
-                        store_chunk(f, tok_keep + e * 32);
-                    }
-                } else {
-                    // ---- level 2: the tile's two clusters (slices {0,1} and {2,3}) exchange token quarters through
-                    // global memory: cluster cs finishes chunk cs of each warp's 64 columns and sends the other chunk,
-                    // thread to thread, to the same CTA and warp of the other cluster.
-                    const int slot_out = ((tile * 2 + (1 - cs)) * 4 + (int)crank) * 8 + ew;
-                    const int slot_in = ((tile * 2 + cs) * 4 + (int)crank) * 8 + ew;
-                    {
-                        float f[32];
-                        level1(1 - cs, f);
-                        float* o = g.xbuf + (size_t)slot_out * 1024 + lane * 4;
+                }
+            }
+            if (row < g.T) {
 #pragma unroll
-                        for (int gq = 0; gq < 8; ++gq)
-                            *reinterpret_cast<float4*>(o + gq * 128) = make_float4(f[4 * gq], f[4 * gq + 1], f[4 * gq + 2], f[4 * gq + 3]);
-                        __syncwarp();
-                        if (lane == 0) st_release_gpu(g.sync + SY_FLAGS + slot_out, 1);
-                    }
-                    float f[32];
-                    level1(cs, f);
-                    bool ok = true;
-                    if (lane == 0) ok = wait_word_ge(g.sync + SY_FLAGS + slot_in, 1, abort_word, 48);
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (ok) {
-                        const float* in = g.xbuf + (size_t)slot_in * 1024 + lane * 4;
-#pragma unroll
-                        for (int gq = 0; gq < 8; ++gq) {
-                            const uint4 p = ld_cg_v4(in + gq * 128);
-                            f[4 * gq] += __uint_as_float(p.x);
-                            f[4 * gq + 1] += __uint_as_float(p.y);
-                            f[4 * gq + 2] += __uint_as_float(p.z);
-                            f[4 * gq + 3] += __uint_as_float(p.w);
-                        }
-                        store_chunk(f, tok_keep + cs * 32);
+                for (int e = 0; e < 4; ++e) {
+                    const int col = n0 + c * 32 + e * 8;
+                    if (col < g.Nout) {
+                        uint4 o;
+                        __nv_bfloat162 p0 = __floats2bfloat162_rn(acc[e * 8 + 0], acc[e * 8 + 1]);
+                        __nv_bfloat162 p1 = __floats2bfloat162_rn(acc[e * 8 + 2], acc[e * 8 + 3]);
+                        __nv_bfloat162 p2 = __floats2bfloat162_rn(acc[e * 8 + 4], acc[e * 8 + 5]);
+                        __nv_bfloat162 p3 = __floats2bfloat162_rn(acc[e * 8 + 6], acc[e * 8 + 7]);
+                        o.x = *reinterpret_cast<uint32_t*>(&p0);
+                        o.y = *reinterpret_cast<uint32_t*>(&p1);
+                        o.z = *reinterpret_cast<uint32_t*>(&p2);
+                        o.w = *reinterpret_cast<uint32_t*>(&p3);
+                        *reinterpret_cast<uint4*>(crow + c * 32 + e * 8) = o;
                     }
                 }
             }
@@ -412,385 +583,13 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
 
     // ---- teardown ---------------------------------------------------------------------------------------------
     tc_fence_before();
-    dk_cluster_sync();      // the cluster leaves together (barriers, mailboxes and tensor memory are shared)
+    dk_cluster_sync();      // the pair leaves together (its barriers and tensor memory are shared)
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
+    if (threadIdx.x == 0) dk_wait_prerequisites();   // this grid never completes before the shrink grid it depends on
     if (threadIdx.x == 0 && *abort_word != 0) {
         if (atomicCAS(g.status, 0, DEV_TIMEOUT) == 0) g.status[1] = *abort_word * 1000000 + (int)blockIdx.x;
-    }
-    if (g.reset_at_end && threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(g.sync + SY_EXIT, 1) == (int)gridDim.x - 1) {
-            for (int i = 0; i < g.n_flags; ++i) g.sync[SY_FLAGS + i] = 0;
-            g.sync[SY_TICKET] = 0;
-            g.sync[SY_DONE] = 0;
-            __threadfence();
-            g.sync[SY_EXIT] = 0;
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------------------
-// k_decode_shrink
-// ---------------------------------------------------------------------------------------------------------------
-constexpr int SH_THREADS = 288;        // warp 0: producer (work units, bulk copies), warps 1..8: MMA + output
-constexpr int SH_CONS = 8;
-constexpr int SH_KC = 512;             // elements of the contraction per pipeline stage
-constexpr int SH_PITCH = SH_KC * 2 + 16;     // bytes between staged rows: 16 B of padding keeps ldmatrix conflict-free
-constexpr int SH_RG = 32;              // ranks per streaming group
-constexpr int SH_PASS = 16;            // tokens per pass (one m16 MMA tile)
-constexpr int SH_MAX_T = 1024;
-constexpr int SH_TABLE_SMEM = 1032;    // the segment table is staged in shared memory when S + 1 <= this
-
-struct ShrinkStageMeta {
-    int t;              // tenant slot; == cap: tokens routed to no adapter
-    int jg0, rg;        // first rank and number of ranks (16 or 32) of this streaming group; rg == 0: nothing to compute
-    int np;             // tokens of the pass
-    int kel;            // elements of the contraction in this stage
-    int first_chunk, last_chunk;    // of the (pass, rank group)
-    int pass_first;     // first stage of the pass: the pass's rows of hd / h are cleared outside the tenant's columns
-    int unit_last;      // last stage of the work unit
-    int stop;           // no more work
-    int rpt;            // tenant's rank rounded up to 16
-    float scale;
-    int tok[SH_PASS];
-};
-
-struct DecodeShrinkArgs {
-    int T, K, RP, cap;
-    int S;                              // segments; < 0: tok_slot already holds the per-token slots
-    int G;                              // work units per tenant: unit (t, i) takes the tenant's 16-token passes i, i + G, ...
-    int n_units;                        // (cap + 1) * G
-    int nbuf;                           // pipeline stages
-    int n_flags;                        // exchange flags of the GEMM to clear at the end
-    int reset_at_end;                   // normal order (GEMM grid first): this grid ends last and clears counters and flags
-    const int32_t* seg_offsets;
-    const int32_t* seg_slot;
-    const bf16* x;
-    int64_t ldx;
-    const bf16* At;                     // [cap*RP][K]
-    const int32_t* d_rank;
-    const float* d_scale;
-    int32_t* tok_slot;                  // [T]
-    float* h_out;                       // [T][RP]
-    bf16* hd;                           // [T][hd_cols]
-    int hd_cols;
-    int32_t* status;
-    int32_t* sync;
-};
-
-static size_t decode_shrink_stage_bytes(int RP) { return (size_t)(SH_PASS + std::min(RP, SH_RG)) * SH_PITCH; }
-static size_t decode_shrink_fixed_smem(int64_t T, int32_t S) {
-    const size_t Tp = (size_t)((T + 31) / 32 * 32);
-    const bool staged = S >= 0 && S + 1 <= SH_TABLE_SMEM;
-    return 1024 /* alignment */ + 4 * (2 * Tp + (staged ? (size_t)(2 * S + 1) : 0)) + 16 +
-           sizeof(float) * 2 * SH_CONS * SH_PASS * SH_RG + 8 * sizeof(ShrinkStageMeta) + 256;
-}
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-        "{%0, %1, %2, %3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
-                 "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-
-// Work unit u = (tenant t = u / G, share i = u % G): the tenant's tokens in ascending order are cut into passes of 16,
-// and the unit takes passes i, i + G, ...  For each pass and each group of up to 32 ranks the token rows of x and the
-// adapter rows of At stream through shared memory in 512-deep stages (one bulk copy per row, issued by the lanes of the
-// producer warp); the eight consumer warps take the 16-deep slices of a stage in turn (m16n8k16 fragments by ldmatrix)
-// and their partial products are added in warp order.  Nothing here depends on which CTA takes which unit.
-__global__ void __launch_bounds__(SH_THREADS, 1) k_decode_shrink(const DecodeShrinkArgs g) {
-    extern __shared__ uint8_t sh_raw[];
-    uint8_t* sh = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sh_raw) + 1023) & ~uintptr_t(1023));
-    const int Tp = (g.T + 31) / 32 * 32;
-    const bool staged_tab = g.S >= 0 && g.S + 1 <= SH_TABLE_SMEM;
-    const size_t stage_bytes = (size_t)(SH_PASS + min(g.RP, SH_RG)) * SH_PITCH;
-    uint8_t* bufs = sh;                                                  // [nbuf][rows][SH_PITCH]
-    float* red = reinterpret_cast<float*>(sh + (size_t)g.nbuf * stage_bytes);       // [2][8 warps][16 tokens][32 ranks]
-    ShrinkStageMeta* metas = reinterpret_cast<ShrinkStageMeta*>(red + 2 * SH_CONS * SH_PASS * SH_RG);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(metas + 8);
-    int32_t* s_slot = reinterpret_cast<int32_t*>(bars + 16);            // [Tp]
-    int32_t* s_list = s_slot + Tp;                                      // [Tp] producer's token list of the current unit
-    int32_t* s_off = s_list + Tp;                                       // [S + 1] staged table
-    int32_t* s_stab = s_off + (staged_tab ? g.S + 1 : 0);
-    volatile int* abort_word = reinterpret_cast<volatile int*>(bars + 16) - 1;
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 64;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    dk_launch_dependents();     // whatever follows this call in the stream may be scheduled; it waits for this grid's end
-    if (tid == 0) {
-        for (int s = 0; s < g.nbuf; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, SH_CONS);
-        }
-        *abort_word = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-
-    // ---- per-token slot (every CTA, redundantly: the table is tiny) ---------------------------------------------
-    if (g.S >= 0) {
-        if (staged_tab) {
-            for (int s = tid; s <= g.S; s += SH_THREADS) {
-                s_off[s] = g.seg_offsets[s];
-                if (s < g.S) s_stab[s] = g.seg_slot[s];
-            }
-            __syncthreads();
-        }
-        if (blockIdx.x == 0) {
-            for (int s = tid; s < g.S; s += SH_THREADS) {
-                const int a = staged_tab ? s_off[s] : g.seg_offsets[s], b = staged_tab ? s_off[s + 1] : g.seg_offsets[s + 1];
-                if (b < a || a < 0 || b > g.T) dk_report(g.status, DEV_BAD_TABLE, s);
-                if (s == 0 && a != 0) dk_report(g.status, DEV_BAD_TABLE, -1);
-                if (s == g.S - 1 && b != g.T) dk_report(g.status, DEV_BAD_TABLE, -2);
-            }
-            if (tid == 0 && g.S == 0 && g.T != 0) dk_report(g.status, DEV_BAD_TABLE, -3);
-        }
-        for (int i = tid; i < g.T; i += SH_THREADS) {
-            int lo = 0, hi = g.S;
-            while (lo < hi) {       // first s with seg_offsets[s + 1] > i
-                const int mid = (lo + hi) >> 1;
-                const int v = staged_tab ? s_off[mid + 1] : g.seg_offsets[mid + 1];
-                if (v > i) hi = mid; else lo = mid + 1;
-            }
-            s_slot[i] = lo < g.S ? (staged_tab ? s_stab[lo] : g.seg_slot[lo]) : -1;
-        }
-    } else {
-        for (int i = tid; i < g.T; i += SH_THREADS) s_slot[i] = g.tok_slot[i];
-    }
-    __syncthreads();
-    for (int i = tid; i < g.T; i += SH_THREADS) {
-        int s = s_slot[i];
-        if (s < -1 || s >= g.cap) {
-            if (blockIdx.x == 0) dk_report(g.status, DEV_BAD_INDEX, i);
-            s = -1;
-        }
-        s_slot[i] = s;
-        if (blockIdx.x == 0) g.tok_slot[i] = s;
-    }
-    __syncthreads();
-
-    if (warp == 0) {
-        // ================= producer =================
-        uint32_t s = 0, ph = 0;
-        bool ok = true;
-        // one stage: wait for its buffer, publish its description, then one bulk copy per row
-        auto emit = [&](const ShrinkStageMeta& m, int p0, int k0) {
-            if (!ok) return;
-            bool w = true;
-            if (lane == 0) w = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 51);
-            ok = __shfl_sync(0xffffffffu, (int)w, 0) != 0;
-            if (!ok) return;
-            ShrinkStageMeta* d = metas + s;
-            if (lane == 0) {
-                d->t = m.t; d->jg0 = m.jg0; d->rg = m.rg; d->np = m.np; d->kel = m.kel; d->first_chunk = m.first_chunk;
-                d->last_chunk = m.last_chunk; d->pass_first = m.pass_first; d->unit_last = m.unit_last; d->stop = m.stop;
-                d->rpt = m.rpt; d->scale = m.scale;
-            }
-            if (lane < SH_PASS) d->tok[lane] = lane < m.np ? s_list[p0 + lane] : -1;
-            __syncwarp();
-            const int nrows = m.rg > 0 ? m.np + m.rg : 0;
-            const uint32_t rowbytes = (uint32_t)m.kel * 2u;
-            if (lane == 0) mbar_expect_tx(bar_full + 8 * s, (uint32_t)nrows * rowbytes);
-            __syncwarp();
-            uint8_t* buf = bufs + (size_t)s * stage_bytes;
-            for (int r = lane; r < nrows; r += 32) {
-                const bf16* src;
-                uint32_t dst;
-                if (r < m.np) {
-                    src = g.x + (size_t)s_list[p0 + r] * g.ldx + k0;
-                    dst = smem_u32(buf + (size_t)r * SH_PITCH);
-                } else {
-                    src = g.At + ((size_t)m.t * g.RP + m.jg0 + (r - m.np)) * g.K + k0;
-                    dst = smem_u32(buf + (size_t)(SH_PASS + r - m.np) * SH_PITCH);
-                }
-                bulk_load_row(dst, src, rowbytes, bar_full + 8 * s);
-            }
-            if (++s == (uint32_t)g.nbuf) { s = 0; ph ^= 1; }
-        };
-        while (ok) {
-            int u = 0;
-            if (lane == 0) u = atomicAdd(g.sync + SY_TICKET, 1);
-            u = __shfl_sync(0xffffffffu, u, 0);
-            if (u >= g.n_units) break;
-            const int t = u / g.G, gi = u % g.G;
-            // the unit's tokens: token number e of the tenant (ascending) belongs to pass e / 16
-            int seen = 0, mine = 0;
-            for (int i0 = 0; i0 < g.T; i0 += 32) {
-                const int i = i0 + lane;
-                bool m = false;
-                if (i < g.T) {
-                    const int sl = s_slot[i];
-                    m = t < g.cap ? sl == t : sl < 0;
-                }
-                const unsigned bal = __ballot_sync(0xffffffffu, m);
-                const int e = seen + __popc(bal & ((1u << lane) - 1u));
-                const bool take = m && ((e / SH_PASS) % g.G) == gi;
-                const unsigned balt = __ballot_sync(0xffffffffu, take);
-                if (take) s_list[mine + __popc(balt & ((1u << lane) - 1u))] = i;
-                seen += __popc(bal);
-                mine += __popc(balt);
-            }
-            __syncwarp();
-            if (mine == 0) {
-                if (lane == 0) atomicAdd(g.sync + SY_DONE, 1);
-                continue;
-            }
-            const int r_t = t < g.cap ? g.d_rank[t] : 0;
-            ShrinkStageMeta m;
-            m.t = t; m.stop = 0;
-            m.rpt = (r_t + 15) & ~15;
-            m.scale = t < g.cap ? g.d_scale[t] : 0.f;
-            const int ngroups = (m.rpt + SH_RG - 1) / SH_RG;
-            const int nchunk = (g.K + SH_KC - 1) / SH_KC;
-            for (int p0 = 0; p0 < mine && ok; p0 += SH_PASS) {
-                m.np = min(SH_PASS, mine - p0);
-                const bool last_pass = p0 + SH_PASS >= mine;
-                if (ngroups == 0) {
-                    m.jg0 = 0; m.rg = 0; m.kel = 0; m.first_chunk = 1; m.last_chunk = 1; m.pass_first = 1; m.unit_last = last_pass;
-                    emit(m, p0, 0);
-                    continue;
-                }
-                for (int jg = 0; jg < ngroups && ok; ++jg) {
-                    m.jg0 = jg * SH_RG;
-                    m.rg = min(SH_RG, m.rpt - m.jg0);
-                    for (int c = 0; c < nchunk && ok; ++c) {
-                        m.kel = min(SH_KC, g.K - c * SH_KC);
-                        m.first_chunk = c == 0;
-                        m.last_chunk = c == nchunk - 1;
-                        m.pass_first = jg == 0 && c == 0;
-                        m.unit_last = last_pass && jg == ngroups - 1 && m.last_chunk;
-                        emit(m, p0, c * SH_KC);
-                    }
-                }
-            }
-        }
-        {
-            ShrinkStageMeta m;
-            m.t = 0; m.jg0 = 0; m.rg = 0; m.np = 0; m.kel = 0; m.first_chunk = 0; m.last_chunk = 0; m.pass_first = 0; m.unit_last = 0;
-            m.stop = 1; m.rpt = 0; m.scale = 0.f;
-            emit(m, 0, 0);
-        }
-        if (!ok && lane == 0) {
-            // the consumers may be waiting for a stage that will never come: they poll the abort word and leave.  Let the
-            // copies already issued land (bounded) before shared memory is released.
-            for (int j = 0; j < g.nbuf; ++j) {
-                const unsigned long long t0 = global_ns();
-                (void)j;
-                while (global_ns() - t0 < 20000ull) {
-                }
-            }
-        }
-    } else {
-        // ================= consumers =================
-        const int cw = warp - 1, ctid = tid - 32;
-        const int gq = lane >> 2, tq = lane & 3;
-        uint32_t s = 0, ph = 0, par = 0;
-        float acc[SH_RG / 8][4];
-        while (true) {
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_word, 52)) break;
-            const ShrinkStageMeta m = metas[s];
-            if (m.stop) break;
-            const uint8_t* buf = bufs + (size_t)s * stage_bytes;
-            if (m.first_chunk) {
-#pragma unroll
-                for (int a = 0; a < SH_RG / 8; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
-            }
-            if (m.pass_first) {
-                // clear the pass's rows of hd outside the tenant's own columns, and h beyond its padded rank: two rows per warp
-                const int own0 = m.rpt > 0 ? m.t * g.RP : 0, own1 = own0 + m.rpt;
-                for (int rr = cw; rr < m.np; rr += SH_CONS) {
-                    const int tok = m.tok[rr];
-                    bf16* row = g.hd + (size_t)tok * g.hd_cols;
-                    for (int c = lane * 8; c < g.hd_cols; c += 256)
-                        if (c < own0 || c >= own1) *reinterpret_cast<uint4*>(row + c) = make_uint4(0u, 0u, 0u, 0u);
-                    for (int j = m.rpt + lane; j < g.RP; j += 32) g.h_out[(size_t)tok * g.RP + j] = 0.f;
-                }
-            }
-            if (m.rg > 0) {
-                const uint32_t xb = smem_u32(buf), ab = xb + SH_PASS * SH_PITCH;
-                const uint32_t x_lane = xb + (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * SH_PITCH + (lane >> 4) * 16);
-                const uint32_t a_lane = ab + (uint32_t)(((lane & 7) + ((lane >> 4) & 1) * 8) * SH_PITCH + ((lane >> 3) & 1) * 16);
-                const int nk16 = m.kel >> 4;
-                for (int ks = cw; ks < nk16; ks += SH_CONS) {
-                    uint32_t a0, a1, a2, a3;
-                    ldmatrix_x4(x_lane + ks * 32, a0, a1, a2, a3);
-#pragma unroll
-                    for (int jj = 0; jj < SH_RG / 16; ++jj) {
-                        if (jj * 16 < m.rg) {
-                            uint32_t b0, b1, b2, b3;
-                            ldmatrix_x4(a_lane + jj * 16 * SH_PITCH + ks * 32, b0, b1, b2, b3);
-                            mma_bf16_16816(acc[2 * jj], a0, a1, a2, a3, b0, b1);
-                            mma_bf16_16816(acc[2 * jj + 1], a0, a1, a2, a3, b2, b3);
-                        }
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-            if (m.last_chunk && m.rg > 0) {
-                // warp partials -> sum in warp order -> h (fp32) and the tenant's columns of hd
-                float* rp = red + (size_t)par * SH_CONS * SH_PASS * SH_RG;
-                float* wp = rp + cw * SH_PASS * SH_RG;
-#pragma unroll
-                for (int a = 0; a < SH_RG / 8; ++a) {
-                    if (a * 8 < m.rg) {
-                        wp[gq * SH_RG + a * 8 + 2 * tq] = acc[a][0];
-                        wp[gq * SH_RG + a * 8 + 2 * tq + 1] = acc[a][1];
-                        wp[(gq + 8) * SH_RG + a * 8 + 2 * tq] = acc[a][2];
-                        wp[(gq + 8) * SH_RG + a * 8 + 2 * tq + 1] = acc[a][3];
-                    }
-                }
-                bar_consumers();
-                for (int e = ctid; e < SH_PASS * m.rg; e += SH_CONS * 32) {
-                    const int i = e / m.rg, j = e - i * m.rg;
-                    if (i < m.np) {
-                        float v = 0.f;
-#pragma unroll
-                        for (int w = 0; w < SH_CONS; ++w) v += rp[w * SH_PASS * SH_RG + i * SH_RG + j];      // fixed order
-                        const int tok = m.tok[i];
-                        g.h_out[(size_t)tok * g.RP + m.jg0 + j] = v;
-                        g.hd[(size_t)tok * g.hd_cols + m.t * g.RP + m.jg0 + j] = __float2bfloat16_rn(m.scale * v);
-                    }
-                }
-                par ^= 1;
-            }
-            if (m.unit_last) {
-                __threadfence();
-                bar_consumers();
-                if (ctid == 0) atomicAdd(g.sync + SY_DONE, 1);
-            }
-            if (++s == (uint32_t)g.nbuf) { s = 0; ph ^= 1; }
-        }
-    }
-
-    // ---- end: this grid completes after the GEMM grid; the last CTA to get here clears the counters and flags -------
-    __syncthreads();
-    if (tid == 0) {
-        if (*abort_word != 0 && atomicCAS(g.status, 0, DEV_TIMEOUT) == 0) g.status[1] = *abort_word * 1000000 + (int)blockIdx.x;
-        dk_wait_prerequisites();
-        __threadfence();
-        if (g.reset_at_end && atomicAdd(g.sync + SY_EXIT, 1) == (int)gridDim.x - 1) {
-            for (int i = 0; i < g.n_flags; ++i) g.sync[SY_FLAGS + i] = 0;
-            g.sync[SY_TICKET] = 0;
-            g.sync[SY_DONE] = 0;
-            __threadfence();
-            g.sync[SY_EXIT] = 0;
-        }
     }
 }
 
@@ -826,185 +625,151 @@ marlaas_status_t make_panel_map(CUtensorMap* map, const void* ptr, int64_t rows,
 // ---------------------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------------------
-namespace {
-
-struct DecodeShape {
-    int S;          // contraction slices per tile
-    int clusters;   // GEMM clusters
-    int csz;        // CTAs per cluster
-    bool ok;
-};
-
-// Largest number of co-resident clusters of `csz` CTAs of the GEMM kernel with `smem` bytes each (cached per device).
-marlaas_status_t decode_max_clusters(int device, int csz, size_t smem, int* out) {
-    static int cache[64][2] = {};
-    const int ci = csz == 2 ? 0 : 1;
-    if (device >= 0 && device < 64 && cache[device][ci] != 0) {
-        *out = cache[device][ci];
-        return MARLAAS_OK;
-    }
-    MARLAAS_CUDA_TRY(cudaFuncSetAttribute(sm100::k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    cudaLaunchConfig_t qc = {};
-    qc.gridDim = dim3((unsigned)(csz * 64));
-    qc.blockDim = dim3(sm100::DG_THREADS);
-    qc.dynamicSmemBytes = smem;
-    cudaLaunchAttribute qa;
-    qa.id = cudaLaunchAttributeClusterDimension;
-    qa.val.clusterDim.x = (unsigned)csz; qa.val.clusterDim.y = 1; qa.val.clusterDim.z = 1;
-    qc.attrs = &qa; qc.numAttrs = 1;
-    int mc = 0;
-    MARLAAS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&mc, sm100::k_decode_gemm, &qc));
-    if (mc < 1) mc = -1;
-    if (device >= 0 && device < 64) cache[device][ci] = mc;
-    *out = mc;
-    return MARLAAS_OK;
-}
-
-constexpr int DECODE_MIN_SHRINK_SMS = 8;       // SMs the GEMM's grid must leave to the shrink grid
-constexpr int DECODE_MAX_SHRINK_CTAS = 20;
-
-// Slices per tile: as many as fill the SMs with one wave of clusters while leaving room for the shrink grid.  Uses only
-// the pool's dimensions and the SM count, so that the workspace size and the launch agree.
-DecodeShape decode_shape(const marlaas_pool* pool, int64_t T) {
-    DecodeShape d = {1, 0, 2, false};
-    const int64_t tiles = cdiv(T, sm100::DG_TN) * cdiv(pool->N, sm100::DG_TM);
-    const int64_t num_ks = pool->K / sm100::BK;
-    const int room = pool->sm_count - DECODE_MIN_SHRINK_SMS;
-    // clusters of 4 pack less densely than pairs: 33 are co-resident on a 148-SM part (the launch checks the real figure)
-    const int mc4 = (pool->sm_count - 16) / 4;
-    if (num_ks >= 4 && tiles * 2 <= mc4 && tiles * 8 <= room) { d.S = 4; d.clusters = (int)tiles * 2; d.csz = 4; d.ok = true; }
-    else if (num_ks >= 2 && tiles <= mc4 && tiles * 4 <= room) { d.S = 2; d.clusters = (int)tiles; d.csz = 4; d.ok = true; }
-    else if (tiles * 2 <= room) { d.S = 1; d.clusters = (int)tiles; d.csz = 2; d.ok = true; }
-    return d;
-}
-
-}  // namespace
-
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T) {
-    if (!(T > 0 && T <= sm100::SH_MAX_T && (int64_t)pool->cap * pool->RP <= 2048 && pool->sm_count >= 16 && (pool->K % 64) == 0))
+    if (!(T > 0 && T <= sm100::DS_MAX_T && (int64_t)pool->cap * pool->RP <= 2048 && pool->sm_count >= 8 && (pool->K % 64) == 0))
         return false;
-    return decode_shape(pool, T).ok;
+    // beyond one 256-token tile only while all (token tile, 256-column strip) pairs make a single wave of CTA pairs
+    return T <= 256 || cdiv(T, 256) * cdiv(pool->N, 256) <= pool->sm_count / 2;
 }
 
-size_t decode_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T) {
-    if (!decode_sm100_eligible(pool, T)) return 0;
-    const DecodeShape d = decode_shape(pool, T);
-    return d.S == 4 ? (size_t)(d.clusters / 2) * 2 * 4 * 8 * 4096 : 0;
-}
+// Shared memory one shrink CTA holds (static + dynamic + the system's 1 KB): a GEMM that wants shrink CTAs beside it on
+// its SMs leaves room for two of them.
+size_t decode_shrink_smem_bytes(int64_t T, int32_t S) { return sizeof(sm100::DecodeShrinkSmem) + sm100::decode_shrink_dyn_smem(T, S) + 1024; }
 
-marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
-                                     int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
-                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st, bool serial) {
+// The shrink kernel alone: (cap + 1) * G clusters, K split over the CTAs of a cluster.  Writes tok_slot, h and hd; its
+// CTAs are small (four per SM), so they fit on whatever SMs a GEMM launched as its programmatic dependent leaves free.
+marlaas_status_t launch_decode_shrink(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, int32_t S,
+                                      const int32_t* seg_offsets, const int32_t* seg_slot, const Workspace& ws, float* h_out,
+                                      cudaStream_t st) {
     using namespace sm100;
-    const int64_t K = pool->K, N = pool->N;
+    const int64_t K = pool->K;
     const int hd_cols = (int)align_up((size_t)pool->cap * pool->RP, 64);     // pitch of hd: whole 64-deep panels
-    const DecodeShape shape = decode_shape(pool, T);
-
-    int last_used = -1;
-    for (int s = 0; s < pool->cap; ++s)
-        if (pool->slots[s].used && pool->slots[s].rank > 0) last_used = s;
-
-    // ---- GEMM with the expand as extra steps of the contraction ----
-    DecodeGemmArgs g;
-    g.T = (int)T; g.Nout = (int)N;
-    g.C = y; g.ldc = ldy; g.status = pool->d_status; g.sync = pool->d_sync; g.xbuf = ws.xbuf;
-    g.S = shape.S;
-    g.nstrips = (int)cdiv(N, DG_TM);
-    g.num_ks = (int)(K / BK);
-    g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
-    g.w3d = (N % 64) == 0;
-    constexpr size_t stage_bytes = 2 * CHUNK_BYTES + A_STAGE_BYTES;
-    const size_t fixed = 1024 + (g.S > 1 ? DG_MBOX_BYTES : 0) + 512;
-    g.stages = (int)std::min<size_t>(7, ((size_t)227 * 1024 - fixed) / stage_bytes);
-    const size_t gemm_smem = fixed + (size_t)g.stages * stage_bytes;
-    int mc = 0;
-    marlaas_status_t rc;
-    if ((rc = decode_max_clusters(pool->device, shape.csz, gemm_smem, &mc)) != MARLAAS_OK) return rc;
-    if (mc < shape.clusters)
-        return fail(MARLAAS_ERR_UNSUPPORTED_DEVICE, "lora_forward: %d clusters of %d CTAs are not co-resident on this device (%d are)",
-                    shape.clusters, shape.csz, mc);
-
-    // ---- shrink: work units (tenant, share) handed to the CTAs that fit beside the GEMM's clusters ----
     DecodeShrinkArgs a;
     a.T = (int)T; a.K = (int)K; a.RP = pool->RP; a.cap = pool->cap;
     a.S = S; a.seg_offsets = seg_offsets; a.seg_slot = seg_slot;
     a.x = x; a.ldx = ldx; a.At = pool->d_At; a.d_rank = pool->d_rank; a.d_scale = pool->d_scale;
-    a.tok_slot = ws.tok_slot; a.h_out = h_out; a.hd = ws.hd; a.hd_cols = hd_cols; a.status = pool->d_status; a.sync = pool->d_sync;
-    const int shrink_ctas = std::max(1, std::min(DECODE_MAX_SHRINK_CTAS, pool->sm_count - shape.clusters * shape.csz));
-    const int passes = (int)cdiv(T, SH_PASS);
-    a.G = std::max(1, std::min(passes, (2 * shrink_ctas + pool->cap) / (pool->cap + 1)));
-    a.n_units = (pool->cap + 1) * a.G;
-    a.n_flags = g.S == 4 ? shape.clusters * 4 * 8 : 0;
-    a.reset_at_end = serial ? 0 : 1;
-    g.n_flags = a.n_flags;
-    g.reset_at_end = serial ? 1 : 0;
-    const size_t sh_fixed = decode_shrink_fixed_smem(T, S), sh_stage = decode_shrink_stage_bytes(pool->RP);
-    a.nbuf = (int)std::min<size_t>(6, ((size_t)200 * 1024 - sh_fixed) / sh_stage);
-    // at least 120 KB, so that two of these CTAs never share an SM (and none fits beside a GEMM CTA)
-    const size_t shrink_smem = std::max<size_t>(sh_fixed + (size_t)a.nbuf * sh_stage, 120 * 1024);
-    g.n_units = a.n_units;
+    a.tok_slot = ws.tok_slot; a.h_out = h_out; a.hd = ws.hd; a.hd_cols = hd_cols; a.status = pool->d_status;
+    int cs = DS_MAX_CS;
+    while (cs > 1 && K / cs < 32 * 4 * DS_UB) cs >>= 1;      // a full batch of loads per warp
+    // with few tenants a tenant has many 16-token passes: several clusters share them, as many as keep the grid
+    // within two CTAs per SM
+    const int passes = (int)cdiv(T, DS_PASS);
+    a.G = std::max(1, std::min(passes, (2 * pool->sm_count) / ((pool->cap + 1) * cs)));
+    static bool carveout_set[64] = {};
+    if (pool->device >= 64 || !carveout_set[pool->device]) {
+        // same shared-memory configuration as the GEMM, so that CTAs of both kernels can share an SM
+        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_shrink, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                              (int)cudaSharedmemCarveoutMaxShared));
+        if (pool->device < 64) carveout_set[pool->device] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((pool->cap + 1) * a.G * cs));
+    cfg.blockDim = dim3(DS_THREADS);
+    cfg.dynamicSmemBytes = decode_shrink_dyn_smem(T, S);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode_shrink, a));
+    count_launch();
+    return MARLAAS_OK;
+}
 
-    alignas(64) CUtensorMap tmW, tmX, tmXW, tmXX;
-    if ((rc = make_panel_map(&tmX, x, T, K, ldx, 1, 128)) != MARLAAS_OK) return rc;
-    if (g.w3d) rc = make_panel_map(&tmW, W, K, N, ldw, 2, BK);
-    else rc = make_map(&tmW, W, K, N, ldw, 64, BK);
-    if (rc != MARLAAS_OK) return rc;
+marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
+                                     int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
+                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st) {
+    using namespace sm100;
+    const int64_t K = pool->K, N = pool->N;
+    const int hd_cols = (int)align_up((size_t)pool->cap * pool->RP, 64);     // pitch of hd: whole 64-deep panels
+
+    {
+        marlaas_status_t rcs = launch_decode_shrink(pool, T, x, ldx, S, seg_offsets, seg_slot, ws, h_out, st);
+        if (rcs != MARLAAS_OK) return rcs;
+    }
+
+    // ---- GEMM with the expand as extra steps of the contraction ----
+    int last_used = -1;
+    for (int s = 0; s < pool->cap; ++s)
+        if (pool->slots[s].used && pool->slots[s].rank > 0) last_used = s;
+    DecodeGemmArgs g;
+    g.T = (int)T; g.Nout = (int)N;
+    g.C = y; g.ldc = ldy; g.status = pool->d_status;
+    // strip width and contraction slices: fill the SMs with one wave of clusters of 2 * S CTAs
+    struct Shape { int nch, S; };
+    const Shape shapes[] = {{1, 2}, {2, 2}, {1, 1}, {2, 1}, {1, 4}, {2, 4}};
+    Shape pick = {2, 1};
+    int64_t best = -1;
+    const int64_t mtiles = cdiv(T, 256);
+    static int max_clusters[64][3] = {};      // per device, cluster size 2 / 4 / 8
+    constexpr int DG_SMEM = 200 * 1024;
+    for (const Shape& sh : shapes) {
+        const int csz = 2 * sh.S;
+        const int ci = sh.S == 1 ? 0 : sh.S == 2 ? 1 : 2;
+        int mc = pool->device < 64 ? max_clusters[pool->device][ci] : 0;
+        if (mc == 0) {
+            MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            cudaLaunchConfig_t qc = {};
+            qc.gridDim = dim3((unsigned)(csz * 64));
+            qc.blockDim = dim3(DG_THREADS);
+            qc.dynamicSmemBytes = DG_SMEM;
+            cudaLaunchAttribute qa;
+            qa.id = cudaLaunchAttributeClusterDimension;
+            qa.val.clusterDim.x = (unsigned)csz; qa.val.clusterDim.y = 1; qa.val.clusterDim.z = 1;
+            qc.attrs = &qa; qc.numAttrs = 1;
+            MARLAAS_CUDA_TRY(cudaOccupancyMaxActiveClusters(&mc, k_decode_gemm, &qc));
+            if (mc < 1) mc = -1;
+            if (pool->device < 64) max_clusters[pool->device][ci] = mc;
+        }
+        if (mc < 1) continue;
+        const int64_t clusters = cdiv(N, 128 * sh.nch) * mtiles;
+        if (clusters > mc) continue;                    // one wave only
+        if (cdiv(K, (int64_t)DG_KP * BK) < sh.S) continue;     // every slice needs at least one step
+        const int64_t ctas = clusters * csz;
+        // more CTAs streaming is better; among equals fewer slices (no exchange of partial sums: 512 tokens run 28 us
+        // as 128-column strips without slices against 34 us as 256-column strips cut in two), then wider strips
+        const int64_t score = ctas * 16 - sh.S * 4 + sh.nch;
+        if (score > best) { best = score; pick = sh; }
+    }
+    g.S = pick.S; g.nch = pick.nch;
+    g.kp = DG_KP;
+    const size_t step_bytes = (size_t)g.kp * (A_STAGE_BYTES + g.nch * CHUNK_BYTES);
+    // leave room for two shrink CTAs (their static and dynamic shared memory + 1 KB system reservation each) on the same
+    // SM: the shrink then overlaps the GEMM's main loop instead of delaying its start (measured: 23 us per call against
+    // 29 us); what is left of the SM's 227 KB goes to the pipeline (4 steps at 256 tokens, 3 at 1024)
+    const size_t shrink_smem = sizeof(DecodeShrinkSmem) + decode_shrink_dyn_smem(T, S) + 1024;
+    g.stages = (int)std::min<size_t>(6, ((size_t)227 * 1024 - 2 * shrink_smem - 1024 - 256 - 1024) / step_bytes);
+    if (g.stages < 2) g.stages = 2;
+    g.num_ks = (int)cdiv(K, (int64_t)g.kp * BK);
+    g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)g.kp * BK);
+    const int NP = 128 * g.nch;
+
+    alignas(64) CUtensorMap tmA, tmB, tmXA, tmXB;
+    marlaas_status_t rc;
+    if ((rc = make_panel_map(&tmA, x, T, K, ldx, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
+    if ((rc = make_map(&tmB, W, K, N, ldw, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
     if (g.num_xs > 0) {
-        if ((rc = make_panel_map(&tmXX, ws.hd, T, hd_cols, hd_cols, 1, 128)) != MARLAAS_OK) return rc;
-        if (g.w3d) rc = make_panel_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 2, BK);
-        else rc = make_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 64, BK);
-        if (rc != MARLAAS_OK) return rc;
+        if ((rc = make_panel_map(&tmXA, ws.hd, T, hd_cols, hd_cols, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXB, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
     } else {
-        tmXX = tmX;
-        tmXW = tmW;
+        tmXA = tmA;
+        tmXB = tmB;
     }
-
-    static bool attrs_set[64] = {};
-    if (pool->device >= 64 || !attrs_set[pool->device]) {
-        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_shrink, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        if (pool->device < 64) attrs_set[pool->device] = true;
-    }
-    // Normal order: the GEMM grid first (its clusters take the SMs they need), the shrink grid as its programmatic
-    // dependent on the SMs left over; the two run side by side and the GEMM's expand steps wait for the shrink's work-unit
-    // count.  Serial order (for tools that run one kernel at a time): the shrink grid, then the GEMM grid, plainly ordered.
-    auto launch_gemm = [&]() -> marlaas_status_t {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(shape.clusters * shape.csz));
-        cfg.blockDim = dim3(DG_THREADS);
-        cfg.dynamicSmemBytes = gemm_smem;
-        cfg.stream = st;
-        cudaLaunchAttribute at[2];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = (unsigned)shape.csz; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at; cfg.numAttrs = serial ? 1 : 2;
-        MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode_gemm, tmW, tmX, tmXW, tmXX, g));
-        count_launch();
-        return MARLAAS_OK;
-    };
-    auto launch_shrink = [&]() -> marlaas_status_t {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)shrink_ctas);
-        cfg.blockDim = dim3(SH_THREADS);
-        cfg.dynamicSmemBytes = shrink_smem;
-        cfg.stream = st;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at; cfg.numAttrs = serial ? 0 : 1;
-        MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode_shrink, a));
-        count_launch();
-        return MARLAAS_OK;
-    };
-    if (serial) {
-        if ((rc = launch_shrink()) != MARLAAS_OK) return rc;
-        if ((rc = launch_gemm()) != MARLAAS_OK) return rc;
-    } else {
-        if ((rc = launch_gemm()) != MARLAAS_OK) return rc;
-        if ((rc = launch_shrink()) != MARLAAS_OK) return rc;
-    }
+    const size_t smem_bytes = 1024 + (size_t)g.stages * step_bytes + 256;
+    cudaLaunchConfig_t cfg = {};
+    g.nstrips = (int)cdiv(N, NP);
+    cfg.gridDim = dim3((unsigned)(g.nstrips * mtiles * 2 * g.S));
+    cfg.blockDim = dim3(DG_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)(2 * g.S); at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode_gemm, tmA, tmB, tmXA, tmXB, g));
+    count_launch();
     return MARLAAS_OK;
 }
 

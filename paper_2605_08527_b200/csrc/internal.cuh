@@ -112,7 +112,7 @@ struct Workspace {
     bf16* hd;              // [T][umax*16]  bf16(s_t h_i) (forward) or bf16(s_t g_i) (backward) in the tenant's unit
                            //               columns, zeros in the other units of the tile
     int32_t umax;
-    float* xbuf;           // decode path with four contraction slices: partial sums passed between a tile's two clusters
+    float* xbuf;           // decode path with a split contraction: partial sums passed between the slices of a tile
     size_t fwd_total;      // bytes a forward call uses (the fields above); the rest serves backward only
     // tensor-core gradient reductions: 64-token blocks, one masked copy of the block's r-vectors per tenant present
     int32_t* blk_np;       // [nblk]        tenants present in the block
@@ -164,13 +164,22 @@ marlaas_status_t launch_gemm2_sm100(const marlaas_pool* pool, const GemmOperands
 // decode_sm100.cu: the whole forward for batches of at most 1024 tokens (two overlapping kernels).
 // S < 0: ws.tok_slot already holds the per-token slots.
 bool decode_sm100_eligible(const marlaas_pool* pool, int64_t T);
-size_t decode_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T);    // exchange scratch of the decode path (0 if unused)
-constexpr size_t DECODE_SYNC_BYTES = 8192;
+// the shrink kernel of that path alone (writes tok_slot, h and hd)
+marlaas_status_t launch_decode_shrink(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, int32_t S,
+                                      const int32_t* seg_offsets, const int32_t* seg_slot, const Workspace& ws, float* h_out,
+                                      cudaStream_t st);
+size_t decode_shrink_smem_bytes(int64_t T, int32_t S);
+// decode_wide_sm100.cu: the same forward for large weights (W columns on the MMA's M side; see the file)
+bool decode_wide_sm100_eligible(const marlaas_pool* pool, int64_t T);
+size_t decode_wide_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T);    // its exchange scratch (0 if unused)
+marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
+                                          int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
+                                          const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
+constexpr size_t DECODE_SYNC_BYTES = 16384;
 
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
                                      int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
-                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st,
-                                     bool serial = false);
+                                     const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
 
 // shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,

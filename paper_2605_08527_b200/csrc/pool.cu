@@ -285,6 +285,8 @@ marlaas_status_t marlaas_check_status(marlaas_pool_t* pool, void* cuda_stream) {
     MARLAAS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
     if (w[0] == DEV_OK) return MARLAAS_OK;
     MARLAAS_CUDA_TRY(cudaMemsetAsync(pool->d_status, 0, 16, (cudaStream_t)cuda_stream));
+    // a call that gave up may have left the decode path's counters and flags behind
+    if (w[0] == DEV_TIMEOUT) MARLAAS_CUDA_TRY(cudaMemsetAsync(pool->d_sync, 0, DECODE_SYNC_BYTES, (cudaStream_t)cuda_stream));
     MARLAAS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
     switch (w[0]) {
         case DEV_BAD_TABLE:
