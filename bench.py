@@ -33,12 +33,29 @@ from paper_2605_08527_b200 import workloads as wl  # noqa: E402
 METRIC = "multi-LoRA layer tokens/s (fwd+bwd)"
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed ncu captures
-# (profiles/); None where the kernel has changed since its counters were taken.
-TRAFFIC = {
-    "cfg3": 1.49e9,    # k_gemm2_sm100, mean of the forward (0.94 GB) and dx (2.04 GB) launches: profiles/gemm2_sm100_cfg3_ncu_full.txt
-    "cfg2": 46.5e6,    # k_decode_shrink (6.3 MB) + k_decode_gemm (40.2 MB) of one call: profiles/decode_cfg2_ncu_full.txt
-}
+
+
+def profile_traffic(workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the workload's dominant kernel, from the committed ncu
+    summaries under profiles/ (a line `bench-traffic <workload> <bytes per launch> <source file> <sha256[:16] of that
+    file when the counters were taken>`).  None, with the reason, when no capture exists or the kernel's source has
+    changed since."""
+    import glob
+    import hashlib
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.txt"))):
+        for line in open(path):
+            f = line.split()
+            if len(f) >= 5 and f[0] == "bench-traffic" and f[1] == workload:
+                src = os.path.join(ROOT, f[3])
+                if not os.path.exists(src):
+                    return None, f"{os.path.basename(path)}: {f[3]} no longer exists"
+                sha = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+                if sha != f[4]:
+                    return None, f"{os.path.basename(path)}: {f[3]} has changed since the counters were taken"
+                return float(f[2]), os.path.basename(path)
+    return None, "no ncu capture of this workload under profiles/"
+
+
 CFG_OF = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
 CFG_DESC = {
     "cfg1": "tiny: W 512x512, 4 tenants r=8, 256 tokens, fwd+bwd",
@@ -59,6 +76,8 @@ SWEEPS = {
 def workload_desc(name):
     if name in CFG_DESC:
         return CFG_DESC[name]
+    if name in wl.VARIANTS:
+        return wl.VARIANTS[name]
     kind, T, n = name.split("-")
     if kind in ("qkv", "qkvsep", "gateup", "gateupsep"):
         shape = "q, k, v (4096x4096 each)" if kind.startswith("qkv") else "gate, up (4096x11008 each)"
@@ -357,7 +376,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg3",
                     help="cfg1 .. cfg5, a forward-only sweep point decode-T-n / prefill-T-n (T tokens, n tenants), or adamw-n "
@@ -372,6 +391,9 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra MARLAAS_FLAG_* bits for every call (diagnostics)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches even for forward-only workloads")
     ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
+    ap.add_argument("--headline-only", action="store_true", help="default workload without the `configs` entries of the other workloads")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the sustained leg of the default run (steps issued back to back for this long)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
     if args.workload.startswith("adamw-") and args.workload[6:].isdigit():
@@ -404,7 +426,55 @@ def main():
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
 
+    ctx = {"torch": torch, "B": B, "dist": dist, "dev": dev, "rank": rank, "local_rank": local_rank, "world": world}
     w = wl.make_named_workload(args.workload)
+    full = args.workload == "cfg3" and world == 1 and not args.headline_only
+    out = measure(ctx, args, w, args.workload, args.steps, args.warmup, args.repeats, args.e2e_steps, not args.no_cpu_baseline,
+                  sustained_s=args.sustained_seconds if full else 0.0)
+    if full and rank == 0:
+        # The metric names forward and forward+backward tokens/s and the fraction of the tensor / HBM roofline: the
+        # headline above is the training-shaped configuration; the other configured workloads (and the variants that
+        # show how much the segment table matters) follow in `configs`, each measured by the same code with fewer steps.
+        configs = {}
+
+        def extra(name, wk, steps=10, repeats=3):
+            t0 = time.time()
+            d = measure(ctx, args, wk, name, steps, 3, repeats, 0, False)
+            configs[name] = summarize(d, time.time() - t0)
+
+        extra("cfg3-fwd", wl.make_variant("cfg3-fwd", w))
+        extra("cfg3-alltenants", wl.make_variant("cfg3-alltenants", w))
+        del w
+        extra("cfg2", wl.make_named_workload("cfg2"), steps=50, repeats=5)
+        extra("cfg4", wl.make_named_workload("cfg4"))
+        w5 = wl.make_named_workload("cfg5")
+        extra("cfg5", w5)
+        extra("cfg5-alltenants", wl.make_variant("cfg5-alltenants", w5))
+        extra("cfg5-decode", wl.make_variant("cfg5-decode", w5), steps=20, repeats=5)
+        out["configs"] = configs
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def summarize(d, seconds):
+    """The figures of one extra workload that the one-line report carries."""
+    r = d["roofline"]
+    keep = {"metric": d["metric"], "tokens_per_s": d["value"], "ms_per_step": d["ms_per_step"], "ms_per_step_min": d["ms_per_step_min"],
+            "steps": d["steps"], "timed_as": d["config"]["timed_as"], "segments": d["config"]["segments"],
+            "tenants_present": d["config"]["tenants_present"], "gpu_launches": d["gpu_launches"], "clocks": d["clocks"],
+            "work_per_step": d["work_per_step"], "wall_s": round(seconds, 1),
+            "roofline": {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "traffic_source", "peak_source", "kernel",
+                                           "whole_step_frac", "whole_step_tflops", "frac_of_nominal_2250", "frac_of_nominal_8TBs",
+                                           "frac_of_measured_sustained", "avg_launch_ms") if k in r}}
+    return keep
+
+
+def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, sustained_s=0.0):
+    """One workload through the layer on this rank's GPU; returns the JSON-line dictionary (rank 0) or None."""
+    torch, B, dist, dev = ctx["torch"], ctx["B"], ctx["dist"], ctx["dev"]
+    rank, local_rank, world = ctx["rank"], ctx["local_rank"], ctx["world"]
     work = algorithmic_work(w)
     ts_np = w.tok_slot()
 
@@ -449,7 +519,8 @@ def main():
             st = {"p": p, "pool": pool, "W": dev_bf16(p.W_bits), "x": x_cache[key], "x_host": pinned[key],
                   "y": torch.empty((w.T, p.d_out), dtype=torch.bfloat16, device=dev),
                   "h": torch.empty((w.T, pool.rank_stride), dtype=torch.float32, device=dev),
-                  "ws": torch.empty(B.marlaas_lora_workspace_bytes(pool, w.T), dtype=torch.uint8, device=dev)}
+                  "ws": None}
+            ws_bytes[0] = max(ws_bytes[0], B.marlaas_lora_workspace_bytes(pool, w.T))
             if Tb:
                 st["dy"] = dev_bf16(p.dy_bits)
                 if id(p.dy_bits) not in pinned:
@@ -461,7 +532,14 @@ def main():
             projs.append(st)
         return projs
 
+    ws_bytes = [0]
     copies = [build_copy() for _ in range(R)]
+    # one workspace for every call of the step loop: it is scratch, the calls are ordered on one stream, and a caller
+    # would not keep one per projection either
+    shared_ws = torch.empty(max(ws_bytes[0], 256), dtype=torch.uint8, device=dev)
+    for c in copies:
+        for st_ in c:
+            st_["ws"] = shared_ws
     projs = copies[0]
     all_projs = [s for c in copies for s in c]
 
@@ -477,7 +555,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, R)):
+    for i in range(max(warmup, R)):
         step(i)
     for s in all_projs:
         B.marlaas_check_status(s["pool"])
@@ -494,7 +572,7 @@ def main():
             with torch.cuda.stream(side):
                 g_ = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g_, stream=side):
-                    for i in range(args.steps):
+                    for i in range(steps):
                         step(i)
             torch.cuda.current_stream().wait_stream(side)
             graph = g_
@@ -506,7 +584,7 @@ def main():
             wb.record()
             barrier()
             # enough replays for the clock sampler to see the GPU under this load (about 0.3 s), at least --repeats
-            args.repeats = int(min(5000, max(args.repeats, 0.3e3 / max(wa.elapsed_time(wb) / 3, 1e-3))))
+            repeats = int(min(5000, max(repeats, 0.3e3 / max(wa.elapsed_time(wb) / 3, 1e-3))))
         except Exception as e:  # noqa: BLE001
             print(f"bench.py: CUDA graph capture failed ({e}); timing direct launches", file=sys.stderr)
             graph = None
@@ -515,14 +593,14 @@ def main():
         if graph is not None:
             graph.replay()
         else:
-            for i in range(args.steps):
+            for i in range(steps):
                 step(i)
 
     # ---- timed region: device-resident inputs ------------------------------------------------------------------
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    reps = max(1, args.repeats)
+    reps = max(1, repeats)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
     barrier()
     n0 = B.marlaas_kernel_launch_count()
@@ -544,7 +622,7 @@ def main():
         rep_ms = [a.elapsed_time(b) for a, b in evs]
     clocks = sampler.stop() if rank == 0 else None
     total_ms = max_over_ranks(float(np.median(rep_ms)), dist, dev)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     tokens_per_step = w.T * world
     value = aggregate_tokens_per_s(w.T, world, ms_per_step)
 
@@ -552,7 +630,7 @@ def main():
     for s in all_projs:
         B.marlaas_kernel_timing_begin(s["pool"])
     n1 = B.marlaas_kernel_launch_count()
-    for i in range(args.steps):
+    for i in range(steps):
         step(i)
     launches_direct = B.marlaas_kernel_launch_count() - n1
     if launches is None:
@@ -563,6 +641,7 @@ def main():
         gemm_ms += ms
         gemm_n += n
     peaks, peak_src = measured_peaks()
+    traffic, traffic_src = profile_traffic(wname)
     gemm_flops_per_step = float(sum(work["gemm_flops"]))
     avg_launch_ms = gemm_ms / max(gemm_n, 1)
     flops_per_launch = gemm_flops_per_step / max(len(work["gemm_flops"]), 1)
@@ -572,33 +651,57 @@ def main():
     if hbm_bound:
         ach = work["fwd_bytes"] / (ms_per_step * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"], "traffic": TRAFFIC.get(args.workload), "peak_source": f"of {peak_src}",
-                    "kernel": "whole forward call: k_decode_shrink and k_decode_gemm (base GEMM + expand), overlapped; "
+                    "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "traffic_source": traffic_src, "peak_source": f"of {peak_src}",
+                    "kernel": "whole forward call: k_decode_shrink and the decode GEMM (base product + expand), overlapped; "
                               "bytes = W + x + y + present adapters, each once",
                     "bytes_per_launch": work["fwd_bytes"], "avg_launch_ms": ms_per_step,
                     "direct_launch_event_ms": avg_launch_ms,
                     "frac_of_nominal_8TBs": ach / NOMINAL["hbm_gbs"]}
     else:
         ach = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12 if gemm_n else 0.0
-        # The GEMM launches are timed inside the step loop.  When that loop ran power-capped (SM clock well under its
-        # maximum with sw_power_cap active) the matching denominator is the sustained cuBLAS figure, otherwise the burst one.
-        capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and "sw_power_cap" in clocks.get("reasons", [])
-                      and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
-        peak_t = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+        # One denominator: the measured burst figure (the GEMM launches are timed one by one with events, inside a loop of
+        # tens of milliseconds).  The sustained and nominal figures are reported beside it, never substituted for it.
+        peak_t = peaks["bf16_tflops"]
+        whole = (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": ach, "peak": peak_t, "unit": "TFLOP/s",
-                    "frac": ach / peak_t, "traffic": TRAFFIC.get(args.workload),
-                    "peak_source": f"of {peak_src} ({'sustained: the timed loop ran power-capped' if capped else 'burst'})",
-                    "frac_of_measured_burst": ach / peaks["bf16_tflops"],
+                    "frac": ach / peak_t, "traffic": traffic, "traffic_source": traffic_src,
+                    "peak_source": f"of {peak_src} (burst)",
                     "kernel": "base GEMM with fused LoRA expand (forward y and backward dx launches)" if Tb else "base GEMM with fused LoRA expand (forward launches)",
                     "launches_timed": gemm_n, "avg_launch_ms": avg_launch_ms, "flops_per_launch": flops_per_launch,
                     "frac_of_nominal_2250": ach / NOMINAL["bf16_tflops"],
                     "frac_of_measured_sustained": ach / peaks["bf16_tflops_sustained"],
-                    "whole_step_tflops": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12,
-                    "whole_step_frac": (work["fwd_flops"] + work["bwd_flops"]) / (ms_per_step * 1e-3) / 1e12 / peak_t}
+                    "whole_step_tflops": whole, "whole_step_frac": whole / peak_t,
+                    "whole_step_frac_of_nominal_2250": whole / NOMINAL["bf16_tflops"]}
+
+    # ---- sustained leg: the same steps issued back to back for seconds, clocks sampled throughout -------------------
+    sustained = None
+    if sustained_s > 0 and rank == 0:
+        n_sus = int(max(steps, sustained_s * 1e3 / max(ms_per_step, 1e-3)))
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a_.record()
+        for i in range(n_sus):
+            step(i)
+        b_.record()
+        torch.cuda.synchronize()
+        clk2 = sampler2.stop()
+        sus_ms = a_.elapsed_time(b_) / n_sus
+        whole_s = (work["fwd_flops"] + work["bwd_flops"]) / (sus_ms * 1e-3) / 1e12
+        bins = {}
+        for smp in sampler2.samples:
+            k = int(round(smp[0] / 100.0) * 100)
+            bins[k] = bins.get(k, 0) + 1
+        sustained = {"steps": n_sus, "seconds": a_.elapsed_time(b_) / 1e3, "ms_per_step": sus_ms, "tokens_per_s": w.T / (sus_ms * 1e-3),
+                     "whole_step_tflops": whole_s, "whole_step_frac_of_measured_sustained": whole_s / peaks["bf16_tflops_sustained"],
+                     "whole_step_frac_of_measured_burst": whole_s / peaks["bf16_tflops"], "clocks": clk2,
+                     "sm_mhz_histogram_100mhz_bins": {str(k): v for k, v in sorted(bins.items())},
+                     "ms_per_step_times_median_sm_ghz": sus_ms * (clk2.get("sm_mhz") or 0) / 1e3}
 
     # ---- end to end: host inputs -> device -> layer -> host outputs, all inside the timed region ------------
     e2e = None
-    if args.e2e_steps > 0:
+    if e2e_steps > 0:
         host_out = []
         for s in projs:
             o = {"y": torch.empty((w.T, s["p"].d_out), dtype=torch.bfloat16).pin_memory()}
@@ -640,46 +743,51 @@ def main():
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for _ in range(args.e2e_steps):
+        for _ in range(e2e_steps):
             h2d, d2h = e2e_step()
         b.record()
         barrier()
         e_ms = max_over_ranks(a.elapsed_time(b), dist, dev)
-        e2e = {"value": tokens_per_step / (e_ms / args.e2e_steps * 1e-3), "unit": "tokens/s",
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": args.e2e_steps,
-               "ms_per_step": e_ms / args.e2e_steps}
+        e2e = {"value": tokens_per_step / (e_ms / e2e_steps * 1e-3), "unit": "tokens/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+               "ms_per_step": e_ms / e2e_steps}
 
     for s in all_projs:
         B.marlaas_check_status(s["pool"])
 
     # ---- the oracle on the host cores, bounded sample (rank 0, single-GPU runs only) ------------------------
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and want_cpu:
         import oracle
         n_tok = min(w.T, args.cpu_baseline_tokens)
         sec = oracle_step_sample(w, n_tok)
         cpu_baseline = {"value": n_tok / sec, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-                        "sample": f"first {n_tok} of {w.T} tokens of {args.workload}, all projections, one timed execution "
+                        "sample": f"first {n_tok} of {w.T} tokens of {wname}, all projections, one timed execution "
                                   f"({sec:.1f} s)"}
 
+    out = None
     if rank == 0:
         out = {
             "metric": METRIC if Tb else "multi-LoRA layer tokens/s (fwd)", "value": value, "unit": "tokens/s",
-            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "desc": workload_desc(args.workload), "tokens_per_step_per_gpu": w.T,
-                       "backward_tokens": Tb, "segments": int(len(w.seg_slot)), "l2": l2_note,
+            "config": {"workload": wname, "desc": workload_desc(wname), "tokens_per_step_per_gpu": w.T,
+                       "backward_tokens": Tb, "segments": int(len(w.seg_slot)),
+                       "tenants_present": int(len(set(int(v) for v in ts_np.tolist() if v >= 0))), "l2": l2_note,
                        "timed_as": "one CUDA graph of K steps, median of %d replays" % reps if graph is not None else "K direct steps",
                        "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "sustained": sustained, "gpu_launches": int(launches),
             "clocks": clocks,
             "work_per_step": {"fwd_gflop": work["fwd_flops"] / 1e9, "bwd_gflop": work["bwd_flops"] / 1e9,
                               "fwd_mb": work["fwd_bytes"] / 1e6, "bwd_mb": work["bwd_bytes"] / 1e6},
-            "ms_per_step_min": float(min(rep_ms)) / args.steps,
+            "ms_per_step_min": float(min(rep_ms)) / steps,
         }
-        print(json.dumps(out))
-    if dist is not None:
-        dist.destroy_process_group()
+    for c in copies:
+        for st_ in c:
+            st_.clear()
+    del copies, projs, all_projs
+    torch.cuda.empty_cache()
+    return out if rank == 0 else None
 
 
 if __name__ == "__main__":

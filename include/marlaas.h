@@ -60,7 +60,8 @@ enum {
 enum {
     MARLAAS_FLAG_ACCUMULATE = 1u,     /* backward: dA_t, dB_t += instead of overwrite */
     MARLAAS_FLAG_HOST_TABLE = 2u,     /* seg_offsets / seg_slot are HOST arrays: validated on the host, then copied
-                                         into the workspace in stream order */
+                                         into the workspace in stream order (not while the stream is being captured:
+                                         refused with MARLAAS_ERR_INVALID_ARG) */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
     MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
 };
@@ -183,8 +184,10 @@ marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T,
  * segments.  h_saved: what forward wrote to h_save for the same batch and adapters, or NULL = recompute.
  * Part of the work (the adapter-gradient kernels, when h_saved is given) may be issued on a stream that the pool
  * owns, forked from cuda_stream after the call's first kernels and joined to it before the call returns (events;
- * legal inside a stream capture): everything the call writes is ordered on cuda_stream as if issued there.  Calls
- * on one pool are not to be issued from several host threads at once. */
+ * legal inside a stream capture): everything the call writes is ordered on cuda_stream as if issued there.  Inside a
+ * stream capture, pools of more than 64 slots copy dA_slots / dB_slots with a memcpy node that keeps the HOST pointers:
+ * the caller's tables must then stay alive and unchanged for every replay.  Calls on one pool are not to be issued from
+ * several host threads at once. */
 marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx,
                                        const void* W, int64_t ldw, const void* dy, int64_t lddy,
                                        void* dx, int64_t lddx, float* const* dA_slots, float* const* dB_slots,
@@ -203,6 +206,13 @@ marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const
 /* Synchronise `cuda_stream`, read and clear the pool's device status word: MARLAAS_OK, or the first
  * device-side finding since the last check (BAD_SEGMENT_TABLE, DEVICE_BAD_INDEX, DEVICE_TIMEOUT). */
 marlaas_status_t marlaas_check_status(marlaas_pool_t* pool, void* cuda_stream);
+
+/* Diagnostic (no counterpart in the paper): every wait inside the tensor-core kernels is bounded, and a wait that runs
+ * out makes its kernel drain and return with MARLAAS_ERR_DEVICE_TIMEOUT recorded in the pool's status word.  This call
+ * exercises exactly that path without starving a real kernel: one small CTA waits, with the kernels' own wait routine,
+ * on a barrier that nobody arrives on, gives up after limit_ns (at most 100 ms) and returns normally.  The next
+ * marlaas_check_status on the pool then returns MARLAAS_ERR_DEVICE_TIMEOUT (and clears it); the pool stays usable. */
+marlaas_status_t marlaas_debug_wait_runs_out(marlaas_pool_t* pool, uint64_t limit_ns, void* cuda_stream);
 
 /* Message for the last non-OK status returned on the calling thread ("" if none). */
 const char* marlaas_last_error(void);

@@ -36,7 +36,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",
     "marlaas_adapter_pool_register", "marlaas_adapter_pool_unregister", "marlaas_adapter_pool_lookup",
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
-    "marlaas_lora_forward_workspace_bytes",
+    "marlaas_lora_forward_workspace_bytes", "marlaas_debug_wait_runs_out",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
     "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
@@ -108,6 +108,8 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_lora_build_index.argtypes = [vp, i64, P(marlaas_segments_t), vp, vp, vp, vp, vp, sz, u32, vp]
     L.marlaas_check_status.restype = i32
     L.marlaas_check_status.argtypes = [vp, vp]
+    L.marlaas_debug_wait_runs_out.restype = i32
+    L.marlaas_debug_wait_runs_out.argtypes = [vp, ctypes.c_uint64, vp]
     L.marlaas_kernel_timing_begin.restype = i32
     L.marlaas_kernel_timing_begin.argtypes = [vp]
     L.marlaas_kernel_timing_end.restype = i32
@@ -351,6 +353,11 @@ def marlaas_lora_build_index(pool: AdapterPool, T: int, seg: Segments, workspace
 
 def marlaas_check_status(pool: AdapterPool, stream=None) -> None:
     _check(load_library().marlaas_check_status(pool.handle, _stream(stream)))
+
+
+def marlaas_debug_wait_runs_out(pool: AdapterPool, limit_ns: int = 1_000_000, stream=None) -> None:
+    """Diagnostic: one small CTA lets a bounded wait run out; the next marlaas_check_status raises DEVICE_TIMEOUT."""
+    _check(load_library().marlaas_debug_wait_runs_out(pool.handle, int(limit_ns), _stream(stream)))
 
 
 def marlaas_kernel_timing_begin(pool: AdapterPool) -> None:

@@ -125,6 +125,16 @@ static marlaas_status_t shrink(const marlaas_pool* pool, int64_t T, const bf16* 
     return launch_shrink_hd(pool, T, src, ld, D, store, ws, out, st);
 }
 
+// Host tables are copied from temporaries of the call: a stream capture would keep pointers into them for its replays.
+static marlaas_status_t reject_host_table_in_capture(const char* fn, uint32_t flags, cudaStream_t st) {
+    if (!(flags & MARLAAS_FLAG_HOST_TABLE)) return MARLAAS_OK;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    MARLAAS_CUDA_TRY(cudaStreamIsCapturing(st, &cs));
+    if (cs != cudaStreamCaptureStatusNone)
+        return fail(MARLAAS_ERR_INVALID_ARG, "%s: MARLAAS_FLAG_HOST_TABLE cannot be used while the stream is being captured", fn);
+    return MARLAAS_OK;
+}
+
 static marlaas_status_t finish(marlaas_pool* pool, uint32_t flags, cudaStream_t st) {
     if (flags & MARLAAS_FLAG_VALIDATE_SYNC) return marlaas_check_status(pool, (void*)st);
     return MARLAAS_OK;
@@ -162,6 +172,7 @@ marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
     int32_t* ts = tok_slot ? tok_slot : ws.tok_slot;
     rc = make_tok_slot(pool, T, seg, flags, host_ts, ts, st);
     if (rc != MARLAAS_OK) return rc;
@@ -193,6 +204,7 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.fwd_total);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
 
     float* h = h_save ? h_save : ws.h;
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH) && decode_sm100_eligible(pool, T)) {
@@ -274,6 +286,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.total);
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
     const bool acc = (flags & MARLAAS_FLAG_ACCUMULATE) != 0;
 
     const bool tc_path = !(flags & MARLAAS_FLAG_CUDA_CORE_PATH);
@@ -337,18 +350,26 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         if (overlap) {
             cudaStream_t gs = pool->side;
             MARLAAS_CUDA_TRY(cudaStreamWaitEvent(gs, pool->ev_fork, 0));
-            if ((rc = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return rc;
-            // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
-            if (want_dB && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
-                                                   gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return rc;
-            if (want_dA && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
-                                                   gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return rc;
-            if (want_dB && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
-                                                   gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return rc;
-            if (want_dA && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
-                                                   gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return rc;
+            // whatever happens from here on, the side stream is joined again before the call returns: a forked stream left
+            // unjoined would invalidate a capture the caller's stream may be part of
+            auto side_work = [&]() -> marlaas_status_t {
+                marlaas_status_t r;
+                if ((r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
+                // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
+                if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
+                                                      gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
+                if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
+                                                      gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
+                if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
+                                                      gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
+                if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
+                                                      gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
+                return MARLAAS_OK;
+            };
+            rc = side_work();
             MARLAAS_CUDA_TRY(cudaEventRecord(pool->ev_join, gs));
             MARLAAS_CUDA_TRY(cudaStreamWaitEvent(st, pool->ev_join, 0));
+            if (rc != MARLAAS_OK) return rc;
             return finish(pool, flags, st);
         }
         if (tc_grad && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;

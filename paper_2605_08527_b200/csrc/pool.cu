@@ -6,9 +6,30 @@
 
 #include <new>
 
-#include "internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace marlaas {
+
+// One CTA waits, with the tensor-core kernels' own bounded wait, on a barrier that nobody arrives on, gives up after
+// limit_ns and reports it the way those kernels do (abort word -> status word); then it returns normally.
+__global__ void k_wait_runs_out(int32_t* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_word;
+    const uint32_t b = sm100::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(b, 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = sm100::mbar_wait_limit(b, 0, &abort_word, 99, limit_ns);
+    __syncthreads();
+    // every other thread sees the abort word, as the other roles of a kernel would, and leaves
+    if (threadIdx.x == 0 && !ok && abort_word != 0) {
+        if (atomicCAS(status, 0, DEV_TIMEOUT) == 0) status[1] = abort_word * 1000000 + (int)blockIdx.x;
+    }
+}
 
 static thread_local char g_err[512] = "";
 static std::atomic<uint64_t> g_launches{0};
@@ -274,6 +295,16 @@ marlaas_status_t marlaas_adapter_pool_export(marlaas_pool_t* pool, int32_t slot,
     k_export<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(pool->d_At, pool->d_Bs, (bf16*)A_out, (bf16*)B_out, slot, r,
                                                             pool->RP, pool->K, pool->N);
     MARLAAS_LAUNCH_CHECK("k_export");
+    return MARLAAS_OK;
+}
+
+marlaas_status_t marlaas_debug_wait_runs_out(marlaas_pool_t* pool, uint64_t limit_ns, void* cuda_stream) {
+    if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "debug_wait_runs_out: pool is NULL");
+    if (limit_ns == 0 || limit_ns > 100ull * 1000 * 1000)
+        return fail(MARLAAS_ERR_INVALID_ARG, "debug_wait_runs_out: limit must be in (0, 100 ms]");
+    MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
+    k_wait_runs_out<<<1, 64, 0, (cudaStream_t)cuda_stream>>>(pool->d_status, (unsigned long long)limit_ns);
+    MARLAAS_LAUNCH_CHECK("k_wait_runs_out");
     return MARLAAS_OK;
 }
 

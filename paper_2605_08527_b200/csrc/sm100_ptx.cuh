@@ -44,9 +44,10 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after WAIT_LIMIT_NS or as soon as another role of this CTA has given up; the first to
-// give up records its site in the CTA's abort word.  Returns false on abort.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int site) {
+// Bounded wait: gives up after limit_ns or as soon as another role of this CTA has given up; the first to give up
+// records its site in the CTA's abort word.  Returns false on abort.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_word, int site,
+                                                unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;      // the global timer is slow to read: sampled every 256 polls only
     uint32_t spins = 0;
@@ -56,12 +57,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_word != 0) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
+            else if (now - t0 > limit_ns) {
                 atomicCAS((int*)abort_word, 0, site);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int site) {
+    return mbar_wait_limit(bar, parity, abort_word, site, WAIT_LIMIT_NS);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {

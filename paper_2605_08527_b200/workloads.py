@@ -345,6 +345,61 @@ def fuse_projections(w: Workload, names: Optional[List[str]] = None) -> Workload
 
 SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|gateup|gateupsep)-(\d+)-(\d+)$"
 
+# Variants of the configured workloads (same tensors, another pass or another table):
+VARIANTS = {
+    "cfg3-fwd": "cfg3, forward only",
+    "cfg3-alltenants": "cfg3 with a table of the same recipe in which all 10 tenants appear (13 to 16 segments)",
+    "cfg5-decode": "the decode part of cfg5 alone: its 256 decode tokens through the 7 projections, forward only",
+    "cfg5-alltenants": "cfg5 whose 4096 training rows hold all 32 tenants (same recipe, lengths divided by 8)",
+}
+
+
+def _table_with_all_tenants(seed: int, T: int, n: int, shrink: int, lo: int, hi: int):
+    """First table of the lognormal recipe (sub-stream 1, 2, ...) with lo..hi segments in which every tenant appears."""
+    for sub in range(1, 200):
+        off, sl = lognormal_segments(seed, T, n, sub=sub, shrink=shrink)
+        if lo <= len(sl) <= hi and len(set(sl.tolist())) == n:
+            return off, sl
+    raise RuntimeError("no table with every tenant present in the first 200 sub-streams")
+
+
+def make_variant(name: str, base: Optional[Workload] = None) -> Workload:
+    """See VARIANTS.  ``base`` may pass the already generated cfg3 / cfg5 workload (generation is the slow part); its
+    tensors are shared, not copied."""
+    if name not in VARIANTS:
+        raise ValueError(f"unknown variant {name!r}")
+    cfg = int(name[3])
+    w = base if base is not None else make_workload(cfg)
+    if name == "cfg3-fwd":
+        projs = [dataclasses.replace(p, dy_bits=None) for p in w.projections]
+        return Workload(name, w.T, 0, w.seg_offsets, w.seg_slot, projs, w.n_tenants, w.max_rank)
+    if name == "cfg3-alltenants":
+        off, sl = _table_with_all_tenants(BASE_SEED + 3, w.T, w.n_tenants, 1, 13, 16)
+        return Workload(name, w.T, w.T_bwd, off, sl, w.projections, w.n_tenants, w.max_rank)
+    if name == "cfg5-decode":
+        Tt = w.T_bwd
+        keep = [s for s in range(len(w.seg_slot)) if w.seg_offsets[s] >= Tt]
+        off = np.array([int(w.seg_offsets[s]) - Tt for s in keep] + [w.T - Tt], dtype=np.int32)
+        projs = [dataclasses.replace(p, x_bits=np.ascontiguousarray(p.x_bits[Tt:]), dy_bits=None) for p in w.projections]
+        # projections that shared their input keep sharing it
+        first = {}
+        for p, p0 in zip(projs, w.projections):
+            key = id(p0.x_bits)
+            if key in first:
+                p.x_bits = first[key]
+            else:
+                first[key] = p.x_bits
+        return Workload(name, w.T - Tt, 0, off, w.seg_slot[keep].astype(np.int32), projs, w.n_tenants, w.max_rank)
+    if name == "cfg5-alltenants":
+        Tt = w.T_bwd
+        o1, s1 = _table_with_all_tenants(BASE_SEED + 5, Tt, w.n_tenants, 8, 32, 64)
+        keep = [s for s in range(len(w.seg_slot)) if w.seg_offsets[s] >= Tt]
+        o2 = np.array([int(w.seg_offsets[s]) for s in keep] + [w.T], dtype=np.int32)
+        off = np.concatenate([o1[:-1], o2]).astype(np.int32)
+        sl = np.concatenate([s1, w.seg_slot[keep]]).astype(np.int32)
+        return Workload(name, w.T, w.T_bwd, off, sl, w.projections, w.n_tenants, w.max_rank)
+    raise ValueError(name)
+
 
 def make_named_workload(name: str) -> Workload:
     """``cfgN`` gives make_workload(N).  Two forward-only families for sweeps over the rollout phases, both on a
@@ -358,6 +413,8 @@ def make_named_workload(name: str) -> Workload:
     import re
     if name.startswith("cfg") and name[3:].isdigit():
         return make_workload(int(name[3:]))
+    if name in VARIANTS:
+        return make_variant(name)
     m = re.match(SWEEP_NAME, name)
     if not m:
         raise ValueError(f"unknown workload {name!r}")

@@ -382,3 +382,22 @@ def test_backward_inside_a_stream_capture_replays_to_the_same_bits():
             if a is not None:
                 assert torch.equal(a, b)
     B.marlaas_check_status(dc.pool)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_pool_stays_usable():
+    # A bounded wait inside a kernel gives up after its limit, the kernel returns normally and the status word says
+    # DEVICE_TIMEOUT.  No product kernel is starved for this: a diagnostic CTA waits 1 ms on a barrier nobody arrives on.
+    w = wl.make_workload(1)
+    p = w.projections[0]
+    dc, ref = _check_case(w, p)
+    B.marlaas_debug_wait_runs_out(dc.pool, limit_ns=1_000_000)
+    with pytest.raises(B.MarlaasError) as e:
+        B.marlaas_check_status(dc.pool)
+    assert e.value.status == B.MARLAAS_ERR_DEVICE_TIMEOUT
+    assert "site 99" in str(e.value)
+    B.marlaas_check_status(dc.pool)                      # the finding was cleared by the read
+    y = dc.forward()                                     # and the pool computes as before
+    assert_close(to_np(y), ref["y"], "forward after a reported timeout")
+    B.marlaas_check_status(dc.pool)
+    with pytest.raises(B.MarlaasError):
+        B.marlaas_debug_wait_runs_out(dc.pool, limit_ns=10**12)      # limits beyond 100 ms are refused on the host
