@@ -391,6 +391,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra MARLAAS_FLAG_* bits for every call (diagnostics)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches even for forward-only workloads")
     ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
+    ap.add_argument("--multi", action="store_true",
+                    help="forward-only multi-projection workloads: q,k,v and gate,up through marlaas_lora_forward_multi (measured: no faster)")
     ap.add_argument("--headline-only", action="store_true", help="default workload without the `configs` entries of the other workloads")
     ap.add_argument("--sustained-seconds", type=float, default=2.0,
                     help="length of the sustained leg of the default run (steps issued back to back for this long)")
@@ -543,12 +545,43 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
     projs = copies[0]
     all_projs = [s for c in copies for s in c]
 
+    # A step is all forwards of the layer's projections, then all backwards (as a training step runs them).  The
+    # projections see the same mixed batch, so the second and later calls of each pass reuse the plan the first one
+    # left in the shared workspace (MARLAAS_FLAG_REUSE_PLAN): the plan is built once per pass, not once per projection.
+    # Forward-only steps over several projections (a decode step of a decoder layer): the projections that read the same
+    # activations -- q, k, v and gate, up -- do not depend on one another and go through ONE marlaas_lora_forward_multi
+    # call each, which may run them side by side; o and down stay calls of their own (in a model they wait for attention
+    # and for the activation function).  Concurrent calls need a workspace each.
+    GROUPS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
+    use_multi = (not Tb) and len(w.projections) > 1 and args.multi
+    if use_multi:
+        for c in copies:
+            for st_ in c:
+                st_["ws"] = torch.empty(max(B.marlaas_lora_forward_workspace_bytes(st_["pool"], w.T), 256), dtype=torch.uint8, device=dev)
+
     def step(i=0, x_of=lambda s: s["x"], dy_of=lambda s: s["dy"]):
-        for s in copies[i % R]:
-            B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=args.flags)
-            if Tb:
+        cs = copies[i % R]
+        if use_multi:
+            by_name = {s["p"].name: s for s in cs}
+            done = set()
+            for grp in GROUPS:
+                members = [by_name[nm] for nm in grp if nm in by_name]
+                if members:
+                    B.marlaas_lora_forward_multi([dict(pool=s["pool"], x=x_of(s), W=s["W"], seg=seg, y=s["y"], h_save=s["h"],
+                                                       workspace=s["ws"]) for s in members], flags=args.flags)
+                    done.update(s["p"].name for s in members)
+            for s in cs:
+                if s["p"].name not in done:
+                    B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=args.flags)
+            return
+        for j, s in enumerate(cs):
+            fl = args.flags | (B.MARLAAS_FLAG_REUSE_PLAN if j > 0 else 0)
+            B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=fl)
+        if Tb:
+            for j, s in enumerate(cs):
+                fl = args.flags | (B.MARLAAS_FLAG_REUSE_PLAN if j > 0 else 0)
                 B.marlaas_lora_backward(s["pool"], x_of(s)[:Tb], s["W"], dy_of(s), seg_b, dx=s["dx"], dA=s["dA"], dB=s["dB"],
-                                        h_saved=s["h"][:Tb], workspace=s["ws"], flags=args.flags)
+                                        h_saved=s["h"][:Tb], workspace=s["ws"], flags=fl)
 
     def barrier():
         if dist is not None:
@@ -775,6 +808,7 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
                        "backward_tokens": Tb, "segments": int(len(w.seg_slot)),
                        "tenants_present": int(len(set(int(v) for v in ts_np.tolist() if v >= 0))), "l2": l2_note,
                        "timed_as": "one CUDA graph of K steps, median of %d replays" % reps if graph is not None else "K direct steps",
+                       "calls": "q,k,v and gate,up through marlaas_lora_forward_multi (independent projections side by side)" if use_multi else "one call per projection and pass",
                        "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "sustained": sustained, "gpu_launches": int(launches),
             "clocks": clocks,

@@ -63,7 +63,14 @@ enum {
                                          into the workspace in stream order (not while the stream is being captured:
                                          refused with MARLAAS_ERR_INVALID_ARG) */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
-    MARLAAS_FLAG_CUDA_CORE_PATH = 8u  /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
+    MARLAAS_FLAG_CUDA_CORE_PATH = 8u, /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
+    MARLAAS_FLAG_REUSE_PLAN = 16u     /* the workspace still holds the plan of the previous call of the same kind
+                                         (forward after forward, backward after backward) and that call had the same T,
+                                         the same segment table contents and a pool of the same capacity and max_rank:
+                                         the per-token slots and per-tile unit lists are not rebuilt.  For the
+                                         projections of one decoder layer, which all see the same mixed batch.  The
+                                         caller vouches for the condition; batches of at most 1024 tokens ignore the
+                                         flag (their plan is built inside the first kernel anyway). */
 };
 
 /* Token-to-adapter segment table of one mixed batch: segment s covers tokens
@@ -150,6 +157,27 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
                                       const void* W, int64_t ldw, void* y, int64_t ldy,
                                       const marlaas_segments_t* seg, float* h_save, void* workspace,
                                       size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/* Several forward calls that do not depend on one another, as one call: the projections of a decoder layer that read
+ * the same activations (q, k, v; gate, up) during rollout, when every adapted projection of the shared base model serves
+ * all tenants' decode tokens at once (paper: Methods, "Multi-LoRA Rollout with Single-Task Training"; Introduction:
+ * rollouts dominate the run time).  Each entry holds the arguments of one marlaas_lora_forward.  The caller states that
+ * no call's output is another's input and that pools, outputs, h_save arrays and workspaces are pairwise distinct; the
+ * library may then run the calls side by side (on streams it owns, forked from cuda_stream and joined to it before the
+ * call returns; events only, so legal inside a stream capture), which lets one projection's epilogue overlap the next
+ * one's pass over its weight.  Everything the call writes is ordered on cuda_stream as if issued there.  All entries are
+ * validated before anything is launched.  MARLAAS_FLAG_VALIDATE_SYNC and MARLAAS_FLAG_REUSE_PLAN are refused. */
+typedef struct {
+    marlaas_pool_t* pool;
+    int64_t T;
+    const void* x; int64_t ldx;
+    const void* W; int64_t ldw;
+    void* y; int64_t ldy;
+    const marlaas_segments_t* seg;
+    float* h_save;
+    void* workspace; size_t workspace_bytes;
+} marlaas_forward_call_t;
+marlaas_status_t marlaas_lora_forward_multi(int32_t n, const marlaas_forward_call_t* calls, uint32_t flags, void* cuda_stream);
 
 /* The same forward pass for callers that cannot allocate device memory (no counterpart in the paper: an
  * addition for deployments, not part of the method).  Some hosts of this layer may not call cudaMalloc at all:

@@ -31,12 +31,13 @@ MARLAAS_FLAG_ACCUMULATE = 1
 MARLAAS_FLAG_HOST_TABLE = 2
 MARLAAS_FLAG_VALIDATE_SYNC = 4
 MARLAAS_FLAG_CUDA_CORE_PATH = 8
+MARLAAS_FLAG_REUSE_PLAN = 16
 
 EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",
     "marlaas_adapter_pool_register", "marlaas_adapter_pool_unregister", "marlaas_adapter_pool_lookup",
     "marlaas_adapter_pool_export", "marlaas_adapter_pool_rank_stride", "marlaas_lora_workspace_bytes",
-    "marlaas_lora_forward_workspace_bytes", "marlaas_debug_wait_runs_out",
+    "marlaas_lora_forward_workspace_bytes", "marlaas_debug_wait_runs_out", "marlaas_lora_forward_multi",
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
     "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
@@ -108,6 +109,8 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_lora_build_index.argtypes = [vp, i64, P(marlaas_segments_t), vp, vp, vp, vp, vp, sz, u32, vp]
     L.marlaas_check_status.restype = i32
     L.marlaas_check_status.argtypes = [vp, vp]
+    L.marlaas_lora_forward_multi.restype = i32
+    L.marlaas_lora_forward_multi.argtypes = [ctypes.c_int32, vp, ctypes.c_uint32, vp]
     L.marlaas_debug_wait_runs_out.restype = i32
     L.marlaas_debug_wait_runs_out.argtypes = [vp, ctypes.c_uint64, vp]
     L.marlaas_kernel_timing_begin.restype = i32
@@ -143,6 +146,13 @@ def marlaas_last_error() -> str:
 
 def marlaas_kernel_launch_count() -> int:
     return int(load_library().marlaas_kernel_launch_count())
+
+
+class marlaas_forward_call_t(ctypes.Structure):
+    _fields_ = [("pool", ctypes.c_void_p), ("T", ctypes.c_int64), ("x", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("W", ctypes.c_void_p), ("ldw", ctypes.c_int64), ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64),
+                ("seg", ctypes.c_void_p), ("h_save", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
 
 
 class Segments:
@@ -287,6 +297,37 @@ def marlaas_lora_forward(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, se
                                                ctypes.byref(seg.c), _dptr(h_save), _dptr(ws), ws.numel(),
                                                flags | seg.flags, _stream(stream)))
     return y
+
+
+def marlaas_lora_forward_multi(calls, flags: int = 0, stream=None):
+    """Independent forward calls as one (see marlaas.h): `calls` is a list of dicts with the keyword arguments of
+    marlaas_lora_forward (pool, x, W, seg, and y / h_save / workspace, which must be distinct per call; missing y and
+    workspace are allocated).  Returns the list of outputs."""
+    n = len(calls)
+    arr = (marlaas_forward_call_t * max(n, 1))()
+    keep, ys = [], []
+    fl = flags
+    for i, c in enumerate(calls):
+        pool, x, W, seg = c["pool"], c["x"], c["W"], c["seg"]
+        T = x.shape[0]
+        y = c.get("y")
+        if y is None:
+            y = torch.empty((T, pool.d_out), dtype=torch.bfloat16, device=x.device)
+        ws = c.get("workspace")
+        if ws is None:
+            ws = torch.empty(max(marlaas_lora_forward_workspace_bytes(pool, T), 256), dtype=torch.uint8, device=x.device)
+        hs = c.get("h_save")
+        if hs is not None:
+            assert hs.dtype == torch.float32 and hs.is_contiguous() and tuple(hs.shape) == (T, pool.rank_stride)
+        assert W.shape[0] == pool.d_in
+        arr[i] = marlaas_forward_call_t(pool.handle, T, _dptr(x), _mat(x, pool.d_in, "x"), _dptr(W), _mat(W, pool.d_out, "W"),
+                                        _dptr(y), _mat(y, pool.d_out, "y"), ctypes.cast(ctypes.byref(seg.c), ctypes.c_void_p),
+                                        _dptr(hs), _dptr(ws), ws.numel())
+        fl |= seg.flags
+        keep.append((ws, hs, seg))
+        ys.append(y)
+    _check(load_library().marlaas_lora_forward_multi(n, ctypes.cast(arr, ctypes.c_void_p), fl, _stream(stream)))
+    return ys
 
 
 def marlaas_lora_static_workspace_limit() -> int:

@@ -1,6 +1,8 @@
 // The exported layer calls: argument validation on the host, then the kernel sequence on the caller's stream.
 #include <string.h>
 
+#include <mutex>
+
 #include "internal.cuh"
 
 namespace marlaas {
@@ -183,11 +185,11 @@ marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const
     return finish(pool, flags, st);
 }
 
-marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
-                                      int64_t ldw, void* y, int64_t ldy, const marlaas_segments_t* seg,
-                                      float* h_save, void* workspace, size_t workspace_bytes, uint32_t flags,
-                                      void* cuda_stream) {
-    const char* fn = "lora_forward";
+// The forward call: validation first (launch = false stops after it), then the kernel sequence on the stream.
+static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
+                                     int64_t ldw, void* y, int64_t ldy, const marlaas_segments_t* seg,
+                                     float* h_save, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                     void* cuda_stream, bool launch, const char* fn) {
     if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
     if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
     if (T == 0) return MARLAAS_OK;
@@ -205,6 +207,7 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
     if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
+    if (!launch) return MARLAAS_OK;
 
     float* h = h_save ? h_save : ws.h;
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH) && decode_sm100_eligible(pool, T)) {
@@ -230,7 +233,7 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
         // programmatic dependent of the one before and overlaps its tail)
         const bool pre_zero = T >= 512 && shrink_split_sm100_eligible(pool, T, pool->K);
         if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(h, 0, sizeof(float) * (size_t)T * pool->RP, st));
-        if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
+        if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
         if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st, pre_zero)) != MARLAAS_OK) return rc;
         GemmOperands o;
         o.M = T; o.Nout = pool->N; o.Kc = pool->K;
@@ -255,6 +258,81 @@ marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const voi
                                         (bf16*)y, ldy, h, pool->d_Bs, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
     return finish(pool, flags, st);
+}
+
+marlaas_status_t marlaas_lora_forward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
+                                      int64_t ldw, void* y, int64_t ldy, const marlaas_segments_t* seg,
+                                      float* h_save, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                      void* cuda_stream) {
+    return forward_impl(pool, T, x, ldx, W, ldw, y, ldy, seg, h_save, workspace, workspace_bytes, flags, cuda_stream, true,
+                        "lora_forward");
+}
+
+marlaas_status_t marlaas_lora_forward_multi(int32_t n, const marlaas_forward_call_t* calls, uint32_t flags, void* cuda_stream) {
+    const char* fn = "lora_forward_multi";
+    if (n < 0 || (n > 0 && !calls)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: bad call list", fn);
+    if (n == 0) return MARLAAS_OK;
+    if (flags & (MARLAAS_FLAG_VALIDATE_SYNC | MARLAAS_FLAG_REUSE_PLAN))
+        return fail(MARLAAS_ERR_INVALID_ARG, "%s: VALIDATE_SYNC and REUSE_PLAN do not apply to a set of concurrent calls", fn);
+    marlaas_status_t rc;
+    // every call is validated before anything is launched
+    for (int i = 0; i < n; ++i) {
+        const marlaas_forward_call_t& c = calls[i];
+        if (!c.pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: call %d has no pool", fn, i);
+        if (c.pool->device != calls[0].pool->device) return fail(MARLAAS_ERR_INVALID_ARG, "%s: the calls' pools are on different devices", fn);
+        if ((rc = forward_impl(c.pool, c.T, c.x, c.ldx, c.W, c.ldw, c.y, c.ldy, c.seg, c.h_save, c.workspace, c.workspace_bytes, flags,
+                               cuda_stream, false, fn)) != MARLAAS_OK) return rc;
+        for (int j = 0; j < i; ++j) {
+            const marlaas_forward_call_t& d = calls[j];
+            if (c.pool == d.pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: calls %d and %d use the same pool", fn, j, i);
+            const char *a0 = (const char*)c.workspace, *b0 = (const char*)d.workspace;
+            if (c.T > 0 && d.T > 0 && a0 < b0 + d.workspace_bytes && b0 < a0 + c.workspace_bytes)
+                return fail(MARLAAS_ERR_INVALID_ARG, "%s: calls %d and %d share workspace memory", fn, j, i);
+        }
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int dev = calls[0].pool->device;
+    MARLAAS_CUDA_TRY(cudaSetDevice(dev));
+    if (n == 1 || dev < 0 || dev >= 64) {
+        for (int i = 0; i < n; ++i) {
+            const marlaas_forward_call_t& c = calls[i];
+            if ((rc = forward_impl(c.pool, c.T, c.x, c.ldx, c.W, c.ldw, c.y, c.ldy, c.seg, c.h_save, c.workspace, c.workspace_bytes, flags,
+                                   cuda_stream, true, fn)) != MARLAAS_OK) return rc;
+        }
+        return MARLAAS_OK;
+    }
+    // Fork: call 0 stays on the caller's stream, the others go to side streams of the device (created on first use, never
+    // destroyed), round robin; join: the caller's stream waits for every side stream.  Events only: legal inside a capture.
+    constexpr int NSIDE = 3;
+    static std::mutex mu;
+    static cudaStream_t side[64][NSIDE] = {};
+    static cudaEvent_t ev_fork[64] = {}, ev_join[64][NSIDE] = {};
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!ev_fork[dev]) {
+            for (int k = 0; k < NSIDE; ++k) {
+                MARLAAS_CUDA_TRY(cudaStreamCreateWithFlags(&side[dev][k], cudaStreamNonBlocking));
+                MARLAAS_CUDA_TRY(cudaEventCreateWithFlags(&ev_join[dev][k], cudaEventDisableTiming));
+            }
+            MARLAAS_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork[dev], cudaEventDisableTiming));
+        }
+    }
+    const int used = n - 1 < NSIDE ? n - 1 : NSIDE;
+    MARLAAS_CUDA_TRY(cudaEventRecord(ev_fork[dev], st));
+    for (int k = 0; k < used; ++k) MARLAAS_CUDA_TRY(cudaStreamWaitEvent(side[dev][k], ev_fork[dev], 0));
+    marlaas_status_t first_err = MARLAAS_OK;
+    for (int i = 0; i < n && first_err == MARLAAS_OK; ++i) {
+        const marlaas_forward_call_t& c = calls[i];
+        cudaStream_t cs = i == 0 ? st : side[dev][(i - 1) % NSIDE];
+        first_err = forward_impl(c.pool, c.T, c.x, c.ldx, c.W, c.ldw, c.y, c.ldy, c.seg, c.h_save, c.workspace, c.workspace_bytes, flags,
+                                 (void*)cs, true, fn);
+    }
+    // whatever happened, the side streams are joined again
+    for (int k = 0; k < used; ++k) {
+        MARLAAS_CUDA_TRY(cudaEventRecord(ev_join[dev][k], side[dev][k]));
+        MARLAAS_CUDA_TRY(cudaStreamWaitEvent(st, ev_join[dev][k], 0));
+    }
+    return first_err;
 }
 
 marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const void* x, int64_t ldx, const void* W,
@@ -293,7 +371,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     const bool pre_zero = tc_path && T >= 512 && (dx || want_dA) && shrink_split_sm100_eligible(pool, T, pool->N);
     if (tc_path && T > 0) {
         if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.g, 0, sizeof(float) * (size_t)T * pool->RP, st));   // see forward
-        if ((rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
+        if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
     } else {
         if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
@@ -354,7 +432,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             // unjoined would invalidate a capture the caller's stream may be part of
             auto side_work = [&]() -> marlaas_status_t {
                 marlaas_status_t r;
-                if ((r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
+                if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
                 // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
                 if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
                                                       gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
@@ -372,7 +450,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             if (rc != MARLAAS_OK) return rc;
             return finish(pool, flags, st);
         }
-        if (tc_grad && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
+        if (tc_grad && !(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
         if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
         if (want_dB) {
             const float* h = h_saved;

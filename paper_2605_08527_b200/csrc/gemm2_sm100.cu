@@ -381,6 +381,9 @@ static marlaas_status_t launch_gemm2_t(const marlaas_pool* pool, const GemmOpera
     g.num_n_tiles = (int)cdiv(o.Nout, G2_BN);
     g.num_kb = (int)cdiv(o.Kc, (int64_t)BK * KP);      // pipeline steps
     g.group_m = g.num_m_tiles >= 32 ? 16 : 8;      // row tiles per band (measured: 8-16 best; 32 loses the band's x rows from L2)
+    // A band's rows of A should stay in L2 while the band's column tiles pass over them: with a deep contraction (the dx
+    // launch: 11008) sixteen row tiles are 90 MB and are read again by every wave of the band; eight are 45 MB.
+    while (g.group_m > 4 && (int64_t)g.group_m * 256 * o.Kc * 2 > (int64_t)48 << 20) g.group_m >>= 1;
     g.b_mn = o.b_mn ? 1 : 0;
     g.tile_nunits = o.tile_nunits;
     g.tile_units = o.tile_units;

@@ -72,3 +72,32 @@ def test_fused_projection_equals_the_separate_projections(T, K, Ns, n, rank, per
                     assert_close(got_B[i * rank:(i + 1) * rank, offs[i]:offs[i + 1]], dBs[i][t],
                                  f"dB of tenant {t}, projection {i} (diagonal block)")
     B.marlaas_check_status(dc.pool)
+
+
+def test_independent_projections_as_one_multi_call():
+    # q, k, v shaped: three pools, one decode batch, one call; every output against the oracle of its own projection,
+    # and bit for bit against the three single calls (the same kernels, only on side streams)
+    T, K, Ns, n, rank = 130, 256, (256, 128, 320), 5, 16
+    w = _separate_case(977, T, K, Ns, n, rank, True)
+    ts = w.tok_slot()
+    dcs = [DeviceCase(w, p, capacity=n + 1) for p in w.projections]
+    calls = [dict(pool=dc.pool, x=dc.x, W=dc.W, seg=dc.seg,
+                  h_save=torch.empty((T, dc.pool.rank_stride), dtype=torch.float32, device="cuda:0")) for dc in dcs]
+    ys = B.marlaas_lora_forward_multi(calls)
+    torch.cuda.synchronize()
+    for dc, p, y, c in zip(dcs, w.projections, ys, calls):
+        r, s, A, Bm = oracle.adapters_of(p)
+        ry, rh = oracle.forward(p.x, p.W, r, s, A, Bm, ts)
+        assert_close(to_np(y), ry, f"multi call: y of {p.name}")
+        hs = torch.empty_like(c["h_save"])
+        y1 = dc.forward(h_save=hs)
+        assert torch.equal(y1, y) and torch.equal(hs, c["h_save"])
+        B.marlaas_check_status(dc.pool)
+    # two entries on one pool, or sharing a workspace, are refused before anything is launched
+    n0 = B.marlaas_kernel_launch_count()
+    with pytest.raises(B.MarlaasError):
+        B.marlaas_lora_forward_multi([calls[0], dict(calls[0])])
+    shared = torch.empty(1 << 22, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(B.MarlaasError):
+        B.marlaas_lora_forward_multi([dict(calls[0], workspace=shared), dict(calls[1], workspace=shared)])
+    assert B.marlaas_kernel_launch_count() == n0
