@@ -432,7 +432,12 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             // unjoined would invalidate a capture the caller's stream may be part of
             auto side_work = [&]() -> marlaas_status_t {
                 marlaas_status_t r;
-                if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
+                if (!(flags & MARLAAS_FLAG_REUSE_PLAN)) {
+                    if ((r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
+                } else {
+                    // the plan kernel also zeroes the reductions' work-item counters; a reused plan needs them zeroed again
+                    MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), gs));
+                }
                 // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
                 if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
                                                       gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
@@ -451,6 +456,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             return finish(pool, flags, st);
         }
         if (tc_grad && !(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
+        if (tc_grad && (flags & MARLAAS_FLAG_REUSE_PLAN)) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), st));
         if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
         if (want_dB) {
             const float* h = h_saved;

@@ -101,3 +101,38 @@ def test_independent_projections_as_one_multi_call():
     with pytest.raises(B.MarlaasError):
         B.marlaas_lora_forward_multi([dict(calls[0], workspace=shared), dict(calls[1], workspace=shared)])
     assert B.marlaas_kernel_launch_count() == n0
+
+
+@pytest.mark.parametrize("T,K,Ns,n,rank", [
+    (1300, 128, (256, 128, 192), 5, 16),      # 2-CTA GEMM, tensor-core gradient reductions on the side stream
+    (600, 192, (128, 256), 4, 8),             # 1-CTA GEMM
+])
+def test_a_layers_projections_reuse_the_plan_of_the_first(T, K, Ns, n, rank):
+    # Projections of one layer see the same mixed batch: the first forward (backward) builds the plan in the shared
+    # workspace, the others run with MARLAAS_FLAG_REUSE_PLAN.  Every projection's outputs against its own oracle run.
+    w = _separate_case(1200 + T, T, K, Ns, n, rank, False)
+    ts = w.tok_slot()
+    dcs = [DeviceCase(w, p, capacity=n + 1) for p in w.projections]
+    ws = torch.empty(max(B.marlaas_lora_workspace_bytes(dc.pool, T) for dc in dcs), dtype=torch.uint8, device="cuda:0")
+    hs = [torch.empty((T, dc.pool.rank_stride), dtype=torch.float32, device="cuda:0") for dc in dcs]
+    ys = []
+    for j, dc in enumerate(dcs):
+        ys.append(B.marlaas_lora_forward(dc.pool, dc.x, dc.W, dc.seg, h_save=hs[j], workspace=ws,
+                                         flags=B.MARLAAS_FLAG_REUSE_PLAN if j else 0))
+    outs = []
+    for j, dc in enumerate(dcs):
+        dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda:0")
+        dA, dB = dc.grads(fill=3.0)
+        B.marlaas_lora_backward(dc.pool, dc.x, dc.W, dc.dy, dc.seg, dx=dx, dA=dA, dB=dB, h_saved=hs[j], workspace=ws,
+                                flags=B.MARLAAS_FLAG_REUSE_PLAN if j else 0)
+        outs.append((dx, dA, dB))
+    torch.cuda.synchronize()
+    for j, (dc, p) in enumerate(zip(dcs, w.projections)):
+        r, s, A, Bm = oracle.adapters_of(p)
+        assert_close(to_np(ys[j]), oracle.forward(p.x, p.W, r, s, A, Bm, ts)[0], f"{p.name}: y with a reused plan")
+        assert_close(to_np(outs[j][0]), oracle.backward_dx(p.dy, p.W, r, s, A, Bm, ts)[0], f"{p.name}: dx with a reused plan")
+        rdA, rdB = oracle.backward_dAdB(p.x, p.dy, r, s, A, Bm, ts)
+        for t in range(n):
+            assert_close(to_np(outs[j][1][t]), rdA[t], f"{p.name}: dA[{t}] with a reused plan")
+            assert_close(to_np(outs[j][2][t]), rdB[t], f"{p.name}: dB[{t}] with a reused plan")
+        B.marlaas_check_status(dc.pool)
