@@ -98,6 +98,35 @@ marlaas_status_t marlaas_adapter_pool_create(marlaas_pool_t** out, int device, i
                                              size_t storage_bytes, void* cuda_stream);
 marlaas_status_t marlaas_adapter_pool_destroy(marlaas_pool_t* pool);
 
+/* One pool for several projections that read the same activations (q, k, v; gate, up), served as ONE layer of width
+ * d_out = part_d_out[0] + ... + part_d_out[n_parts-1] whose weight is the projections' weights side by side,
+ * W = [W_1 | ... | W_P] (paper: Methods, "Multi-LoRA Rollout with Single-Task Training" -- every adapted projection of
+ * the shared base model serves all tenants' tokens at once; Introduction -- rollout dominates the run time, so the
+ * decode-shaped pass over the projections of a decoder layer is what one such call shortens).  Tenant t holds one
+ * adapter pair per projection, all of the tenant's rank r_t and scale s_t:
+ *
+ *     y_i[:, columns of projection p] = x_i W_p + s_t (x_i A_t,p) B_t,p
+ *
+ * The store keeps one block of A rows per projection and the B matrices side by side ([r_t][d_out]): nothing is stored
+ * or streamed for the zero blocks that the projections' adapters would have as one block-diagonal adapter of rank P r_t.
+ * 1 <= n_parts <= 4; every part_d_out[p] is a positive multiple of 256.  On such a pool
+ *  - register / export / adamw_commit take A as n_parts blocks [d_in][rank] one after another and B as n_parts blocks
+ *    [rank][part_d_out[p]] one after another (the projections' own matrices, concatenated in memory); the fp32 masters,
+ *    moments and gradients of adamw_commit and the dA_t / dB_t of backward have the same block layout;
+ *  - forward / backward take W with d_out columns (the projections' weights side by side, leading dimension ldw),
+ *    y / dy with d_out columns, and dx sums over the projections;
+ *  - h_save / h_saved are [n_parts][T][rank_stride] (one plane per projection);
+ *  - marlaas_lora_forward_static_ws and MARLAAS_FLAG_REUSE_PLAN work as on any pool.
+ * With n_parts = 1 the pool is an ordinary one (but for the multiple-of-256 rule). */
+size_t marlaas_adapter_pool_storage_bytes_segmented(int64_t d_in, int32_t n_parts, const int64_t* part_d_out,
+                                                    int32_t max_rank, int32_t capacity);
+marlaas_status_t marlaas_adapter_pool_create_segmented(marlaas_pool_t** out, int device, int64_t d_in, int32_t n_parts,
+                                                       const int64_t* part_d_out /* HOST */, int32_t max_rank,
+                                                       int32_t capacity, void* storage, size_t storage_bytes,
+                                                       void* cuda_stream);
+/* Number of projections the pool holds (1 for a pool made by marlaas_adapter_pool_create). */
+int32_t marlaas_adapter_pool_parts(const marlaas_pool_t* pool);
+
 /* Commit adapter version `version` of tenant `tenant_id` into the pool ("Commit updated parameters to M",
  * Algorithm 1; Asynchronous Execution, training step).  A: bf16 [d_in][rank], B: bf16 [rank][d_out],
  * both row-major device memory, copied and re-laid-out in stream order (the caller may reuse them once the

@@ -41,6 +41,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
     "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
+    "marlaas_adapter_pool_storage_bytes_segmented", "marlaas_adapter_pool_create_segmented", "marlaas_adapter_pool_parts",
 ]
 
 
@@ -80,6 +81,12 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_adapter_pool_create.argtypes = [P(vp), ctypes.c_int, i64, i64, i32, i32, vp, sz, vp]
     L.marlaas_adapter_pool_destroy.restype = i32
     L.marlaas_adapter_pool_destroy.argtypes = [vp]
+    L.marlaas_adapter_pool_storage_bytes_segmented.restype = sz
+    L.marlaas_adapter_pool_storage_bytes_segmented.argtypes = [i64, i32, P(i64), i32, i32]
+    L.marlaas_adapter_pool_create_segmented.restype = i32
+    L.marlaas_adapter_pool_create_segmented.argtypes = [P(vp), ctypes.c_int, i64, i32, P(i64), i32, i32, vp, sz, vp]
+    L.marlaas_adapter_pool_parts.restype = i32
+    L.marlaas_adapter_pool_parts.argtypes = [vp]
     L.marlaas_adapter_pool_register.restype = i32
     L.marlaas_adapter_pool_register.argtypes = [vp, u64, u64, i32, f32, vp, vp, P(i32), vp]
     L.marlaas_adapter_pool_unregister.restype = i32
@@ -174,23 +181,38 @@ class Segments:
 
 
 class AdapterPool:
-    """marlaas_pool_t plus the torch tensor that owns its device storage."""
+    """marlaas_pool_t plus the torch tensor that owns its device storage.  With `parts` (the widths of several
+    projections that read the same activations) the pool is made by marlaas_adapter_pool_create_segmented and d_out
+    is their sum."""
 
-    def __init__(self, d_in: int, d_out: int, max_rank: int, capacity: int, device="cuda:0", stream=None):
+    def __init__(self, d_in: int, d_out: int, max_rank: int, capacity: int, device="cuda:0", stream=None,
+                 parts: Optional[Sequence[int]] = None):
         L = load_library()
         self.device = torch.device(device)
         if self.device.type != "cuda":
             raise MarlaasError(MARLAAS_ERR_UNSUPPORTED_DEVICE, "the layer runs on a CUDA device only")
         idx = self.device.index if self.device.index is not None else torch.cuda.current_device()
+        self.parts = None if parts is None else [int(p) for p in parts]
+        if self.parts is not None:
+            assert d_out == sum(self.parts)
+        self.n_parts = 1 if self.parts is None else len(self.parts)
         self.d_in, self.d_out, self.max_rank, self.capacity = d_in, d_out, max_rank, capacity
-        nbytes = L.marlaas_adapter_pool_storage_bytes(d_in, d_out, max_rank, capacity)
+        if self.parts is None:
+            nbytes = L.marlaas_adapter_pool_storage_bytes(d_in, d_out, max_rank, capacity)
+        else:
+            widths = (ctypes.c_int64 * len(self.parts))(*self.parts)
+            nbytes = L.marlaas_adapter_pool_storage_bytes_segmented(d_in, len(self.parts), widths, max_rank, capacity)
         if nbytes == 0:
             raise MarlaasError(MARLAAS_ERR_INVALID_ARG, "invalid pool dimensions")
         with torch.cuda.device(idx):
             self.storage = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
             h = ctypes.c_void_p()
-            _check(L.marlaas_adapter_pool_create(ctypes.byref(h), idx, d_in, d_out, max_rank, capacity,
-                                                 _dptr(self.storage), nbytes, _stream(stream)))
+            if self.parts is None:
+                _check(L.marlaas_adapter_pool_create(ctypes.byref(h), idx, d_in, d_out, max_rank, capacity,
+                                                     _dptr(self.storage), nbytes, _stream(stream)))
+            else:
+                _check(L.marlaas_adapter_pool_create_segmented(ctypes.byref(h), idx, d_in, len(self.parts), widths, max_rank,
+                                                               capacity, _dptr(self.storage), nbytes, _stream(stream)))
         self.handle = h
         self.rank_stride = int(L.marlaas_adapter_pool_rank_stride(h))
         self._workspaces = {}
@@ -218,7 +240,15 @@ class AdapterPool:
 
 def marlaas_adapter_pool_register(pool: AdapterPool, tenant_id: int, version: int, rank: int, alpha: float,
                                   A: Optional[torch.Tensor], B: Optional[torch.Tensor], stream=None) -> int:
-    if rank > 0:
+    if rank > 0 and pool.n_parts > 1:
+        # one pair per projection, handed to the library as blocks one after another
+        assert len(A) == pool.n_parts and len(B) == pool.n_parts
+        for p in range(pool.n_parts):
+            assert tuple(A[p].shape) == (pool.d_in, rank) and tuple(B[p].shape) == (rank, pool.parts[p])
+        A = torch.cat([a.contiguous().reshape(-1) for a in A])
+        B = torch.cat([b.contiguous().reshape(-1) for b in B])
+        assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.device == pool.device and B.device == pool.device
+    elif rank > 0:
         assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.is_contiguous() and B.is_contiguous()
         assert tuple(A.shape) == (pool.d_in, rank) and tuple(B.shape) == (rank, pool.d_out)
         assert A.device == pool.device and B.device == pool.device
@@ -263,10 +293,19 @@ def marlaas_adapter_pool_lookup(pool: AdapterPool, tenant_id: int):
 
 
 def marlaas_adapter_pool_export(pool: AdapterPool, slot: int, rank: int, stream=None):
-    A = torch.empty((pool.d_in, rank), dtype=torch.bfloat16, device=pool.device)
-    B = torch.empty((rank, pool.d_out), dtype=torch.bfloat16, device=pool.device)
+    """The slot's adapter in the caller's layout; for a pool over several projections, two lists (one A and one B per
+    projection)."""
+    A = torch.empty((pool.n_parts * pool.d_in, rank), dtype=torch.bfloat16, device=pool.device)
+    B = torch.empty(rank * pool.d_out, dtype=torch.bfloat16, device=pool.device)
     _check(load_library().marlaas_adapter_pool_export(pool.handle, slot, _dptr(A), _dptr(B), _stream(stream)))
-    return A, B
+    if pool.n_parts == 1:
+        return A, B.view(rank, pool.d_out)
+    As = [A[p * pool.d_in:(p + 1) * pool.d_in] for p in range(pool.n_parts)]
+    Bs, o = [], 0
+    for w in pool.parts:
+        Bs.append(B[o:o + rank * w].view(rank, w))
+        o += rank * w
+    return As, Bs
 
 
 def marlaas_lora_workspace_bytes(pool: AdapterPool, T: int) -> int:
@@ -292,7 +331,7 @@ def marlaas_lora_forward(pool: AdapterPool, x: torch.Tensor, W: torch.Tensor, se
     ldx, ldw, ldy = _mat(x, pool.d_in, "x"), _mat(W, pool.d_out, "W"), _mat(y, pool.d_out, "y")
     assert W.shape[0] == pool.d_in
     if h_save is not None:
-        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and tuple(h_save.shape) == (T, pool.rank_stride)
+        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and h_save.numel() == pool.n_parts * T * pool.rank_stride
     _check(load_library().marlaas_lora_forward(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(y), ldy,
                                                ctypes.byref(seg.c), _dptr(h_save), _dptr(ws), ws.numel(),
                                                flags | seg.flags, _stream(stream)))
@@ -318,7 +357,7 @@ def marlaas_lora_forward_multi(calls, flags: int = 0, stream=None):
             ws = torch.empty(max(marlaas_lora_forward_workspace_bytes(pool, T), 256), dtype=torch.uint8, device=x.device)
         hs = c.get("h_save")
         if hs is not None:
-            assert hs.dtype == torch.float32 and hs.is_contiguous() and tuple(hs.shape) == (T, pool.rank_stride)
+            assert hs.dtype == torch.float32 and hs.is_contiguous() and hs.numel() == pool.n_parts * T * pool.rank_stride
         assert W.shape[0] == pool.d_in
         arr[i] = marlaas_forward_call_t(pool.handle, T, _dptr(x), _mat(x, pool.d_in, "x"), _dptr(W), _mat(W, pool.d_out, "W"),
                                         _dptr(y), _mat(y, pool.d_out, "y"), ctypes.cast(ctypes.byref(seg.c), ctypes.c_void_p),
@@ -343,7 +382,7 @@ def marlaas_lora_forward_static_ws(pool: AdapterPool, x: torch.Tensor, W: torch.
     ldx, ldw, ldy = _mat(x, pool.d_in, "x"), _mat(W, pool.d_out, "W"), _mat(y, pool.d_out, "y")
     assert W.shape[0] == pool.d_in and y.shape[0] == T
     if h_save is not None:
-        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and tuple(h_save.shape) == (T, pool.rank_stride)
+        assert h_save.dtype == torch.float32 and h_save.is_contiguous() and h_save.numel() == pool.n_parts * T * pool.rank_stride
     _check(load_library().marlaas_lora_forward_static_ws(pool.handle, T, _dptr(x), ldx, _dptr(W), ldw, _dptr(y), ldy,
                                                          ctypes.byref(seg.c), _dptr(h_save), flags | seg.flags,
                                                          _stream(stream)))

@@ -15,19 +15,20 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     auto take = [&](size_t bytes) { char* q = p ? p + o : nullptr; o += align_up(bytes, 256); return q; };
     // forward's fields first: a forward call needs only the first fwd_total bytes
     w.tok_slot = (int32_t*)take(sizeof(int32_t) * Tn);
-    w.h = (float*)take(sizeof(float) * Tn * pool->RP);
+    const size_t P = (size_t)pool->P;       // a pool over P projections keeps one plane of h, g and hd per projection
+    w.h = (float*)take(sizeof(float) * P * Tn * pool->RP);
     const size_t ntiles = (Tn + 255) / 256;
     w.umax = (pool->cap < 256 ? pool->cap : 256) * (pool->RP / 16);
     w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
-    w.hd = (bf16*)take(sizeof(bf16) * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
+    w.hd = (bf16*)take(sizeof(bf16) * P * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
     w.xbuf = (float*)take(decode_wide_sm100_xbuf_bytes(pool, (int64_t)Tn));
     w.fwd_total = o;
     w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
     w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
     w.slot_offset = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 2));
-    w.g = (float*)take(sizeof(float) * Tn * pool->RP);
+    w.g = (float*)take(sizeof(float) * P * Tn * pool->RP);
     w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     const size_t nblk = (Tn + 63) / 64;
@@ -119,12 +120,28 @@ static marlaas_status_t make_plan(const marlaas_pool* pool, int64_t T, const mar
 // Shrink for the tensor-core path: batches with several 128-token tiles go through the tcgen05 kernel, small
 // (decode-shaped) batches through the per-token gather kernel, which spreads over more SMs.
 static marlaas_status_t shrink(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                               const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                               const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st,
                                bool out_is_zero = false) {
     if (T >= 512 && shrink_split_sm100_eligible(pool, T, D))
-        return launch_shrink_split_sm100(pool, T, src, ld, D, store, ws, out, st, out_is_zero);
-    if (T >= 512) return launch_shrink_sm100(pool, T, src, ld, D, store, ws, out, st);
-    return launch_shrink_hd(pool, T, src, ld, D, store, ws, out, st);
+        return launch_shrink_split_sm100(pool, T, src, ld, D, store, sld, ws, out, st, out_is_zero);
+    if (T >= 512) return launch_shrink_sm100(pool, T, src, ld, D, store, sld, ws, out, st);
+    return launch_shrink_hd(pool, T, src, ld, D, store, sld, ws, out, st);
+}
+
+// Projection p of a pool over several: the plan (per-token slots, unit lists, gradient block lists) is shared, h, g and hd
+// are planes of T rows each.
+static Workspace part_workspace(const marlaas_pool* pool, const Workspace& ws, int p, int64_t T) {
+    Workspace w = ws;
+    w.h = ws.h + (size_t)p * T * pool->RP;
+    w.g = ws.g + (size_t)p * T * pool->RP;
+    w.hd = ws.hd + (size_t)p * T * ((size_t)ws.umax * 16);
+    return w;
+}
+
+static void set_parts(const marlaas_pool* pool, GemmOperands* o, bool all_parts) {
+    o->parts = pool->P;
+    o->all_parts = all_parts;
+    for (int p = 0; p < pool->P; ++p) o->part_end[p] = pool->part_begin[p + 1];
 }
 
 // Host tables are copied from temporaries of the call: a stream capture would keep pointers into them for its replays.
@@ -228,34 +245,44 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
         }
         return finish(pool, flags, st);
     }
+    const int NP = pool->P;
     if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH)) {
         // h is cleared before the plan so that plan -> shrink -> GEMM are consecutive kernels (each is launched as a
         // programmatic dependent of the one before and overlaps its tail)
         const bool pre_zero = T >= 512 && shrink_split_sm100_eligible(pool, T, pool->K);
-        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(h, 0, sizeof(float) * (size_t)T * pool->RP, st));
+        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(h, 0, sizeof(float) * (size_t)NP * T * pool->RP, st));
         if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
-        if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, h, st, pre_zero)) != MARLAAS_OK) return rc;
+        // one shrink per projection (its block of A rows, its plane of h and hd), then ONE product over the side-by-side W
+        for (int p = 0; p < NP; ++p) {
+            const Workspace wp = part_workspace(pool, ws, p, T);
+            if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K, pool->K, wp,
+                             h + (size_t)p * T * pool->RP, st, pre_zero)) != MARLAAS_OK) return rc;
+        }
         GemmOperands o;
         o.M = T; o.Nout = pool->N; o.Kc = pool->K;
         o.A = (const bf16*)x; o.lda = ldx;
         o.B = (const bf16*)W; o.ldb = ldw; o.b_mn = true;
         o.C = (bf16*)y; o.ldc = ldy;
         o.XA = ws.hd; o.xa_cols = (int64_t)ws.umax * 16;
-        o.XB = pool->d_Bs; o.xb_rows = (int64_t)pool->cap * pool->RP;
+        o.XB = pool->d_Bs; o.xb_rows = (int64_t)pool->cap * pool->RP; o.xb_ld = pool->ldB;
         o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
+        set_parts(pool, &o, false);
         {
             TimedLaunch timed(pool, st);
-            rc = gemm2_sm100_eligible(pool, T) ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
+            rc = (NP > 1 || gemm2_sm100_eligible(pool, T)) ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
             if (rc != MARLAAS_OK) return rc;
         }
         return finish(pool, flags, st);
     }
     if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
-    if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, h, st)) != MARLAAS_OK) return rc;
-    {
+    for (int p = 0; p < NP; ++p) {      // the plain kernels take one projection at a time
+        const int64_t c0 = pool->part_begin[p], Np = pool->part_begin[p + 1] - c0;
+        float* hp = h + (size_t)p * T * pool->RP;
+        if ((rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K, pool->K,
+                                ws.tok_slot, hp, st)) != MARLAAS_OK) return rc;
         TimedLaunch timed(pool, st);
-        if ((rc = launch_gemm_cuda_core(pool, T, pool->N, pool->K, (const bf16*)x, ldx, (const bf16*)W, ldw, false,
-                                        (bf16*)y, ldy, h, pool->d_Bs, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+        if ((rc = launch_gemm_cuda_core(pool, T, Np, pool->K, (const bf16*)x, ldx, (const bf16*)W + c0, ldw, false,
+                                        (bf16*)y + c0, ldy, hp, pool->d_Bs + c0, pool->ldB, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
     return finish(pool, flags, st);
 }
@@ -365,29 +392,57 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
     if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
+    if (pool->P > 1 && pool->cap > 64 && (want_dA || want_dB)) {
+        // the per-projection pointer tables of such a pool are temporaries of this call, copied by memcpy nodes
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        MARLAAS_CUDA_TRY(cudaStreamIsCapturing(st, &cs));
+        if (cs != cudaStreamCaptureStatusNone)
+            return fail(MARLAAS_ERR_INVALID_ARG, "%s: adapter gradients of a pool over several projections with more than 64 slots "
+                        "cannot be captured", fn);
+    }
     const bool acc = (flags & MARLAAS_FLAG_ACCUMULATE) != 0;
 
     const bool tc_path = !(flags & MARLAAS_FLAG_CUDA_CORE_PATH);
+    const int NP = pool->P;
+    const size_t plane = (size_t)T * pool->RP;      // floats per projection in h, g (and h_saved)
     const bool pre_zero = tc_path && T >= 512 && (dx || want_dA) && shrink_split_sm100_eligible(pool, T, pool->N);
     if (tc_path && T > 0) {
-        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.g, 0, sizeof(float) * (size_t)T * pool->RP, st));   // see forward
+        if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.g, 0, sizeof(float) * NP * plane, st));   // see forward
         if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
     } else {
         if ((rc = make_tok_slot(pool, T, seg, flags, host_ts, ws.tok_slot, st)) != MARLAAS_OK) return rc;
     }
+    // g_p = dy[:, columns of projection p] B_p^T: one pass over dy in all
     if (T > 0 && (dx || want_dA)) {
-        if (tc_path) {
-            if ((rc = shrink(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws, ws.g, st, pre_zero)) != MARLAAS_OK) return rc;
-        } else {
-            if ((rc = launch_rowdot(pool, T, (const bf16*)dy, lddy, pool->N, pool->d_Bs, ws.tok_slot, ws.g, st)) != MARLAAS_OK) return rc;
+        for (int p = 0; p < NP; ++p) {
+            const int64_t c0 = pool->part_begin[p], Np = pool->part_begin[p + 1] - c0;
+            const Workspace wp = part_workspace(pool, ws, p, T);
+            if (tc_path) {
+                if ((rc = shrink(pool, T, (const bf16*)dy + c0, lddy, Np, pool->d_Bs + c0, pool->ldB, wp, wp.g, st, pre_zero)) != MARLAAS_OK) return rc;
+            } else {
+                if ((rc = launch_rowdot(pool, T, (const bf16*)dy + c0, lddy, Np, pool->d_Bs + c0, pool->ldB, ws.tok_slot, wp.g, st)) != MARLAAS_OK) return rc;
+            }
         }
     }
+    // per-projection views of the caller's gradient tables: block p of dA_t is [K][r_t], block p of dB_t is [r_t][N_p]
+    std::vector<float*> dA_part, dB_part;
+    auto part_tables = [&](int p) {
+        if (NP == 1) return;
+        dA_part.assign((size_t)pool->cap, nullptr);
+        dB_part.assign((size_t)pool->cap, nullptr);
+        for (int s = 0; s < pool->cap; ++s) {
+            const size_t r = (size_t)pool->slots[s].rank;
+            if (want_dA && dA_slots[s]) dA_part[s] = dA_slots[s] + (size_t)p * pool->K * r;
+            if (want_dB && dB_slots[s]) dB_part[s] = dB_slots[s] + r * (size_t)pool->part_begin[p];
+        }
+    };
     // The adapter-gradient kernels read none of the dx GEMM's output: when they need no further pass over the workspace
     // the GEMM uses (the saved h is given, the tensor-core reduction is certain to fit) they are issued on a side stream
     // of the pool, forked here and joined at the end, so that their small planning and copy kernels run beside the
     // GEMM instead of after it.
     const bool tc_grad0 = tc_path && (want_dA || want_dB) && grad_sm100_eligible(pool, T);
     const bool fits0 = tc_grad0 && cdiv(T, 64) + (int64_t)seg->num_segments <= (int64_t)ws.max_copies;
+    const bool gemm2 = NP > 1 || gemm2_sm100_eligible(pool, T);
     const bool overlap = fits0 && T > 0 && dx && (!want_dB || h_saved) && gemm2_sm100_eligible(pool, T) && pool->cap <= 64;
     if (overlap) {
         if (!pool->side) {
@@ -406,15 +461,16 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         o.B = (const bf16*)W; o.ldb = ldw; o.b_mn = false;
         o.C = (bf16*)dx; o.ldc = lddx;
         o.XA = ws.hd; o.xa_cols = (int64_t)ws.umax * 16;
-        o.XB = pool->d_At; o.xb_rows = (int64_t)pool->cap * pool->RP;
+        o.XB = pool->d_At; o.xb_rows = (int64_t)NP * pool->cap * pool->RP; o.xb_ld = pool->K;
         o.tile_nunits = ws.tile_nunits; o.tile_units = ws.tile_units; o.umax = ws.umax;
+        set_parts(pool, &o, true);      // the low-rank term of dx sums over every projection
         TimedLaunch timed(pool, st);
-        rc = gemm2_sm100_eligible(pool, T) ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
+        rc = gemm2 ? launch_gemm2_sm100(pool, o, st) : launch_gemm_sm100(pool, o, st);
         if (rc != MARLAAS_OK) return rc;
     } else if (T > 0 && dx) {
         TimedLaunch timed(pool, st);
         if ((rc = launch_gemm_cuda_core(pool, T, pool->K, pool->N, (const bf16*)dy, lddy, (const bf16*)W, ldw, true,
-                                        (bf16*)dx, lddx, ws.g, pool->d_At, ws.tok_slot, st)) != MARLAAS_OK) return rc;
+                                        (bf16*)dx, lddx, ws.g, pool->d_At, pool->K, ws.tok_slot, st, NP, (int64_t)plane)) != MARLAAS_OK) return rc;
     }
     if (want_dA || want_dB) {
         const bool tc_grad = tc_path && grad_sm100_eligible(pool, T);
@@ -432,21 +488,30 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             // unjoined would invalidate a capture the caller's stream may be part of
             auto side_work = [&]() -> marlaas_status_t {
                 marlaas_status_t r;
-                if (!(flags & MARLAAS_FLAG_REUSE_PLAN)) {
-                    if ((r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
-                } else {
-                    // the plan kernel also zeroes the reductions' work-item counters; a reused plan needs them zeroed again
-                    MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), gs));
+                for (int p = 0; p < NP; ++p) {
+                    if (p == 0 && !(flags & MARLAAS_FLAG_REUSE_PLAN)) {
+                        if ((r = launch_grad_plan(pool, T, ws, gs)) != MARLAAS_OK) return r;
+                    } else {
+                        // the plan kernel also zeroes the reductions' work-item counters; a reused plan needs them zeroed again
+                        MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), gs));
+                    }
+                    part_tables(p);
+                    float* const* dAp = NP == 1 ? dA_slots : dA_part.data();
+                    float* const* dBp = NP == 1 ? dB_slots : dB_part.data();
+                    const int64_t c0 = pool->part_begin[p], Np = pool->part_begin[p + 1] - c0;
+                    const bf16* dyp = (const bf16*)dy + c0;
+                    const float* hp = h_saved ? h_saved + p * plane : nullptr;
+                    const float* gp = ws.g + p * plane;
+                    // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
+                    if (want_dB && (r = launch_grad_sm100(pool, T, Np, dyp, lddy, hp, nullptr, dBp, false, acc, ws,
+                                                          gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
+                    if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, gp, nullptr, dAp, true, acc, ws,
+                                                          gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
+                    if (want_dB && (r = launch_grad_sm100(pool, T, Np, dyp, lddy, hp, nullptr, dBp, false, acc, ws,
+                                                          gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
+                    if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, gp, nullptr, dAp, true, acc, ws,
+                                                          gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
                 }
-                // both sets of copies first (small kernels that fit beside the GEMM's CTAs), then the two reductions
-                if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
-                                                      gs, ws.hm, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
-                if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
-                                                      gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
-                if (want_dB && (r = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h_saved, nullptr, dB_slots, false, acc, ws,
-                                                      gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
-                if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, nullptr, dA_slots, true, acc, ws,
-                                                      gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
                 return MARLAAS_OK;
             };
             rc = side_work();
@@ -456,28 +521,38 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             return finish(pool, flags, st);
         }
         if (tc_grad && !(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
-        if (tc_grad && (flags & MARLAAS_FLAG_REUSE_PLAN)) MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), st));
         if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
-        if (want_dB) {
-            const float* h = h_saved;
-            if (!h && T > 0) {
-                if (tc_path) rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws, ws.h, st);
-                else rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, ws.tok_slot, ws.h, st);
-                if (rc != MARLAAS_OK) return rc;
-                h = ws.h;
+        for (int p = 0; p < NP; ++p) {
+            if (tc_grad && (p > 0 || (flags & MARLAAS_FLAG_REUSE_PLAN)))
+                MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), st));
+            part_tables(p);
+            float* const* dAp = NP == 1 ? dA_slots : dA_part.data();
+            float* const* dBp = NP == 1 ? dB_slots : dB_part.data();
+            const int64_t c0 = pool->part_begin[p], Np = pool->part_begin[p + 1] - c0;
+            const bf16* dyp = (const bf16*)dy + c0;
+            const Workspace wp = part_workspace(pool, ws, p, T);
+            if (want_dB) {
+                const float* h = h_saved ? h_saved + p * plane : nullptr;
+                if (!h && T > 0) {
+                    const bf16* Ap = pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K;
+                    if (tc_path) rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, Ap, pool->K, wp, wp.h, st);
+                    else rc = launch_rowdot(pool, T, (const bf16*)x, ldx, pool->K, Ap, pool->K, ws.tok_slot, wp.h, st);
+                    if (rc != MARLAAS_OK) return rc;
+                    h = wp.h;
+                }
+                if (!inline_tables)
+                    MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dBp, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+                if (tc_grad && (rc = launch_grad_sm100(pool, T, Np, dyp, lddy, h, ws.dB_ptrs, dBp, false, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
+                if (!fits && (rc = launch_grad_reduce(pool, Np, dyp, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
+                                                      false, acc, st, run_flag)) != MARLAAS_OK) return rc;
             }
-            if (!inline_tables)
-                MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dB_ptrs, dB_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->N, (const bf16*)dy, lddy, h, ws.dB_ptrs, dB_slots, false, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
-            if (!fits && (rc = launch_grad_reduce(pool, pool->N, (const bf16*)dy, lddy, h, ws.perm, ws.slot_offset, ws.dB_ptrs,
-                                                  false, acc, st, run_flag)) != MARLAAS_OK) return rc;
-        }
-        if (want_dA) {
-            if (!inline_tables)
-                MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dA_slots, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
-            if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, ws.g, ws.dA_ptrs, dA_slots, true, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
-            if (!fits && (rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, ws.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
-                                                  true, acc, st, run_flag)) != MARLAAS_OK) return rc;
+            if (want_dA) {
+                if (!inline_tables)
+                    MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.dA_ptrs, dAp, sizeof(float*) * (size_t)pool->cap, cudaMemcpyHostToDevice, st));
+                if (tc_grad && (rc = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, wp.g, ws.dA_ptrs, dAp, true, acc, ws, st, ws.hm)) != MARLAAS_OK) return rc;
+                if (!fits && (rc = launch_grad_reduce(pool, pool->K, (const bf16*)x, ldx, wp.g, ws.perm, ws.slot_offset, ws.dA_ptrs,
+                                                      true, acc, st, run_flag)) != MARLAAS_OK) return rc;
+            }
         }
     }
     return finish(pool, flags, st);

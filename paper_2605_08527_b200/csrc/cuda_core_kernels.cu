@@ -10,7 +10,7 @@ __device__ __forceinline__ float bf2f(bf16 v) { return __bfloat162float(v); }
 // One CTA per token, one warp per rank index (strided); 16-byte loads along the contiguous dimension,
 // warp-shuffle reduction.  Used for h = x A_t (store = At, D = K) and g = dy B_t^T (store = Bs, D = N).
 __global__ void __launch_bounds__(128) k_rowdot(int64_t D, const bf16* __restrict__ src, int64_t ld,
-                                                const bf16* __restrict__ store, const int32_t* __restrict__ tok_slot,
+                                                const bf16* __restrict__ store, int64_t sld, const int32_t* __restrict__ tok_slot,
                                                 const int32_t* __restrict__ d_rank, int RP, int cap,
                                                 float* __restrict__ out) {
     const int64_t i = blockIdx.x;
@@ -21,7 +21,7 @@ __global__ void __launch_bounds__(128) k_rowdot(int64_t D, const bf16* __restric
     for (int j = warp; j < RP; j += 4) {
         float acc = 0.f;
         if (j < r) {
-            const bf16* a = store + ((size_t)t * RP + j) * D;
+            const bf16* a = store + ((size_t)t * RP + j) * sld;
             for (int64_t d = (int64_t)lane * 8; d < D; d += 256) {
                 const uint4 xv = *reinterpret_cast<const uint4*>(row + d);
                 const uint4 av = *reinterpret_cast<const uint4*>(a + d);
@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(128) k_rowdot(int64_t D, const bf16* __restric
 // Same dot products, plus the token's row of the block-diagonal bf16 operand the tensor-core GEMM multiplies with
 // the adapter rows: bf16(s_t * h) in the columns of the token's own tenant units, zeros in the tile's other units.
 __global__ void __launch_bounds__(128) k_shrink_hd(int64_t D, const bf16* __restrict__ src, int64_t ld,
-                                                   const bf16* __restrict__ store, const int32_t* __restrict__ tok_slot,
+                                                   const bf16* __restrict__ store, int64_t sld, const int32_t* __restrict__ tok_slot,
                                                    const int32_t* __restrict__ tok_uoff,
                                                    const int32_t* __restrict__ tile_nunits,
                                                    const int32_t* __restrict__ d_rank, const float* __restrict__ d_scale,
@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(128) k_shrink_hd(int64_t D, const bf16* __rest
     for (int j = warp; j < RP; j += 4) {
         float acc = 0.f;
         if (j < r) {
-            const bf16* a = store + ((size_t)t * RP + j) * D;
+            const bf16* a = store + ((size_t)t * RP + j) * sld;
             for (int64_t d = (int64_t)lane * 8; d < D; d += 256) {
                 const uint4 xv = *reinterpret_cast<const uint4*>(row + d);
                 const uint4 av = *reinterpret_cast<const uint4*>(a + d);
@@ -103,14 +103,15 @@ __global__ void __launch_bounds__(128) k_shrink_hd(int64_t D, const bf16* __rest
 }
 
 // ---- base GEMM + fused low-rank term ----------------------------------------------------------------------
-// C[i][c] = bf16( sum_k A[i][k] * Wop[k][c] + s_t * sum_j hg[i][j] * store[(t*RP+j)][c] )
-// 64x64 tile, 16-deep k slab, 256 threads x (4x4) outputs.
+// C[i][c] = bf16( sum_k A[i][k] * Wop[k][c] + s_t * sum_p sum_j hg[p][i][j] * store[((p*cap + t)*RP+j)][c] )
+// (nparts = 1 but for the dx of a pool over several projections, whose low-rank term sums over all of them: hg planes
+// hg_plane floats apart, store rows sld elements apart).  64x64 tile, 16-deep k slab, 256 threads x (4x4) outputs.
 template <bool TRANS_W>
 __global__ void __launch_bounds__(256) k_gemm_cuda_core(int64_t T, int64_t Nout, int64_t Kc, const bf16* __restrict__ A,
                                                         int64_t lda, const bf16* __restrict__ W, int64_t ldw,
                                                         bf16* __restrict__ C, int64_t ldc, const float* __restrict__ hg,
-                                                        const bf16* __restrict__ store,
-                                                        const int32_t* __restrict__ tok_slot,
+                                                        const bf16* __restrict__ store, int64_t sld, int nparts,
+                                                        int64_t hg_plane, const int32_t* __restrict__ tok_slot,
                                                         const int32_t* __restrict__ d_rank,
                                                         const float* __restrict__ d_scale, int RP, int cap) {
     __shared__ float sA[16][64 + 1];
@@ -166,7 +167,9 @@ __global__ void __launch_bounds__(256) k_gemm_cuda_core(int64_t T, int64_t Nout,
             const int64_t gc = col0 + tx * 4 + q;
             if (gc >= Nout) continue;
             float d = 0.f;
-            for (int j = 0; j < r; ++j) d = fmaf(hg[gi * RP + j], bf2f(store[((size_t)t * RP + j) * Nout + gc]), d);
+            for (int p = 0; p < nparts; ++p)
+                for (int j = 0; j < r; ++j)
+                    d = fmaf(hg[p * hg_plane + gi * RP + j], bf2f(store[(((size_t)p * cap + t) * RP + j) * sld + gc]), d);
             C[gi * ldc + gc] = __float2bfloat16_rn(acc[p][q] + s * d);
         }
     }
@@ -223,17 +226,17 @@ __global__ void __launch_bounds__(128) k_grad_reduce(int64_t C, const bf16* __re
 }
 
 marlaas_status_t launch_rowdot(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                               const bf16* store, const int32_t* tok_slot, float* out, cudaStream_t st) {
+                               const bf16* store, int64_t sld, const int32_t* tok_slot, float* out, cudaStream_t st) {
     if (T <= 0) return MARLAAS_OK;
-    k_rowdot<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, tok_slot, pool->d_rank, pool->RP, pool->cap, out);
+    k_rowdot<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, sld, tok_slot, pool->d_rank, pool->RP, pool->cap, out);
     MARLAAS_LAUNCH_CHECK("k_rowdot");
     return MARLAAS_OK;
 }
 
 marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                  const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+                                  const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st) {
     if (T <= 0) return MARLAAS_OK;
-    k_shrink_hd<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, ws.tok_slot, ws.tok_uoff, ws.tile_nunits, pool->d_rank,
+    k_shrink_hd<<<(unsigned)T, 128, 0, st>>>(D, src, ld, store, sld, ws.tok_slot, ws.tok_uoff, ws.tile_nunits, pool->d_rank,
                                              pool->d_scale, pool->RP, pool->cap, ws.umax * 16, out, ws.hd);
     MARLAAS_LAUNCH_CHECK("k_shrink_hd");
     return MARLAAS_OK;
@@ -241,15 +244,15 @@ marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf1
 
 marlaas_status_t launch_gemm_cuda_core(const marlaas_pool* pool, int64_t T, int64_t Nout, int64_t Kc,
                                        const bf16* A, int64_t lda, const bf16* W, int64_t ldw, bool trans_w,
-                                       bf16* C, int64_t ldc, const float* hg, const bf16* store,
-                                       const int32_t* tok_slot, cudaStream_t st) {
+                                       bf16* C, int64_t ldc, const float* hg, const bf16* store, int64_t sld,
+                                       const int32_t* tok_slot, cudaStream_t st, int nparts, int64_t hg_plane) {
     if (T <= 0) return MARLAAS_OK;
     dim3 grid((unsigned)cdiv(Nout, 64), (unsigned)cdiv(T, 64));
     if (trans_w)
-        k_gemm_cuda_core<true><<<grid, 256, 0, st>>>(T, Nout, Kc, A, lda, W, ldw, C, ldc, hg, store, tok_slot,
+        k_gemm_cuda_core<true><<<grid, 256, 0, st>>>(T, Nout, Kc, A, lda, W, ldw, C, ldc, hg, store, sld, nparts, hg_plane, tok_slot,
                                                      pool->d_rank, pool->d_scale, pool->RP, pool->cap);
     else
-        k_gemm_cuda_core<false><<<grid, 256, 0, st>>>(T, Nout, Kc, A, lda, W, ldw, C, ldc, hg, store, tok_slot,
+        k_gemm_cuda_core<false><<<grid, 256, 0, st>>>(T, Nout, Kc, A, lda, W, ldw, C, ldc, hg, store, sld, nparts, hg_plane, tok_slot,
                                                       pool->d_rank, pool->d_scale, pool->RP, pool->cap);
     MARLAAS_LAUNCH_CHECK("k_gemm_cuda_core");
     return MARLAAS_OK;

@@ -93,6 +93,10 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     int32_t* const s_list = s_off;
     int32_t* const s_stab = s_off + max(staged_tab ? g.S + 1 : 0, Tp);
     dk_launch_dependents();      // the GEMM may start streaming W now; it waits for this grid before the expand
+    // blockIdx.y = the projection of a pool that holds several: its block of A rows, its plane of h and of hd
+    const bf16* const At = g.At + (size_t)blockIdx.y * g.cap * g.RP * g.K;
+    float* const h_out = g.h_out + (size_t)blockIdx.y * g.T * g.RP;
+    bf16* const hd = g.hd + (size_t)blockIdx.y * g.T * g.hd_cols;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int crank = (int)dk_cluster_ctarank();
@@ -100,7 +104,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(cs));
     const int t = (int)dk_cluster_id_x() / g.G;     // tenant slot served by this cluster; == cap: no adapter
     const int gi = (int)dk_cluster_id_x() % g.G;    // which of the tenant's 16-token passes
-    const bool first = (dk_cluster_id_x() == 0 && crank == 0);      // one CTA also publishes tok_slot and checks the table
+    const bool first = (dk_cluster_id_x() == 0 && crank == 0 && blockIdx.y == 0);      // one CTA also publishes tok_slot and checks the table
     const int r_t = t < g.cap ? g.d_rank[t] : 0;
     const float sc = t < g.cap ? g.d_scale[t] : 0.f;
 
@@ -114,7 +118,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     uint4 ba[DS_UB], bb[DS_UB];     // adapter fragments; held_jg / held_b0 say of which rank group and k-block batch
     int held_jg = 0, held_b0 = wb0;
     {
-        const bf16* ar0 = g.At + ((size_t)(t < g.cap ? t : 0) * g.RP + gq) * g.K;
+        const bf16* ar0 = At + ((size_t)(t < g.cap ? t : 0) * g.RP + gq) * g.K;
         const bf16* ar1 = ar0 + (size_t)8 * g.K;
 #pragma unroll
         for (int u = 0; u < DS_UB; ++u) {
@@ -207,11 +211,11 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
     for (int e = crank * 4 + warp; e < n_t; e += cs * 4) {
         if ((e / DS_PASS) % g.G != gi) continue;     // another cluster's pass
         const int tok = s_list[e];
-        bf16* row = g.hd + (size_t)tok * g.hd_cols;
+        bf16* row = hd + (size_t)tok * g.hd_cols;
         for (int c = lane * 8; c < g.hd_cols; c += 256)
             if (c < own0 || c >= own1) *reinterpret_cast<uint4*>(row + c) = make_uint4(0u, 0u, 0u, 0u);
         if (r_t == 0)
-            for (int j = lane; j < g.RP; j += 32) g.h_out[(size_t)tok * g.RP + j] = 0.f;
+            for (int j = lane; j < g.RP; j += 32) h_out[(size_t)tok * g.RP + j] = 0.f;
     }
     if (r_t == 0) return;        // uniform over the cluster
 
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
         const bf16* xr1 = gq + 8 < np ? g.x + (size_t)s_list[p0 + gq + 8] * g.ldx : nullptr;
         for (int jg = 0; jg < ngroups; ++jg) {
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-            const bf16* ar0 = g.At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
+            const bf16* ar0 = At + ((size_t)t * g.RP + jg * 16 + gq) * g.K;
             const bf16* ar1 = ar0 + (size_t)8 * g.K;
             for (int b0 = wb0; b0 < wb1; b0 += DS_UB) {
                 uint4 xa[DS_UB], xb[DS_UB];
@@ -276,8 +280,8 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
                         float v = 0.f;
                         for (int s = 0; s < cs; ++s) v += sm.part[s][e];   // fixed order
                         const int tok = s_list[p0 + i];
-                        g.h_out[(size_t)tok * g.RP + jg * 16 + j] = v;
-                        g.hd[(size_t)tok * g.hd_cols + own0 + jg * 16 + j] = __float2bfloat16_rn(sc * v);
+                        h_out[(size_t)tok * g.RP + jg * 16 + j] = v;
+                        hd[(size_t)tok * g.hd_cols + own0 + jg * 16 + j] = __float2bfloat16_rn(sc * v);
                     }
                 }
             }
@@ -290,8 +294,8 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
             for (int e = tid; e < np * rest; e += DS_THREADS) {
                 const int i = e / rest, j = ngroups * 16 + e % rest;
                 const int tok = s_list[p0 + i];
-                g.h_out[(size_t)tok * g.RP + j] = 0.f;
-                g.hd[(size_t)tok * g.hd_cols + own0 + j] = __float2bfloat16_rn(0.f);
+                h_out[(size_t)tok * g.RP + j] = 0.f;
+                hd[(size_t)tok * g.hd_cols + own0 + j] = __float2bfloat16_rn(0.f);
             }
         }
     }
@@ -312,6 +316,8 @@ struct DecodeGemmArgs {
     int nch;             // 64-column chunks of the B operand staged per CTA: the pair's strip is 128 * nch columns
     int kp;              // 64-deep panels per pipeline step: one TMA instruction per operand moves all of them
     int stages;
+    int parts;           // projections held by the pool: hd is [parts][T][..] and strip n0 takes the plane of its projection
+    int part_end[4];     // last column + 1 of each projection
     bf16* C;
     int64_t ldc;
     int32_t* status;
@@ -378,6 +384,9 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
     const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
     const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
+    int part = 0;
+    while (part < g.parts - 1 && n0 >= g.part_end[part]) ++part;
+    const int xa_m = my_m + part * g.T;         // this half's rows of the projection's plane of hd
 
     const int ks0 = (int)pairi * g.num_ks / g.S, ks1 = ((int)pairi + 1) * g.num_ks / g.S;
     const int xs0 = (int)pairi * g.num_xs / g.S, xs1 = ((int)pairi + 1) * g.num_xs / g.S;
@@ -434,13 +443,13 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
             if (ok && xs0 < xs1) dk_wait_prerequisites();     // hd comes from the shrink grid
             for (int i = 0; i < npre && ok; ++i, ++it) {
-                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, (xs0 + i) * g.kp);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, xa_m, (xs0 + i) * g.kp);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
             for (int xs = xs0 + npre; xs < xs1 && ok; ++xs, ++it) {
                 if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 42))) break;
                 if (half == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
-                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, my_m, xs * g.kp);
+                if (have_rows) dg_tma_pair_3d(sA + s * a_stage_bytes, &tmXA, full0 + 8 * s, 0, xa_m, xs * g.kp);
                 for (int c = 0; c < my_chunks; ++c)
                     dg_tma_pair(sB + s * b_stage_bytes + c * b_chunk_bytes, &tmXB, full0 + 8 * s, my_n + c * 64, xs * g.kp * BK);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
@@ -654,7 +663,7 @@ marlaas_status_t launch_decode_shrink(const marlaas_pool* pool, int64_t T, const
     // with few tenants a tenant has many 16-token passes: several clusters share them, as many as keep the grid
     // within two CTAs per SM
     const int passes = (int)cdiv(T, DS_PASS);
-    a.G = std::max(1, std::min(passes, (2 * pool->sm_count) / ((pool->cap + 1) * cs)));
+    a.G = std::max(1, std::min(passes, (2 * pool->sm_count) / ((pool->cap + 1) * cs * pool->P)));
     static bool carveout_set[64] = {};
     if (pool->device >= 64 || !carveout_set[pool->device]) {
         // same shared-memory configuration as the GEMM, so that CTAs of both kernels can share an SM
@@ -663,7 +672,7 @@ marlaas_status_t launch_decode_shrink(const marlaas_pool* pool, int64_t T, const
         if (pool->device < 64) carveout_set[pool->device] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((pool->cap + 1) * a.G * cs));
+    cfg.gridDim = dim3((unsigned)((pool->cap + 1) * a.G * cs), (unsigned)pool->P);     // y: the pool's projections
     cfg.blockDim = dim3(DS_THREADS);
     cfg.dynamicSmemBytes = decode_shrink_dyn_smem(T, S);
     cfg.stream = st;
@@ -695,6 +704,8 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
     DecodeGemmArgs g;
     g.T = (int)T; g.Nout = (int)N;
     g.C = y; g.ldc = ldy; g.status = pool->d_status;
+    g.parts = pool->P;
+    for (int p = 0; p < 4; ++p) g.part_end[p] = p < pool->P ? (int)pool->part_begin[p + 1] : 0;
     // strip width and contraction slices: fill the SMs with one wave of clusters of 2 * S CTAs
     struct Shape { int nch, S; };
     const Shape shapes[] = {{1, 2}, {2, 2}, {1, 1}, {2, 1}, {1, 4}, {2, 4}};
@@ -749,8 +760,8 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
     if ((rc = make_panel_map(&tmA, x, T, K, ldx, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
     if ((rc = make_map(&tmB, W, K, N, ldw, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
     if (g.num_xs > 0) {
-        if ((rc = make_panel_map(&tmXA, ws.hd, T, hd_cols, hd_cols, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
-        if ((rc = make_map(&tmXB, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
+        if ((rc = make_panel_map(&tmXA, ws.hd, T * pool->P, hd_cols, hd_cols, (uint32_t)g.kp)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXB, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 64, (uint32_t)(g.kp * BK))) != MARLAAS_OK) return rc;
     } else {
         tmXA = tmA;
         tmXB = tmB;

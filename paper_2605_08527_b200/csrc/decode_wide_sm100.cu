@@ -79,6 +79,8 @@ struct DecodeArgs {
     int S;               // contraction slices per tile: 1, 2 or 4 CTA pairs
     int stages;
     int w3d;             // the W-side operand moves with one 3-D copy per step (N a multiple of 64), else one per chunk
+    int parts;           // projections held by the pool: hd is [parts][T][..] and a strip takes the plane of its projection
+    int part_end[4];     // last column + 1 of each projection
     bf16* C;
     int64_t ldc;
     float* xbuf;         // exchange buffer between the slices of a tile
@@ -141,6 +143,9 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const int n0 = (tile % g.nstrips) * DG_TM;
     const int m0 = (tile / g.nstrips) * DG_TN;
     const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
+    int part = 0;
+    while (part < g.parts - 1 && n0 >= g.part_end[part]) ++part;
+    const int hd_tok = my_tok + part * g.T;          // this half's rows of the projection's plane of hd
     const int ks0 = sl * g.num_ks / g.S, ks1 = (sl + 1) * g.num_ks / g.S;
     const int xs0 = sl * g.num_xs / g.S, xs1 = (sl + 1) * g.num_xs / g.S;
     const int nbase = ks1 - ks0, nstep = nbase + (xs1 - xs0);
@@ -189,7 +194,7 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                     fence_proxy_async_all();
                     hd_ready = true;
                 }
-                if (have_rows) dg_tma_pair_3d(dx, mx, full0 + 8 * s, 0, my_tok, step);
+                if (have_rows) dg_tma_pair_3d(dx, mx, full0 + 8 * s, 0, ex ? hd_tok : my_tok, step);
                 if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
             }
             if (!ok && half == 0) {
@@ -433,6 +438,8 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
     g.num_ks = (int)(K / BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
     g.w3d = (N % 64) == 0;
+    g.parts = pool->P;
+    for (int p = 0; p < 4; ++p) g.part_end[p] = p < pool->P ? (int)pool->part_begin[p + 1] : 0;
     constexpr size_t stage_bytes = 2 * CHUNK_BYTES + A_STAGE_BYTES;
     // The shrink kernel's CTAs are spread over all SMs (two apiece) when this kernel's CTAs arrive: the pipeline takes
     // what two of them leave of an SM's 227 KB, so that neither kernel waits for the other's shared memory.
@@ -451,9 +458,9 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
     else rc = make_map(&tmW, W, K, N, ldw, 64, BK);
     if (rc != MARLAAS_OK) return rc;
     if (g.num_xs > 0) {
-        if ((rc = make_panel_map(&tmXX, ws.hd, T, hd_cols, hd_cols, 1, 128)) != MARLAAS_OK) return rc;
-        if (g.w3d) rc = make_panel_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 2, BK);
-        else rc = make_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, N, 64, BK);
+        if ((rc = make_panel_map(&tmXX, ws.hd, T * pool->P, hd_cols, hd_cols, 1, 128)) != MARLAAS_OK) return rc;
+        if (g.w3d) rc = make_panel_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 2, BK);
+        else rc = make_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 64, BK);
         if (rc != MARLAAS_OK) return rc;
     } else {
         tmXX = tmX;

@@ -31,10 +31,29 @@ struct Gemm2Args {
     const int32_t* tile_nunits;             // per 256-row tile
     const int32_t* tile_units;
     int umax;
+    // A pool over several projections (parts > 1): XA holds one plane of M rows per part; an output tile of the forward
+    // product (all_parts = 0) takes the plane of the part its columns lie in (part_end: the parts' last columns + 1),
+    // the dx product (all_parts = 1) sums over every part's plane against that part's block of XB rows.
+    int parts, all_parts;
+    int part_end[4];
+    int xb_part_rows;
     bf16* C;
     int64_t ldc;
     int32_t* status;
 };
+
+// the parts whose low-rank term enters output columns n0 ...
+__device__ __forceinline__ void tile_parts(const Gemm2Args& g, int n0, int& p_lo, int& p_hi) {
+    p_lo = 0;
+    p_hi = 1;
+    if (g.parts > 1) {
+        if (g.all_parts) p_hi = g.parts;
+        else {
+            while (p_lo < g.parts - 1 && n0 >= g.part_end[p_lo]) ++p_lo;
+            p_hi = p_lo + 1;
+        }
+    }
+}
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -210,15 +229,18 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     waited = true;
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
+                int p_lo, p_hi;
+                tile_parts(g, n0, p_lo, p_hi);
+                for (int p = p_lo; p < p_hi; ++p)
                 for (int x0 = 0; x0 < nun && ok; x0 += 4, ++it) {
                     if (!(ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, abort_word, 32))) break;
                     const uint32_t full = full0 + 8 * s;
                     const int nv = min(4, nun - x0);
                     if (rank == 0)
                         mbar_expect_tx(bar_full + 8 * s, extra_bytes(g, m0, n0, 0, nv) + extra_bytes(g, m0, n0, 1, nv));
-                    if (have_rows) tma_load_2d_pair(sA + s * A_ST, &tmXA, full, x0 * 16, my_m);
+                    if (have_rows) tma_load_2d_pair(sA + s * A_ST, &tmXA, full, x0 * 16, my_m + p * g.M);
                     for (int u = 0; u < nv; ++u) {
-                        const int row = g.tile_units[(size_t)m_idx * g.umax + x0 + u];
+                        const int row = g.tile_units[(size_t)m_idx * g.umax + x0 + u] + (g.all_parts ? p * g.xb_part_rows : 0);
                         for (int c = 0; c < nchunk; ++c)
                             tma_load_2d_pair(sB + s * B_ST + c * CHUNK_BYTES + u * UNIT_BYTES, &tmXB, full,
                                              my_n + c * 64, row);
@@ -282,6 +304,9 @@ k_gemm2_sm100(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     waited = true;
                 }
                 const int nun = g.tile_nunits ? g.tile_nunits[m_idx] : 0;
+                int p_lo, p_hi;
+                tile_parts(g, n_idx * G2_BN, p_lo, p_hi);
+                for (int p = p_lo; p < p_hi; ++p)
                 for (int x0 = 0; x0 < nun && ok; x0 += 4) {
                     if (!(ok = mbar_wait(bar_full + 8 * s, ph, abort_word, 35))) break;
                     tc_fence_after();
@@ -388,6 +413,10 @@ static marlaas_status_t launch_gemm2_t(const marlaas_pool* pool, const GemmOpera
     g.tile_nunits = o.tile_nunits;
     g.tile_units = o.tile_units;
     g.umax = o.umax;
+    g.parts = o.parts > 1 ? o.parts : 1;
+    g.all_parts = o.all_parts ? 1 : 0;
+    for (int p = 0; p < 4; ++p) g.part_end[p] = p < o.parts ? (int)o.part_end[p] : 0;
+    g.xb_part_rows = (int)(o.xb_rows / g.parts);
     g.C = o.C;
     g.ldc = o.ldc;
     g.status = pool->d_status;
@@ -402,8 +431,8 @@ static marlaas_status_t launch_gemm2_t(const marlaas_pool* pool, const GemmOpera
     else rc = make_panel_map(&tmB, o.B, o.Nout, o.Kc, o.ldb, KP);
     if (rc != MARLAAS_OK) return rc;
     if (o.tile_nunits) {
-        if ((rc = make_map(&tmXA, o.XA, o.M, o.xa_cols, o.xa_cols, BK, BM)) != MARLAAS_OK) return rc;
-        if ((rc = make_map(&tmXB, o.XB, o.xb_rows, o.Nout, o.Nout, 64, 16)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXA, o.XA, o.M * g.parts, o.xa_cols, o.xa_cols, BK, BM)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXB, o.XB, o.xb_rows, o.Nout, o.xb_ld, 64, 16)) != MARLAAS_OK) return rc;
     } else {
         tmXA = tmA;
         tmXB = tmB;

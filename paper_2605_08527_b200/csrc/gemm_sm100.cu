@@ -327,7 +327,7 @@ static marlaas_status_t launch_t(const marlaas_pool* pool, const GemmOperands& o
     }
     if (o.tile_nunits) {
         if ((rc = make_map(&tmXA, o.XA, o.M, o.xa_cols, o.xa_cols, BK, BM)) != MARLAAS_OK) return rc;
-        if ((rc = make_map(&tmXB, o.XB, o.xb_rows, o.Nout, o.Nout, 64, 16)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&tmXB, o.XB, o.xb_rows, o.Nout, o.xb_ld, 64, 16)) != MARLAAS_OK) return rc;
     } else {
         tmXA = tmA;
         tmXB = tmB;

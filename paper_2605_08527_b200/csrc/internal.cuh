@@ -61,14 +61,20 @@ struct SlotMeta {
 }  // namespace marlaas
 
 // The pool: host bookkeeping plus pointers into the caller-provided device storage.
-//   At : bf16 [capacity*RP][K]   row (slot*RP + j) = column j of A_t   (zero rows for j >= r_t)
-//   Bs : bf16 [capacity*RP][N]   row (slot*RP + j) = row j of B_t      (zero rows for j >= r_t)
+//   At : bf16 [P][capacity*RP][K]   row (slot*RP + j) of block p = column j of A_t,p   (zero rows for j >= r_t)
+//   Bs : bf16 [capacity*RP][N]      row (slot*RP + j) = row j of [B_t,1 | ... | B_t,P]  (zero rows for j >= r_t)
 // Both serve as gather sources for the shrink (dot products along a contiguous row) and as tensor-core
-// operands for the extra k-steps of the fused expand (rows = rank index).
+// operands for the extra k-steps of the fused expand (rows = rank index).  P = 1 for an ordinary pool; a pool over
+// P projections that read the same activations keeps one A block per projection and the B matrices side by side,
+// so that output range p of the layer pairs with A block p and columns [part_begin[p], part_begin[p+1]) of Bs.
+constexpr int MARLAAS_MAX_PARTS = 4;
 struct marlaas_pool {
     int device = 0;
     int64_t K = 0, N = 0;
     int32_t max_rank = 0, RP = 0, cap = 0;
+    int32_t P = 1;
+    int64_t part_begin[MARLAAS_MAX_PARTS + 1] = {0, 0, 0, 0, 0};
+    int64_t ldB = 0;                // elements between rows of Bs (= N of the whole pool, also in a part's view)
     char* storage = nullptr;
     size_t storage_bytes = 0;
     int32_t* d_status = nullptr;
@@ -93,7 +99,11 @@ namespace marlaas {
 struct StorageLayout {
     size_t off_status, off_sync, off_rank, off_scale, off_At, off_Bs, total;
 };
-StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap);
+StorageLayout storage_layout(int64_t K, int64_t N, int32_t RP, int32_t cap, int32_t parts = 1);
+
+// Part p of a pool over several projections, as a pool of its own (no slot table, no streams: for the kernel launchers
+// only): its A block, its columns of Bs (row pitch ldB unchanged), the shared rank / scale / status arrays.
+void part_view(const marlaas_pool* pool, int p, marlaas_pool* view);
 
 // Per-call workspace (device), carved from the caller's buffer.
 struct Workspace {
@@ -151,10 +161,15 @@ struct GemmOperands {
     bool b_mn;
     bf16* C; int64_t ldc;              // [M][Nout]
     const bf16* XA; int64_t xa_cols;   // [M][xa_cols] (pitch xa_cols)
-    const bf16* XB; int64_t xb_rows;   // [xb_rows][Nout] (pitch Nout)
+    const bf16* XB; int64_t xb_rows;   // [xb_rows][Nout], rows xb_ld elements apart
+    int64_t xb_ld;
     const int32_t* tile_nunits;        // nullptr = no low-rank term
     const int32_t* tile_units;
     int32_t umax;
+    // pools over several projections (the 2-CTA kernel only): XA is [parts][M][xa_cols]; see Gemm2Args
+    int32_t parts = 1;
+    bool all_parts = false;
+    int64_t part_end[4] = {0, 0, 0, 0};
 };
 marlaas_status_t launch_gemm_sm100(const marlaas_pool* pool, const GemmOperands& o, cudaStream_t st);
 // gemm2_sm100.cu: the same product with 2-CTA clusters (256 x 256 tiles), for batches of at least 1024 rows
@@ -182,29 +197,30 @@ marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const 
                                      const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
 
 // shrink_sm100.cu: the same outputs as launch_shrink_hd, computed on the tensor cores tile by tile
+// store: the rows of the pooled store to contract with ([cap*RP] rows of D elements, sld elements apart)
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                     const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
+                                     const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st);
 
 // shrink_split_sm100.cu: the same outputs with one tile per cluster and the contraction split over the cluster's
 // CTAs; applies when all tiles fit one wave
 bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D);
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                                           const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st,
                                            bool out_is_zero = false);
 
 // cuda_core_kernels.cu
 // h/g (fp32, [T][RP]) as launch_rowdot, plus the bf16 block-diagonal operand rows hd for the tensor-core path
 marlaas_status_t launch_shrink_hd(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                  const bf16* store, const Workspace& ws, float* out, cudaStream_t st);
+                                  const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st);
 // out[i][j] = sum_d src[i][d] * store[(slot_i*RP + j)][d] for j < RP (zeros for inactive tokens / padded rows)
 marlaas_status_t launch_rowdot(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                               const bf16* store, const int32_t* tok_slot, float* out, cudaStream_t st);
+                               const bf16* store, int64_t sld, const int32_t* tok_slot, float* out, cudaStream_t st);
 // C[T][Nout] = bf16( A[T][Kc] * op(W) + s_t * sum_j hg[i][j] * store[(slot*RP+j)][c] );
 // trans_w = false: op(W) = W[Kc][Nout] (ldw);  true: op(W) = W^T with W stored [Nout][Kc] (ldw)
 marlaas_status_t launch_gemm_cuda_core(const marlaas_pool* pool, int64_t T, int64_t Nout, int64_t Kc,
                                        const bf16* A, int64_t lda, const bf16* W, int64_t ldw, bool trans_w,
-                                       bf16* C, int64_t ldc, const float* hg, const bf16* store,
-                                       const int32_t* tok_slot, cudaStream_t st);
+                                       bf16* C, int64_t ldc, const float* hg, const bf16* store, int64_t sld,
+                                       const int32_t* tok_slot, cudaStream_t st, int nparts = 1, int64_t hg_plane = 0);
 // out_t[j][c] (transpose_out = false, ld = C) or out_t[c][j] (true, ld = r_t) (+)= s_t * sum_{i in t} hg[i][j] * src[i][c]
 marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const bf16* src, int64_t ld,
                                     const float* hg, const int32_t* perm, const int32_t* slot_offset,

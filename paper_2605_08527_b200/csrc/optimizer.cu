@@ -28,7 +28,7 @@ struct OptTenant {
 struct OptArgs {
     OptTenant t[OPT_MAX_TENANTS];
     int n, RP;
-    int64_t K, N;
+    int64_t K, N, ldB;     // ldB: elements between rows of Bs (N unless the pool holds several projections side by side)
     float lr, b1, b2, eps, wd, gscale, c1, c2;      // c1 = 1 / (1 - beta1^step), c2 = 1 / (1 - beta2^step)
     bf16* At;
     bf16* Bs;
@@ -51,9 +51,20 @@ __global__ void __launch_bounds__(OPT_THREADS) k_adamw_commit(const OptArgs g) {
     const int r = t.rank;
     // ---- B ----
     {
-        bf16* bs = g.Bs + (size_t)t.slot * g.RP * g.N;
+        bf16* bs = g.Bs + (size_t)t.slot * g.RP * g.ldB;
         const int64_t nB = (int64_t)r * g.N;
-        if (t.vec && (g.N & 3) == 0) {
+        if (g.ldB != g.N) {
+            // rows of the store are further apart than rows of B
+            for (int64_t e = (int64_t)blockIdx.x * OPT_THREADS + threadIdx.x; e < nB; e += (int64_t)gridDim.x * OPT_THREADS) {
+                float m = t.mB[e], v = t.vB[e];
+                const float th = adamw_update(t.B[e], t.dB[e], m, v, g);
+                t.mB[e] = m;
+                t.vB[e] = v;
+                t.B[e] = th;
+                const int64_t j = e / g.N;
+                bs[j * g.ldB + (e - j * g.N)] = __float2bfloat16_rn(th);
+            }
+        } else if (t.vec && (g.N & 3) == 0) {
             // four elements per thread and access (r * N is a multiple of 4, rows of the store start 8-byte aligned)
             const int64_t n4 = nB >> 2;
             for (int64_t e = (int64_t)blockIdx.x * OPT_THREADS + threadIdx.x; e < n4; e += (int64_t)gridDim.x * OPT_THREADS) {
@@ -167,26 +178,32 @@ extern "C" marlaas_status_t marlaas_adapter_pool_adamw_commit(marlaas_pool_t* po
     }
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
     OptArgs g;
-    g.RP = pool->RP; g.K = pool->K; g.N = pool->N;
+    g.RP = pool->RP; g.K = pool->K; g.ldB = pool->ldB;
     g.lr = hp->lr; g.b1 = hp->beta1; g.b2 = hp->beta2; g.eps = hp->eps; g.wd = hp->weight_decay; g.gscale = hp->grad_scale;
     g.c1 = (float)(1.0 / (1.0 - std::pow((double)hp->beta1, (double)hp->step)));
     g.c2 = (float)(1.0 / (1.0 - std::pow((double)hp->beta2, (double)hp->step)));
-    g.At = pool->d_At; g.Bs = pool->d_Bs;
+    // a pool over several projections: one pass per part (its A block, its columns of Bs, block p of every array)
+    for (int p = 0; p < pool->P; ++p)
     for (int i0 = 0; i0 < n; i0 += OPT_MAX_TENANTS) {
+        g.N = pool->part_begin[p + 1] - pool->part_begin[p];
+        g.At = pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K;
+        g.Bs = pool->d_Bs + pool->part_begin[p];
         g.n = std::min(OPT_MAX_TENANTS, n - i0);
         int max_rank = 1;
         for (int i = 0; i < g.n; ++i) {
             OptTenant& t = g.t[i];
             const int ii = i0 + i;
-            t.dA = dA[ii]; t.dB = dB[ii]; t.A = A[ii]; t.B = B[ii];
-            t.mA = m_A[ii]; t.vA = v_A[ii]; t.mB = m_B[ii]; t.vB = v_B[ii];
-            t.slot = slot_of[ii]; t.rank = pool->slots[slot_of[ii]].rank;
+            const int32_t r = pool->slots[slot_of[ii]].rank;
+            const size_t oa = (size_t)p * pool->K * r, ob = (size_t)r * pool->part_begin[p];
+            t.dA = dA[ii] + oa; t.dB = dB[ii] + ob; t.A = A[ii] + oa; t.B = B[ii] + ob;
+            t.mA = m_A[ii] + oa; t.vA = v_A[ii] + oa; t.mB = m_B[ii] + ob; t.vB = v_B[ii] + ob;
+            t.slot = slot_of[ii]; t.rank = r;
             t.vec = ((((uintptr_t)t.dA | (uintptr_t)t.dB | (uintptr_t)t.A | (uintptr_t)t.B | (uintptr_t)t.mA | (uintptr_t)t.vA |
                        (uintptr_t)t.mB | (uintptr_t)t.vB) & 15) == 0);
             max_rank = std::max(max_rank, (int)t.rank);
         }
         // enough blocks per tenant to cover its larger matrix once, within a few waves over all tenants
-        const int64_t elems = (int64_t)max_rank * std::max(pool->K, pool->N);
+        const int64_t elems = (int64_t)max_rank * std::max(pool->K, g.N);
         const int64_t want = std::max<int64_t>(cdiv(elems, (int64_t)OPT_THREADS * 8), cdiv(pool->K, (int64_t)OPT_TILE_K));
         const int bx = (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)8 * pool->sm_count / g.n + 1));
         k_adamw_commit<<<dim3((unsigned)bx, (unsigned)g.n), OPT_THREADS, 0, (cudaStream_t)cuda_stream>>>(g);

@@ -235,7 +235,7 @@ k_shrink_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant_
 }  // namespace sm100
 
 marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                     const bf16* store, const Workspace& ws, float* out, cudaStream_t st) {
+                                     const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st) {
     using namespace sm100;
     if (T <= 0) return MARLAAS_OK;
     ShrinkArgs g;
@@ -259,7 +259,7 @@ marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const 
     alignas(64) CUtensorMap tmSrc, tmStore;
     marlaas_status_t rc;
     if ((rc = make_map(&tmSrc, src, T, D, ld, BK, BM)) != MARLAAS_OK) return rc;
-    if ((rc = make_map(&tmStore, store, (int64_t)pool->cap * pool->RP, D, D, BK, 16)) != MARLAAS_OK) return rc;
+    if ((rc = make_map(&tmStore, store, (int64_t)pool->cap * pool->RP, D, sld, BK, 16)) != MARLAAS_OK) return rc;
     MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
     constexpr size_t smem_bytes = 1024 + (size_t)SHRINK_STAGES * (A_STAGE_BYTES + SB_STAGE_BYTES) + 256;
     static bool attr_set[64] = {};

@@ -396,7 +396,7 @@ bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D)
 }
 
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
-                                           const bf16* store, const Workspace& ws, float* out, cudaStream_t st,
+                                           const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st,
                                            bool out_is_zero) {
     using namespace sm100;
     if (T <= 0) return MARLAAS_OK;
@@ -421,7 +421,7 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     marlaas_status_t rc;
     if ((rc = make_panel_map(&tmSrc, src, T, D, ld, SS_KP)) != MARLAAS_OK) return rc;
     for (int i = 0; i < 4; ++i)
-        if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, D, BK, 16u << i)) != MARLAAS_OK) return rc;
+        if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, sld, BK, 16u << i)) != MARLAAS_OK) return rc;
     if (!out_is_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * C));

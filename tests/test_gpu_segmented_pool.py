@@ -1,0 +1,205 @@
+"""A pool over several projections that read the same activations (q, k, v; gate, up): one layer call over the
+side-by-side base weights, the tenants' adapters kept per projection (no block-diagonal zeros stored or streamed).
+The GPU runs the one call; the oracle runs every projection on its own, from the definition.  y must be the separate
+outputs side by side, dx their sum, dA_t / dB_t the separate gradients block after block.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_08527_b200 import binding as B
+from paper_2605_08527_b200 import workloads as wl
+
+from helpers import assert_close, dev_bf16, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(seed, T, K, Ns, ranks, per_token, n_segments=7):
+    """Projections of widths Ns over one x and one segment table; tenant t has rank ranks[t] on every projection."""
+    n = len(ranks)
+    w0 = wl.small_random_case(seed, T, K, Ns[0], list(ranks), n_segments=n_segments)
+    if per_token:
+        ts = wl.uniform_token_slots(seed, T, n).astype(np.int32)
+        ts[min(3, T - 1)] = -1
+        w0.seg_offsets, w0.seg_slot = wl.per_token_table(ts)
+    projs = [w0.projections[0]]
+    for i, N in enumerate(Ns[1:], start=1):
+        wi = wl.small_random_case(seed + 50 * i, T, K, N, list(ranks), n_segments=n_segments)
+        pi = wi.projections[0]
+        pi.x_bits = projs[0].x_bits
+        for a, a0 in zip(pi.adapters, projs[0].adapters):
+            a.tenant_id, a.alpha = a0.tenant_id, a0.alpha
+        projs.append(pi)
+    w0.projections = projs
+    return w0
+
+
+class SegCase:
+    def __init__(self, w, capacity=None):
+        self.w = w
+        ps = w.projections
+        self.Ns = [p.d_out for p in ps]
+        self.K = ps[0].d_in
+        n = len(ps[0].adapters)
+        self.ranks = [a.rank for a in ps[0].adapters]
+        self.pool = B.AdapterPool(self.K, sum(self.Ns), max(self.ranks + [1]), capacity or n, parts=self.Ns)
+        self.W = dev_bf16(np.concatenate([p.W_bits for p in ps], axis=1))
+        self.x = dev_bf16(ps[0].x_bits)
+        self.dy = None if ps[0].dy_bits is None else dev_bf16(np.concatenate([p.dy_bits for p in ps], axis=1))
+        for t in range(n):
+            a0 = ps[0].adapters[t]
+            As = [dev_bf16(p.adapters[t].A_bits) for p in ps] if a0.rank > 0 else None
+            Bs = [dev_bf16(p.adapters[t].B_bits) for p in ps] if a0.rank > 0 else None
+            assert B.marlaas_adapter_pool_register(self.pool, a0.tenant_id, 0, a0.rank, a0.alpha, As, Bs) == t
+        self.seg = B.Segments(torch.from_numpy(w.seg_offsets.astype(np.int32)).cuda(),
+                              torch.from_numpy(w.seg_slot.astype(np.int32)).cuda())
+
+    def grads(self, fill=None):
+        mk = (lambda n: torch.full((n,), fill, dtype=torch.float32, device="cuda:0")) if fill is not None else \
+             (lambda n: torch.empty(n, dtype=torch.float32, device="cuda:0"))
+        dA = [mk(len(self.Ns) * self.K * r) if r > 0 else None for r in self.ranks]
+        dB = [mk(r * sum(self.Ns)) if r > 0 else None for r in self.ranks]
+        return dA, dB
+
+    def split_dA(self, t, dA):
+        r = self.ranks[t]
+        return [to_np(dA[p * self.K * r:(p + 1) * self.K * r]).reshape(self.K, r) for p in range(len(self.Ns))]
+
+    def split_dB(self, t, dB):
+        r, out, o = self.ranks[t], [], 0
+        for N in self.Ns:
+            out.append(to_np(dB[o:o + r * N]).reshape(r, N))
+            o += r * N
+        return out
+
+
+def _oracle_forward(w, ts):
+    ys, hs = [], []
+    for p in w.projections:
+        r, s, A, Bm = oracle.adapters_of(p)
+        y, h = oracle.forward(p.x, p.W, r, s, A, Bm, ts)
+        ys.append(y)
+        hs.append(h)
+    return np.concatenate(ys, axis=1), hs
+
+
+def test_store_roundtrip_of_a_pool_over_three_projections():
+    w = _case(31, 64, 256, (512, 256, 256), (16, 8, 40, 0, 64), True)
+    sc = SegCase(w, capacity=6)
+    assert sc.pool.n_parts == 3
+    for t, r in enumerate(sc.ranks):
+        if r == 0:
+            continue
+        As, Bs = B.marlaas_adapter_pool_export(sc.pool, t, r)
+        for p, proj in enumerate(w.projections):
+            assert np.array_equal(As[p].view(torch.int16).cpu().numpy().view(np.uint16), proj.adapters[t].A_bits)
+            assert np.array_equal(Bs[p].view(torch.int16).cpu().numpy().view(np.uint16), proj.adapters[t].B_bits)
+    # part widths that would let a 256-column tile straddle two projections are refused
+    with pytest.raises(B.MarlaasError):
+        B.AdapterPool(256, 384, 16, 4, parts=[128, 256])
+    B.marlaas_check_status(sc.pool)
+
+
+@pytest.mark.parametrize("T,K,Ns,ranks,per_token,flags", [
+    (200, 256, (512, 256, 256), (16, 16, 32, 8, 64), True, 0),            # q, k, v; decode batch
+    (96, 4096, (8192, 8192), (16, 64, 8), True, 0),                       # gate, up over a large weight (wide decode kernel)
+    (1, 128, (256, 256), (16,), True, 0),                                 # a single token
+    (700, 128, (256, 512), (16, 8, 24, 16), False, 0),                    # training shape below 1024 rows
+    (1500, 192, (256, 256, 512), (16, 32, 8, 64, 16), False, 0),          # training shape, several row tiles
+    (300, 136, (256, 256), (16, 8, 24), False, B.MARLAAS_FLAG_CUDA_CORE_PATH),
+])
+def test_forward_of_a_pool_over_several_projections(T, K, Ns, ranks, per_token, flags):
+    w = _case(900 + T, T, K, Ns, ranks, per_token)
+    ts = w.tok_slot()
+    sc = SegCase(w, capacity=len(ranks) + 1)
+    P = len(Ns)
+    hs = torch.full((P, T, sc.pool.rank_stride), 7.0, dtype=torch.float32, device="cuda:0")
+    y = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs, flags=flags)
+    ry, rh = _oracle_forward(w, ts)
+    assert_close(to_np(y), ry, "y = the projections' outputs side by side")
+    for p in range(P):
+        got = to_np(hs[p])
+        assert_close(got[:, :rh[p].shape[1]], rh[p], f"h of projection {p}", atol=1e-3, rtol=1e-3)
+        assert np.all(got[:, rh[p].shape[1]:] == 0)
+    # the same call again is bit-identical (nothing depends on what the workspace held)
+    y2 = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, flags=flags)
+    assert torch.equal(y, y2)
+    B.marlaas_check_status(sc.pool)
+
+
+@pytest.mark.parametrize("T,K,Ns,ranks,flags,saved", [
+    (1300, 128, (256, 256, 512), (16, 32, 8, 64), 0, True),       # 2-CTA GEMM, gradient reductions on the side stream
+    (1300, 128, (256, 256, 512), (16, 32, 8, 64), 0, False),      # h recomputed
+    (600, 192, (256, 512), (16, 8, 24), 0, True),
+    (150, 64, (256, 256), (16, 8), 0, True),
+    (300, 136, (256, 256), (16, 8, 24), B.MARLAAS_FLAG_CUDA_CORE_PATH, True),
+])
+def test_backward_of_a_pool_over_several_projections(T, K, Ns, ranks, flags, saved):
+    w = _case(1700 + T, T, K, Ns, ranks, False)
+    ts = w.tok_slot()
+    sc = SegCase(w, capacity=len(ranks) + 1)
+    P, n = len(Ns), len(ranks)
+    hs = torch.empty((P, T, sc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+    B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs, flags=flags)
+    dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda:0")
+    dA, dB = sc.grads(fill=3.0)
+    B.marlaas_lora_backward(sc.pool, sc.x, sc.W, sc.dy, sc.seg, dx=dx, dA=dA, dB=dB, h_saved=hs if saved else None, flags=flags)
+    rdx, rdA, rdB = 0.0, [], []
+    for p in w.projections:
+        r, s, A, Bm = oracle.adapters_of(p)
+        rdx = rdx + oracle.backward_dx(p.dy, p.W, r, s, A, Bm, ts)[0]
+        a, b = oracle.backward_dAdB(p.x, p.dy, r, s, A, Bm, ts)
+        rdA.append(a)
+        rdB.append(b)
+    assert_close(to_np(dx), rdx, "dx = sum over the projections")
+    for t in range(n):
+        if ranks[t] == 0:
+            continue
+        gA, gB = sc.split_dA(t, dA[t]), sc.split_dB(t, dB[t])
+        for p in range(P):
+            assert_close(gA[p], rdA[p][t], f"dA of tenant {t}, projection {p}")
+            assert_close(gB[p], rdB[p][t], f"dB of tenant {t}, projection {p}")
+    # accumulate: a second pass adds the same contribution
+    B.marlaas_lora_backward(sc.pool, sc.x, sc.W, sc.dy, sc.seg, dx=None, dA=dA, dB=dB, h_saved=hs if saved else None,
+                            flags=flags | B.MARLAAS_FLAG_ACCUMULATE)
+    for t in range(n):
+        if ranks[t] == 0:
+            continue
+        gA = sc.split_dA(t, dA[t])
+        for p in range(P):
+            assert_close(gA[p], 2 * rdA[p][t], f"accumulated dA of tenant {t}, projection {p}", atol=2e-2)
+    B.marlaas_check_status(sc.pool)
+
+
+def test_adamw_commit_on_a_pool_over_two_projections():
+    T, K, Ns, ranks = 64, 128, (256, 512), (16, 8)
+    w = _case(77, T, K, Ns, ranks, True)
+    sc = SegCase(w, capacity=3)
+    rng = np.random.default_rng(5)
+    ids = [w.projections[0].adapters[t].tenant_id for t in range(2)]
+    tabs = {k: [] for k in ("dA", "dB", "A", "B", "mA", "vA", "mB", "vB")}
+    ref = []
+    for t, r in enumerate(ranks):
+        nA, nB = len(Ns) * K * r, r * sum(Ns)
+        host = {"dA": rng.standard_normal(nA), "dB": rng.standard_normal(nB), "A": rng.standard_normal(nA) * 0.1,
+                "B": rng.standard_normal(nB) * 0.1, "mA": np.zeros(nA), "vA": np.zeros(nA), "mB": np.zeros(nB), "vB": np.zeros(nB)}
+        for k, v in host.items():
+            tabs[k].append(torch.from_numpy(v.astype(np.float32)).cuda())
+        ref.append({k: v.astype(np.float32).astype(np.float64) for k, v in host.items()})
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01, grad_scale=0.5, step=1)
+    B.marlaas_adapter_pool_adamw_commit(sc.pool, ids, tabs["dA"], tabs["dB"], tabs["A"], tabs["B"], tabs["mA"], tabs["vA"],
+                                        tabs["mB"], tabs["vB"], **hp)
+    for t, r in enumerate(ranks):
+        As, Bs = B.marlaas_adapter_pool_export(sc.pool, t, r)
+        newA = oracle.adamw_step(ref[t]["A"], ref[t]["dA"], ref[t]["mA"], ref[t]["vA"], **hp)[0]
+        newB = oracle.adamw_step(ref[t]["B"], ref[t]["dB"], ref[t]["mB"], ref[t]["vB"], **hp)[0]
+        assert_close(to_np(tabs["A"][t]), newA, "fp32 master A", atol=1e-5, rtol=1e-5)
+        assert_close(to_np(tabs["B"][t]), newB, "fp32 master B", atol=1e-5, rtol=1e-5)
+        # the store holds the bf16 rounding of the new masters, block by block
+        gotA = torch.cat([a.reshape(-1) for a in As]).float()
+        gotB = torch.cat([b.reshape(-1) for b in Bs]).float()
+        assert torch.equal(gotA, tabs["A"][t].to(torch.bfloat16).float())
+        assert torch.equal(gotB, tabs["B"][t].to(torch.bfloat16).float())
+    B.marlaas_check_status(sc.pool)
