@@ -69,7 +69,7 @@ SWEEPS = {
     "decode": [f"decode-{T}-{n}" for T in (32, 64, 128, 256, 512, 1024) for n in (1, 8, 32)],
     "prefill": [f"prefill-{T}-{n}" for T in (8192, 16384, 32768) for n in (1, 8, 32)],
     # projections that share their input, fused into one call against one call each, on a decode batch
-    "fused": [f"{k}-{T}-32" for T in (64, 256) for k in ("qkv", "qkvsep", "gateup", "gateupsep")],
+    "fused": [f"{k}-{T}-32" for T in (64, 256) for k in ("qkvseg", "qkv", "qkvsep", "gateupseg", "gateup", "gateupsep")],
 }
 
 
@@ -79,9 +79,11 @@ def workload_desc(name):
     if name in wl.VARIANTS:
         return wl.VARIANTS[name]
     kind, T, n = name.split("-")
-    if kind in ("qkv", "qkvsep", "gateup", "gateupsep"):
+    if kind in ("qkv", "qkvsep", "qkvseg", "gateup", "gateupsep", "gateupseg"):
         shape = "q, k, v (4096x4096 each)" if kind.startswith("qkv") else "gate, up (4096x11008 each)"
-        how = "one call each" if kind.endswith("sep") else "fused into one projection (block-diagonal B), one call"
+        how = "one call each" if kind.endswith("sep") else \
+            "one pool over the projections (B side by side), one call" if kind.endswith("seg") else \
+            "fused into one projection (block-diagonal B), one call"
         return f"{shape}, {how}; {n} tenants r=16 per projection, {T} decode tokens, fwd only"
     what = "decode tokens (one per sequence, tenants uniform and unsorted)" if kind == "decode" else \
         "prompt tokens in whole-prompt lognormal segments"
@@ -200,12 +202,13 @@ def algorithmic_work(w):
     out = {"fwd_flops": 0.0, "bwd_flops": 0.0, "fwd_bytes": 0.0, "bwd_bytes": 0.0, "gemm_flops": []}
     for p in w.projections:
         K, N = p.d_in, p.d_out
+        np_ = len(p.parts) if p.parts else 1        # a pool over several projections holds one A per projection
         ranks = np.array([a.rank for a in p.adapters] + [0])
         r_tok = ranks[ts]
         Tb = 0 if p.dy_bits is None else p.dy_bits.shape[0]
         present = np.unique(ts[ts >= 0])
-        ad_bytes = sum(2 * ranks[t] * (K + N) for t in present)
-        out["fwd_flops"] += 2.0 * w.T * K * N + float(np.sum(2.0 * r_tok * (K + N)))
+        ad_bytes = sum(2 * ranks[t] * (np_ * K + N) for t in present)
+        out["fwd_flops"] += 2.0 * w.T * K * N + float(np.sum(2.0 * r_tok * (np_ * K + N)))
         out["fwd_bytes"] += 2.0 * (K * N + w.T * K + w.T * N) + ad_bytes
         out["gemm_flops"].append(2.0 * w.T * K * N + float(np.sum(2.0 * r_tok * N)))
         if Tb:
@@ -510,8 +513,14 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
     def build_copy():
         projs, x_cache = [], {}
         for p in w.projections:
-            pool = B.AdapterPool(p.d_in, p.d_out, w.max_rank, w.n_tenants, device=dev)
+            pool = B.AdapterPool(p.d_in, p.d_out, w.max_rank, w.n_tenants, device=dev, parts=p.parts)
             for a in p.adapters:
+                if p.parts and a.rank > 0:
+                    cuts = np.concatenate([[0], np.cumsum(p.parts)])
+                    B.marlaas_adapter_pool_register(pool, a.tenant_id, 0, a.rank, a.alpha,
+                                                    [dev_bf16(a.A_bits[:, i * a.rank:(i + 1) * a.rank]) for i in range(len(p.parts))],
+                                                    [dev_bf16(a.B_bits[:, cuts[i]:cuts[i + 1]]) for i in range(len(p.parts))])
+                    continue
                 B.marlaas_adapter_pool_register(pool, a.tenant_id, 0, a.rank, a.alpha, dev_bf16(a.A_bits), dev_bf16(a.B_bits))
             key = id(p.x_bits)
             if key not in x_cache:
@@ -520,7 +529,7 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
                 pinned[key] = pinned_bf16(p.x_bits)
             st = {"p": p, "pool": pool, "W": dev_bf16(p.W_bits), "x": x_cache[key], "x_host": pinned[key],
                   "y": torch.empty((w.T, p.d_out), dtype=torch.bfloat16, device=dev),
-                  "h": torch.empty((w.T, pool.rank_stride), dtype=torch.float32, device=dev),
+                  "h": torch.empty((pool.n_parts * w.T, pool.rank_stride), dtype=torch.float32, device=dev),
                   "ws": None}
             ws_bytes[0] = max(ws_bytes[0], B.marlaas_lora_workspace_bytes(pool, w.T))
             if Tb:

@@ -177,6 +177,11 @@ int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool);
 size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
 /* The part of that workspace a forward call uses (its leading bytes): enough for marlaas_lora_forward alone. */
 size_t marlaas_lora_forward_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
+/* The least a forward call accepts (also leading bytes).  The difference to the size above is scratch through which the
+ * decode-shaped kernels for large weights pass partial sums between CTA pairs (up to about 20 MB); a call given less than
+ * the full size runs the kernels that need no such scratch (slower on those shapes; every result still within the
+ * layer's tolerance of the definition). */
+size_t marlaas_lora_forward_workspace_min_bytes(const marlaas_pool_t* pool, int64_t T);
 
 /* Forward: y[T][d_out] = x[T][d_in] W + s_t (x A_t) B_t with t from the segment table.
  * x (ldx >= d_in), W (ldw >= d_out), y (ldy >= d_out): bf16 row-major.  h_save: optional fp32
@@ -216,7 +221,7 @@ marlaas_status_t marlaas_lora_forward_multi(int32_t n, const marlaas_forward_cal
  * array built into the library (marlaas_lora_static_workspace_limit() bytes, 8 MiB, resident on every GPU that
  * loads the library until the process exits) instead of a caller workspace; x, W, y, the pool storage and h_save
  * are still the caller's.  The call itself allocates and frees nothing on the device.
- *  - Batches whose forward scratch (marlaas_lora_forward_workspace_bytes) exceeds the limit are rejected with
+ *  - Batches whose forward scratch (marlaas_lora_forward_workspace_min_bytes) exceeds the limit are rejected with
  *    MARLAAS_ERR_WORKSPACE_TOO_SMALL before anything is launched: 256 tokens on a pool of 32 slots of rank
  *    up to 64 fit.
  *  - The first call on each device looks up the array's device address.  That lookup is also the moment the CUDA

@@ -41,7 +41,7 @@ EXPORTED_SYMBOLS = [
     "marlaas_lora_forward", "marlaas_lora_backward", "marlaas_lora_build_index", "marlaas_check_status",
     "marlaas_last_error", "marlaas_kernel_launch_count", "marlaas_kernel_timing_begin", "marlaas_kernel_timing_end",
     "marlaas_lora_static_workspace_limit", "marlaas_lora_forward_static_ws", "marlaas_adapter_pool_adamw_commit",
-    "marlaas_adapter_pool_storage_bytes_segmented", "marlaas_adapter_pool_create_segmented", "marlaas_adapter_pool_parts",
+    "marlaas_lora_forward_workspace_min_bytes", "marlaas_adapter_pool_storage_bytes_segmented", "marlaas_adapter_pool_create_segmented", "marlaas_adapter_pool_parts",
 ]
 
 
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
     L.marlaas_lora_workspace_bytes.argtypes = [vp, i64]
     L.marlaas_lora_forward_workspace_bytes.restype = sz
     L.marlaas_lora_forward_workspace_bytes.argtypes = [vp, i64]
+    L.marlaas_lora_forward_workspace_min_bytes.restype = sz
+    L.marlaas_lora_forward_workspace_min_bytes.argtypes = [vp, i64]
     L.marlaas_lora_forward.restype = i32
     L.marlaas_lora_forward.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, P(marlaas_segments_t), vp, vp, sz, u32, vp]
     L.marlaas_lora_static_workspace_limit.restype = sz
@@ -314,6 +316,10 @@ def marlaas_lora_workspace_bytes(pool: AdapterPool, T: int) -> int:
 
 def marlaas_lora_forward_workspace_bytes(pool: AdapterPool, T: int) -> int:
     return int(load_library().marlaas_lora_forward_workspace_bytes(pool.handle, T))
+
+
+def marlaas_lora_forward_workspace_min_bytes(pool: AdapterPool, T: int) -> int:
+    return int(load_library().marlaas_lora_forward_workspace_min_bytes(pool.handle, T))
 
 
 def _mat(t: torch.Tensor, cols: int, name: str):

@@ -23,6 +23,7 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
     w.hd = (bf16*)take(sizeof(bf16) * P * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
+    w.fwd_min = o;
     w.xbuf = (float*)take(decode_wide_sm100_xbuf_bytes(pool, (int64_t)Tn));
     w.fwd_total = o;
     w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
@@ -175,6 +176,11 @@ size_t marlaas_lora_forward_workspace_bytes(const marlaas_pool_t* pool, int64_t 
     return carve_workspace(pool, T, nullptr).fwd_total;
 }
 
+size_t marlaas_lora_forward_workspace_min_bytes(const marlaas_pool_t* pool, int64_t T) {
+    if (!pool || T < 0) return 0;
+    return carve_workspace(pool, T, nullptr).fwd_min;
+}
+
 marlaas_status_t marlaas_lora_build_index(marlaas_pool_t* pool, int64_t T, const marlaas_segments_t* seg,
                                           int32_t* tok_slot, int32_t* slot_count, int32_t* slot_offset,
                                           int32_t* perm, void* workspace, size_t workspace_bytes, uint32_t flags,
@@ -219,15 +225,19 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
     if ((rc = check_segments(fn, pool, T, seg, flags, &host_ts)) != MARLAAS_OK) return rc;
     if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
     const Workspace ws = carve_workspace(pool, T, workspace);
-    if (workspace_bytes < ws.fwd_total)
-        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.fwd_total);
+    if (workspace_bytes < ws.fwd_min)
+        return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.fwd_min);
+    // between the minimum and the full forward size the scratch for exchanged partial sums is missing: the decode kernels
+    // that split a contraction over CTA pairs are then left out (same results up to the summation order of those kernels)
+    const bool has_xbuf = workspace_bytes >= ws.fwd_total;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     MARLAAS_CUDA_TRY(cudaSetDevice(pool->device));
     if ((rc = reject_host_table_in_capture(fn, flags, st)) != MARLAAS_OK) return rc;
     if (!launch) return MARLAAS_OK;
 
     float* h = h_save ? h_save : ws.h;
-    if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH) && decode_sm100_eligible(pool, T)) {
+    const bool stream_k = has_xbuf && decode_stream_sm100_eligible(pool, T);
+    if (!(flags & MARLAAS_FLAG_CUDA_CORE_PATH) && (stream_k || decode_sm100_eligible(pool, T))) {
         int32_t S = seg->num_segments;
         if (flags & MARLAAS_FLAG_HOST_TABLE) {
             MARLAAS_CUDA_TRY(cudaMemcpyAsync(ws.tok_slot, host_ts.data(), sizeof(int32_t) * (size_t)T,
@@ -236,7 +246,10 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
         }
         {
             TimedLaunch timed(pool, st);
-            rc = decode_wide_sm100_eligible(pool, T)
+            rc = stream_k
+                     ? launch_decode_stream_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
+                                                  seg->seg_offsets, seg->seg_slot, ws, h, st)
+                 : (decode_wide_sm100_eligible(pool, T) && (has_xbuf || decode_wide_sm100_xbuf_bytes(pool, T) == 0))
                      ? launch_decode_wide_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
                                                 seg->seg_offsets, seg->seg_slot, ws, h, st)
                      : launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,

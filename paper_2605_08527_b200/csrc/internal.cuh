@@ -123,6 +123,8 @@ struct Workspace {
                            //               columns, zeros in the other units of the tile
     int32_t umax;
     float* xbuf;           // decode path with a split contraction: partial sums passed between the slices of a tile
+    size_t fwd_min;        // bytes a forward call cannot do without (the fields above but xbuf: without it the decode
+                           // kernels that exchange partial sums are not used)
     size_t fwd_total;      // bytes a forward call uses (the fields above); the rest serves backward only
     // tensor-core gradient reductions: 64-token blocks, one masked copy of the block's r-vectors per tenant present
     int32_t* blk_np;       // [nblk]        tenants present in the block
@@ -190,6 +192,11 @@ size_t decode_wide_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T);    // 
 marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
                                           int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
                                           const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
+// the same forward when there are more tiles than CTA pairs: the tiles' steps spread evenly over all pairs
+bool decode_stream_sm100_eligible(const marlaas_pool* pool, int64_t T);
+marlaas_status_t launch_decode_stream_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
+                                            int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
+                                            const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);
 constexpr size_t DECODE_SYNC_BYTES = 16384;
 
 marlaas_status_t launch_decode_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,

@@ -54,7 +54,8 @@ marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T,
     if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
     if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
     if (T == 0) return MARLAAS_OK;
-    const size_t need = marlaas_lora_forward_workspace_bytes(pool, T);     // forward's share of the workspace only
+    // forward's share of the workspace, without the scratch only the kernels that exchange partial sums use
+    const size_t need = marlaas_lora_forward_workspace_min_bytes(pool, T);
     if (need == 0 || need > STATIC_WS_BYTES)
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL,
                     "%s: a batch of %lld tokens on this pool needs %zu bytes of scratch, the built-in array holds %zu; "

@@ -129,6 +129,10 @@ class Projection:
     adapters: List[Adapter]
     x_bits: np.ndarray                  # [T][d_in]
     dy_bits: Optional[np.ndarray]       # [T_bwd][d_out] or None (forward-only workload)
+    # Several projections over one input served as one layer (a pool over several projections): their widths.  W and
+    # dy hold them side by side; an adapter of rank r then has A_bits [d_in][P r] (the A's side by side) and B_bits
+    # [r][d_out] (the B's side by side), and output range p pairs columns p r .. (p+1) r of A with its columns of B.
+    parts: Optional[List[int]] = None
 
     @property
     def W(self) -> np.ndarray:
@@ -316,13 +320,16 @@ def make_workload(cfg: int, scale_down: int = 1, seed: Optional[int] = None) -> 
     raise ValueError(f"unknown config {cfg}")
 
 
-def fuse_projections(w: Workload, names: Optional[List[str]] = None) -> Workload:
+def fuse_projections(w: Workload, names: Optional[List[str]] = None, segmented: bool = False) -> Workload:
     """Several projections that read the same x (q, k, v; gate, up) as ONE adapted projection, so that one layer call
     serves them all: the base weights side by side ([d_in][sum d_out]), A_t side by side ([d_in][P r]), B_t block
     diagonal ([P r][sum d_out], block p = B_t of projection p over that projection's output columns, zeros elsewhere).
     Then y = x W + s (x A) B of the fused projection is the concatenation of the P separate layer outputs; the same
     holds for dx (their sum), dA (side by side) and the diagonal blocks of dB.  Needs the same rank and alpha on
-    every projection of a tenant (so that one scale s = alpha / r serves all: the fused adapter gets alpha P)."""
+    every projection of a tenant (so that one scale s = alpha / r serves all: the fused adapter gets alpha P).
+    segmented = True keeps the tenants' B matrices side by side instead ([r][sum d_out], rank r, alpha unchanged) and
+    records the projections' widths in Projection.parts: the layout of a pool over several projections, which stores
+    and streams none of the block-diagonal form's zeros."""
     projs = [p for p in w.projections if names is None or p.name in names]
     assert projs and all(p.d_in == projs[0].d_in and p.x_bits is projs[0].x_bits for p in projs), "projections must share x"
     P = len(projs)
@@ -333,6 +340,10 @@ def fuse_projections(w: Workload, names: Optional[List[str]] = None) -> Workload
         assert all(a.rank == a0.rank and a.alpha == a0.alpha and a.tenant_id == a0.tenant_id for a in parts)
         r = a0.rank
         A_bits = np.concatenate([a.A_bits for a in parts], axis=1)
+        if segmented:
+            adapters.append(Adapter(a0.tenant_id, r, a0.alpha, np.ascontiguousarray(A_bits),
+                                    np.ascontiguousarray(np.concatenate([a.B_bits for a in parts], axis=1))))
+            continue
         B_bits = np.zeros((P * r, int(offs[-1])), dtype=np.uint16)
         for i, a in enumerate(parts):
             B_bits[i * r:(i + 1) * r, offs[i]:offs[i + 1]] = a.B_bits
@@ -340,10 +351,13 @@ def fuse_projections(w: Workload, names: Optional[List[str]] = None) -> Workload
     dy_bits = None if projs[0].dy_bits is None else np.ascontiguousarray(np.concatenate([p.dy_bits for p in projs], axis=1))
     fused = Projection("+".join(p.name for p in projs), projs[0].d_in, int(offs[-1]),
                        np.ascontiguousarray(np.concatenate([p.W_bits for p in projs], axis=1)), adapters, projs[0].x_bits, dy_bits)
+    if segmented:
+        fused.parts = [p.d_out for p in projs]
+        return Workload(w.name + "-fused", w.T, w.T_bwd, w.seg_offsets, w.seg_slot, [fused], w.n_tenants, w.max_rank)
     return Workload(w.name + "-fused", w.T, w.T_bwd, w.seg_offsets, w.seg_slot, [fused], w.n_tenants, P * w.max_rank)
 
 
-SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|gateup|gateupsep)-(\d+)-(\d+)$"
+SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|qkvseg|gateup|gateupsep|gateupseg)-(\d+)-(\d+)$"
 
 # Variants of the configured workloads (same tensors, another pass or another table):
 VARIANTS = {
@@ -409,7 +423,8 @@ def make_named_workload(name: str) -> Workload:
     ``prefill-T-n``  T prompt tokens in whole-prompt segments (lognormal lengths, median 1024, clipped to
                      [128, 4096]) dealt to n tenants in shuffled order;
     ``qkv-T-n`` / ``gateup-T-n``  a decode batch through the fused q+k+v (4096 x 12288) or gate+up (4096 x 22016)
-                     projection, ``qkvsep`` / ``gateupsep`` through the same projections one call each."""
+                     projection (adapters fused block-diagonally), ``qkvsep`` / ``gateupsep`` through the same
+                     projections one call each, ``qkvseg`` / ``gateupseg`` through one pool over the projections."""
     import re
     if name.startswith("cfg") and name[3:].isdigit():
         return make_workload(int(name[3:]))
@@ -421,7 +436,7 @@ def make_named_workload(name: str) -> Workload:
     kind, T, n = m.group(1), int(m.group(2)), int(m.group(3))
     if T < 1 or n < 1 or n > 4096:
         raise ValueError(f"workload {name!r}: need T >= 1 and 1 <= tenants <= 4096")
-    if kind in ("qkv", "qkvsep", "gateup", "gateupsep"):
+    if kind in ("qkv", "qkvsep", "qkvseg", "gateup", "gateupsep", "gateupseg"):
         # projections of a 7B-shaped decoder layer that share their input, on a decode batch: q, k, v 4096 x 4096 or
         # gate, up 4096 x 11008, rank 16 each; "...sep" runs them as separate projections (one call each), without
         # the suffix they are fused into one (fuse_projections)
@@ -435,7 +450,7 @@ def make_named_workload(name: str) -> Workload:
         w = Workload(name, T, 0, offsets, slots, projs, n, 16)
         if kind.endswith("sep"):
             return w
-        f = fuse_projections(w)
+        f = fuse_projections(w, segmented=kind.endswith("seg"))
         f.name = name
         return f
     seed = BASE_SEED + 100 + (0 if kind == "decode" else 1)

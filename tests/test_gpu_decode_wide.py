@@ -1,7 +1,8 @@
 """GPU parity of the decode-shaped forward over large weights (the kernel with W columns on the MMA's M side), which
 only weights of 64 MB and more reach: one case per way it cuts the contraction -- no split (33 or more tiles), two
-slices and four slices (partial accumulators exchanged through the workspace) -- each element-wise against the oracle,
-plus repeated calls on one pool (the exchange flags carry an epoch from call to call) and bit-identity of two runs.
+slices and four slices (partial accumulators exchanged through the workspace), and more tiles than CTA pairs (the tiles'
+steps spread evenly over all pairs, partial tiles summed by the pair holding a tile's last steps) -- each element-wise
+against the oracle, plus repeated calls on one pool (the exchange flags carry an epoch from call to call) and bit-identity of two runs.
 """
 import numpy as np
 import pytest
@@ -30,6 +31,9 @@ def _case(seed, T, K, N, ranks, per_token):
     (802, 70, 11008, 4096, (16, 32, 16), True),            # 16 tiles: four slices of 43 steps each (uneven: 172 = 4 x 43)
     (803, 300, 11008, 4096, (16, 8, 16, 16), False),       # 2 x 16 tiles: two slices; second token tile has 44 rows
     (804, 256, 4096, 8200, (16, 16, 16, 16, 16, 16), True),   # 33 tiles; N not a multiple of 64: per-chunk copies, 8-column tail
+    (805, 90, 2048, 19200, (16, 8, 16, 32), True),         # 75 tiles on 74 pairs: every pair but the first cuts a tile
+    (806, 257, 4096, 11008, (16, 16, 8, 16), False),       # 2 x 43 tiles; the second token tile has one row
+    (807, 40, 1664, 24584, (16, 16), True),                # 97 tiles, N not a multiple of 64, K / 64 = 26 steps: pairs span 2-3 tiles
 ])
 def test_decode_over_large_weights_matches_the_oracle(seed, T, K, N, ranks, per_token):
     w = _case(seed, T, K, N, ranks, per_token)

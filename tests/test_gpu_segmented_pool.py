@@ -105,6 +105,7 @@ def test_store_roundtrip_of_a_pool_over_three_projections():
 @pytest.mark.parametrize("T,K,Ns,ranks,per_token,flags", [
     (200, 256, (512, 256, 256), (16, 16, 32, 8, 64), True, 0),            # q, k, v; decode batch
     (96, 4096, (8192, 8192), (16, 64, 8), True, 0),                       # gate, up over a large weight (wide decode kernel)
+    (64, 2048, (9728, 9728), (16, 32, 8), True, 0),                       # 76 strips on 74 CTA pairs: tiles cut between pairs
     (1, 128, (256, 256), (16,), True, 0),                                 # a single token
     (700, 128, (256, 512), (16, 8, 24, 16), False, 0),                    # training shape below 1024 rows
     (1500, 192, (256, 256, 512), (16, 32, 8, 64, 16), False, 0),          # training shape, several row tiles
