@@ -455,7 +455,9 @@ def main():
         w5 = wl.make_named_workload("cfg5")
         extra("cfg5", w5)
         extra("cfg5-alltenants", wl.make_variant("cfg5-alltenants", w5))
+        extra("cfg5-fused", wl.make_variant("cfg5-fused", w5))
         extra("cfg5-decode", wl.make_variant("cfg5-decode", w5), steps=20, repeats=5)
+        extra("cfg5-decode-fused", wl.make_variant("cfg5-decode-fused", w5), steps=20, repeats=5)
         out["configs"] = configs
     if rank == 0:
         print(json.dumps(out))
@@ -538,7 +540,11 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
                     pinned[id(p.dy_bits)] = pinned_bf16(p.dy_bits)
                 st["dy_host"] = pinned[id(p.dy_bits)]
                 st["dx"] = torch.empty((Tb, p.d_in), dtype=torch.bfloat16, device=dev)
-                st["dA"] = [torch.empty((p.d_in, a.rank), dtype=torch.float32, device=dev) for a in p.adapters]
+                st["dA"] = [torch.empty((pool.n_parts * p.d_in, a.rank), dtype=torch.float32, device=dev) for a in p.adapters]
+                # a pool over several projections keeps h as one plane of T rows per projection: the backward rows (a prefix
+                # of the batch) are gathered into planes of T_bwd rows before the backward call
+                if pool.n_parts > 1 and Tb < w.T:
+                    st["h_b"] = torch.empty((pool.n_parts, Tb, pool.rank_stride), dtype=torch.float32, device=dev)
                 st["dB"] = [torch.empty((a.rank, p.d_out), dtype=torch.float32, device=dev) for a in p.adapters]
             projs.append(st)
         return projs
@@ -589,8 +595,12 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
         if Tb:
             for j, s in enumerate(cs):
                 fl = args.flags | (B.MARLAAS_FLAG_REUSE_PLAN if j > 0 else 0)
+                hb = s["h"][:Tb]
+                if "h_b" in s:
+                    s["h_b"].copy_(s["h"].view(s["pool"].n_parts, w.T, -1)[:, :Tb])
+                    hb = s["h_b"]
                 B.marlaas_lora_backward(s["pool"], x_of(s)[:Tb], s["W"], dy_of(s), seg_b, dx=s["dx"], dA=s["dA"], dB=s["dB"],
-                                        h_saved=s["h"][:Tb], workspace=s["ws"], flags=fl)
+                                        h_saved=hb, workspace=s["ws"], flags=fl)
 
     def barrier():
         if dist is not None:

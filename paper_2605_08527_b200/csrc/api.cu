@@ -13,23 +13,18 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 1);
     auto take = [&](size_t bytes) { char* q = p ? p + o : nullptr; o += align_up(bytes, 256); return q; };
-    // forward's fields first: a forward call needs only the first fwd_total bytes
+    // 1. The plan of the batch (forward and backward): its layout depends on T, the capacity and the rank stride only, so
+    //    that pools of one layer (same capacity and max_rank, whatever their widths and however many projections they hold)
+    //    find one another's plan in a shared workspace (MARLAAS_FLAG_REUSE_PLAN).
     w.tok_slot = (int32_t*)take(sizeof(int32_t) * Tn);
-    const size_t P = (size_t)pool->P;       // a pool over P projections keeps one plane of h, g and hd per projection
-    w.h = (float*)take(sizeof(float) * P * Tn * pool->RP);
     const size_t ntiles = (Tn + 255) / 256;
     w.umax = (pool->cap < 256 ? pool->cap : 256) * (pool->RP / 16);
     w.tok_uoff = (int32_t*)take(sizeof(int32_t) * Tn);
     w.tile_nunits = (int32_t*)take(sizeof(int32_t) * ntiles);
     w.tile_units = (int32_t*)take(sizeof(int32_t) * ntiles * (size_t)w.umax);
-    w.hd = (bf16*)take(sizeof(bf16) * P * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
-    w.fwd_min = o;
-    w.xbuf = (float*)take(decode_wide_sm100_xbuf_bytes(pool, (int64_t)Tn));
-    w.fwd_total = o;
     w.perm = (int32_t*)take(sizeof(int32_t) * Tn);
     w.slot_count = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 1));
     w.slot_offset = (int32_t*)take(sizeof(int32_t) * (size_t)(pool->cap + 2));
-    w.g = (float*)take(sizeof(float) * P * Tn * pool->RP);
     w.dA_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     w.dB_ptrs = (float**)take(sizeof(float*) * (size_t)pool->cap);
     const size_t nblk = (Tn + 63) / 64;
@@ -44,6 +39,15 @@ Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base) {
     w.ten_blks = (int32_t*)take(sizeof(int32_t) * gb * gc);
     w.ten_pos = (int32_t*)take(sizeof(int32_t) * gb * gc);
     w.gflag = (int32_t*)take(16);
+    // 2. What a forward call writes besides: a pool over P projections keeps one plane of h and hd per projection.
+    const size_t P = (size_t)pool->P;
+    w.h = (float*)take(sizeof(float) * P * Tn * pool->RP);
+    w.hd = (bf16*)take(sizeof(bf16) * P * Tn * align_up((size_t)w.umax * 16, 64));   // decode path: pitch in whole 64-column panels
+    w.fwd_min = o;
+    w.xbuf = (float*)take(decode_wide_sm100_xbuf_bytes(pool, (int64_t)Tn));
+    w.fwd_total = o;
+    // 3. Backward only.
+    w.g = (float*)take(sizeof(float) * P * Tn * pool->RP);
     w.hm = (bf16*)take(sizeof(bf16) * (size_t)w.max_copies * 64 * (size_t)w.HW);
     w.hm2 = (bf16*)take(sizeof(bf16) * (size_t)w.max_copies * 64 * (size_t)w.HW);
     w.total = o;

@@ -365,7 +365,17 @@ VARIANTS = {
     "cfg3-alltenants": "cfg3 with a table of the same recipe in which all 10 tenants appear (13 to 16 segments)",
     "cfg5-decode": "the decode part of cfg5 alone: its 256 decode tokens through the 7 projections, forward only",
     "cfg5-alltenants": "cfg5 whose 4096 training rows hold all 32 tenants (same recipe, lengths divided by 8)",
+    "cfg5-fused": "cfg5 with q, k, v and gate, up each served by one pool over the projections (4 calls per pass instead of 7)",
+    "cfg5-decode-fused": "cfg5-decode with q, k, v and gate, up each served by one pool over the projections",
 }
+
+
+def _fuse_layer(w: Workload, name: str) -> Workload:
+    """q, k, v and gate, up of a decoder-layer workload as one projection each (a pool over the projections)."""
+    by = {p.name: p for p in w.projections}
+    projs = [fuse_projections(w, ["q", "k", "v"], segmented=True).projections[0], by["o"],
+             fuse_projections(w, ["gate", "up"], segmented=True).projections[0], by["down"]]
+    return Workload(name, w.T, w.T_bwd, w.seg_offsets, w.seg_slot, projs, w.n_tenants, w.max_rank)
 
 
 def _table_with_all_tenants(seed: int, T: int, n: int, shrink: int, lo: int, hi: int):
@@ -384,6 +394,10 @@ def make_variant(name: str, base: Optional[Workload] = None) -> Workload:
         raise ValueError(f"unknown variant {name!r}")
     cfg = int(name[3])
     w = base if base is not None else make_workload(cfg)
+    if name == "cfg5-fused":
+        return _fuse_layer(w, name)
+    if name == "cfg5-decode-fused":
+        return _fuse_layer(make_variant("cfg5-decode", w), name)
     if name == "cfg3-fwd":
         projs = [dataclasses.replace(p, dy_bits=None) for p in w.projections]
         return Workload(name, w.T, 0, w.seg_offsets, w.seg_slot, projs, w.n_tenants, w.max_rank)

@@ -204,3 +204,68 @@ def test_adamw_commit_on_a_pool_over_two_projections():
         assert torch.equal(gotA, tabs["A"][t].to(torch.bfloat16).float())
         assert torch.equal(gotB, tabs["B"][t].to(torch.bfloat16).float())
     B.marlaas_check_status(sc.pool)
+
+
+def test_plan_shared_between_a_pool_over_two_projections_and_a_plain_pool():
+    # One layer, one mixed batch, one workspace: the pool over (p0, p1) builds the plan, the plain pool of p2 reuses it
+    # (forward and backward), then the other way round.  The plan's place in the workspace must not depend on how many
+    # projections a pool holds.
+    from helpers import DeviceCase
+    T, K, Ns, ranks = 1300, 128, (256, 512, 384), (16, 8, 16, 16)
+    w = _case(2100, T, K, Ns, ranks, False)
+    ts = w.tok_slot()
+    import copy
+    w2 = copy.copy(w)
+    w2.projections = w.projections[:2]
+    sc = SegCase(w2, capacity=len(ranks) + 1)
+    p2 = w.projections[2]
+    dc = DeviceCase(w, p2, capacity=len(ranks) + 1, max_rank=max(ranks))
+    ws = torch.empty(max(B.marlaas_lora_workspace_bytes(sc.pool, T), B.marlaas_lora_workspace_bytes(dc.pool, T)),
+                     dtype=torch.uint8, device="cuda:0")
+    r2, s2, A2, B2 = oracle.adapters_of(p2)
+    ry2 = oracle.forward(p2.x, p2.W, r2, s2, A2, B2, ts)[0]
+    rdx2 = oracle.backward_dx(p2.dy, p2.W, r2, s2, A2, B2, ts)[0]
+    rdA2, rdB2 = oracle.backward_dAdB(p2.x, p2.dy, r2, s2, A2, B2, ts)
+    ry01 = _oracle_forward(w2, ts)[0]
+    for first_seg in (True, False):
+        hs_s = torch.empty((2, T, sc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+        hs_p = torch.empty((T, dc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+        ws.fill_(0x5a)
+        fl = lambda second: B.MARLAAS_FLAG_REUSE_PLAN if second else 0
+        if first_seg:
+            y01 = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs_s, workspace=ws, flags=fl(False))
+            y2 = B.marlaas_lora_forward(dc.pool, dc.x, dc.W, dc.seg, h_save=hs_p, workspace=ws, flags=fl(True))
+        else:
+            y2 = B.marlaas_lora_forward(dc.pool, dc.x, dc.W, dc.seg, h_save=hs_p, workspace=ws, flags=fl(False))
+            y01 = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs_s, workspace=ws, flags=fl(True))
+        assert_close(to_np(y01), ry01, "pool over two projections, shared plan: y")
+        assert_close(to_np(y2), ry2, "plain pool, shared plan: y")
+        dx2 = torch.empty((T, K), dtype=torch.bfloat16, device="cuda:0")
+        dA2, dB2 = dc.grads(fill=1.0)
+        dxs = torch.empty((T, K), dtype=torch.bfloat16, device="cuda:0")
+        dAs, dBs = sc.grads(fill=1.0)
+        calls = [lambda f: B.marlaas_lora_backward(sc.pool, sc.x, sc.W, sc.dy, sc.seg, dx=dxs, dA=dAs, dB=dBs, h_saved=hs_s,
+                                                   workspace=ws, flags=f),
+                 lambda f: B.marlaas_lora_backward(dc.pool, dc.x, dc.W, dc.dy, dc.seg, dx=dx2, dA=dA2, dB=dB2, h_saved=hs_p,
+                                                   workspace=ws, flags=f)]
+        if not first_seg:
+            calls.reverse()
+        calls[0](fl(False))
+        calls[1](fl(True))
+        assert_close(to_np(dx2), rdx2, "plain pool, shared plan: dx")
+        for t in range(len(ranks)):
+            assert_close(to_np(dA2[t]), rdA2[t], f"plain pool, shared plan: dA[{t}]")
+            assert_close(to_np(dB2[t]), rdB2[t], f"plain pool, shared plan: dB[{t}]")
+        rdx = 0.0
+        for p in w2.projections:
+            r, s, A, Bm = oracle.adapters_of(p)
+            rdx = rdx + oracle.backward_dx(p.dy, p.W, r, s, A, Bm, ts)[0]
+        assert_close(to_np(dxs), rdx, "pool over two projections, shared plan: dx")
+        for pi, p in enumerate(w2.projections):
+            r, s, A, Bm = oracle.adapters_of(p)
+            rdA, rdB = oracle.backward_dAdB(p.x, p.dy, r, s, A, Bm, ts)
+            for t in range(len(ranks)):
+                assert_close(sc.split_dA(t, dAs[t])[pi], rdA[t], f"pool over two projections, shared plan: dA[{t}] of {pi}")
+                assert_close(sc.split_dB(t, dBs[t])[pi], rdB[t], f"pool over two projections, shared plan: dB[{t}] of {pi}")
+    B.marlaas_check_status(sc.pool)
+    B.marlaas_check_status(dc.pool)
