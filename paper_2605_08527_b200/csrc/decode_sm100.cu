@@ -384,8 +384,8 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int n0 = ((int)dk_cluster_id_x() % g.nstrips) * NP;
     const int m0 = ((int)dk_cluster_id_x() / g.nstrips) * 256;      // first row of the cluster's token tile
     const int my_m = m0 + (int)half * 128, my_n = n0 + (int)half * 64 * g.nch;
-    int part = 0;
-    while (part < g.parts - 1 && n0 >= g.part_end[part]) ++part;
+    // the projection whose columns the strip lies in (constant indices: a variable one would move the arguments to local memory)
+    const int part = (g.parts > 1 ? (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]) : 0);
     const int xa_m = my_m + part * g.T;         // this half's rows of the projection's plane of hd
 
     const int ks0 = (int)pairi * g.num_ks / g.S, ks1 = ((int)pairi + 1) * g.num_ks / g.S;

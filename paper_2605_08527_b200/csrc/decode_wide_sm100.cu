@@ -143,8 +143,8 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const int n0 = (tile % g.nstrips) * DG_TM;
     const int m0 = (tile / g.nstrips) * DG_TN;
     const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
-    int part = 0;
-    while (part < g.parts - 1 && n0 >= g.part_end[part]) ++part;
+    // the projection whose columns the strip lies in (constant indices: a variable one would move the arguments to local memory)
+    const int part = (g.parts > 1 ? (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]) : 0);
     const int hd_tok = my_tok + part * g.T;          // this half's rows of the projection's plane of hd
     const int ks0 = sl * g.num_ks / g.S, ks1 = (sl + 1) * g.num_ks / g.S;
     const int xs0 = sl * g.num_xs / g.S, xs1 = (sl + 1) * g.num_xs / g.S;
@@ -495,8 +495,7 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
             while (ok && pi.next(tile, s0, s1)) {
                 const int n0 = (tile % g.nstrips) * DG_TM, m0 = (tile / g.nstrips) * DG_TN;
                 const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
-                int part = 0;
-                while (part < g.parts - 1 && n0 >= g.part_end[part]) ++part;
+                const int part = (g.parts > 1 ? (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]) : 0);
                 const int hd_tok = my_tok + part * g.T;
                 auto x_tx = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? X_BYTES : 0u; };
                 auto w_chunks = [&](int r) -> int { return max(0, min(2, (g.Nout - (n0 + r * 128) + 63) / 64)); };
@@ -797,10 +796,11 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
         tmXW = tmW;
     }
 
-    static bool attrs_set[64] = {};
-    if (pool->device >= 64 || !attrs_set[pool->device]) {
-        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        if (pool->device < 64) attrs_set[pool->device] = true;
+    // the largest dynamic shared memory asked for so far on the device (raised when a call needs more)
+    static size_t smem_set[64] = {};
+    if (pool->device >= 64 || smem_set[pool->device] < smem_bytes) {
+        MARLAAS_CUDA_TRY(cudaFuncSetAttribute(k_decode_gemm_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
+        if (pool->device < 64) smem_set[pool->device] = smem_bytes;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * shape.pairs));

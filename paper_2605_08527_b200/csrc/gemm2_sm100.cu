@@ -48,8 +48,8 @@ __device__ __forceinline__ void tile_parts(const Gemm2Args& g, int n0, int& p_lo
     p_hi = 1;
     if (g.parts > 1) {
         if (g.all_parts) p_hi = g.parts;
-        else {
-            while (p_lo < g.parts - 1 && n0 >= g.part_end[p_lo]) ++p_lo;
+        else {      // constant indices: a variable one would move the kernel's arguments to local memory
+            p_lo = (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]);
             p_hi = p_lo + 1;
         }
     }

@@ -331,7 +331,8 @@ def fuse_projections(w: Workload, names: Optional[List[str]] = None, segmented: 
     records the projections' widths in Projection.parts: the layout of a pool over several projections, which stores
     and streams none of the block-diagonal form's zeros."""
     projs = [p for p in w.projections if names is None or p.name in names]
-    assert projs and all(p.d_in == projs[0].d_in and p.x_bits is projs[0].x_bits for p in projs), "projections must share x"
+    assert projs and all(p.d_in == projs[0].d_in and (p.x_bits is projs[0].x_bits or np.array_equal(p.x_bits, projs[0].x_bits))
+                         for p in projs), "projections must share x"
     P = len(projs)
     offs = np.concatenate([[0], np.cumsum([p.d_out for p in projs])]).astype(np.int64)
     adapters = []
