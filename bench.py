@@ -443,6 +443,7 @@ def main():
         configs = {}
 
         def extra(name, wk, steps=10, repeats=3):
+            time.sleep(1.0)     # the sustained leg ran into the power cap: let the clocks come back before a burst measurement
             t0 = time.time()
             d = measure(ctx, args, wk, name, steps, 3, repeats, 0, False)
             configs[name] = summarize(d, time.time() - t0)

@@ -107,6 +107,7 @@ def test_store_roundtrip_of_a_pool_over_three_projections():
     (96, 4096, (8192, 8192), (16, 64, 8), True, 0),                       # gate, up over a large weight (wide decode kernel)
     (64, 2048, (9728, 9728), (16, 32, 8), True, 0),                       # 76 strips on 74 CTA pairs: tiles cut between pairs
     (1, 128, (256, 256), (16,), True, 0),                                 # a single token
+    (333, 192, (256, 512, 256), (16, 0, 40, 8), True, 0),                 # a registered tenant of rank 0 (base weight only)
     (700, 128, (256, 512), (16, 8, 24, 16), False, 0),                    # training shape below 1024 rows
     (1500, 192, (256, 256, 512), (16, 32, 8, 64, 16), False, 0),          # training shape, several row tiles
     (300, 136, (256, 256), (16, 8, 24), False, B.MARLAAS_FLAG_CUDA_CORE_PATH),
@@ -135,6 +136,7 @@ def test_forward_of_a_pool_over_several_projections(T, K, Ns, ranks, per_token, 
     (1300, 128, (256, 256, 512), (16, 32, 8, 64), 0, False),      # h recomputed
     (600, 192, (256, 512), (16, 8, 24), 0, True),
     (150, 64, (256, 256), (16, 8), 0, True),
+    (1100, 128, (512, 256), (16, 0, 24, 8), 0, True),             # a tenant of rank 0: no gradient arrays, base-only rows
     (300, 136, (256, 256), (16, 8, 24), B.MARLAAS_FLAG_CUDA_CORE_PATH, True),
 ])
 def test_backward_of_a_pool_over_several_projections(T, K, Ns, ranks, flags, saved):
