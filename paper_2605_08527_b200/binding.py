@@ -242,7 +242,7 @@ class AdapterPool:
 
 def marlaas_adapter_pool_register(pool: AdapterPool, tenant_id: int, version: int, rank: int, alpha: float,
                                   A: Optional[torch.Tensor], B: Optional[torch.Tensor], stream=None) -> int:
-    if rank > 0 and pool.n_parts > 1:
+    if rank > 0 and pool.parts is not None:
         # one pair per projection, handed to the library as blocks one after another
         assert len(A) == pool.n_parts and len(B) == pool.n_parts
         for p in range(pool.n_parts):
@@ -300,7 +300,7 @@ def marlaas_adapter_pool_export(pool: AdapterPool, slot: int, rank: int, stream=
     A = torch.empty((pool.n_parts * pool.d_in, rank), dtype=torch.bfloat16, device=pool.device)
     B = torch.empty(rank * pool.d_out, dtype=torch.bfloat16, device=pool.device)
     _check(load_library().marlaas_adapter_pool_export(pool.handle, slot, _dptr(A), _dptr(B), _stream(stream)))
-    if pool.n_parts == 1:
+    if pool.parts is None:
         return A, B.view(rank, pool.d_out)
     As = [A[p * pool.d_in:(p + 1) * pool.d_in] for p in range(pool.n_parts)]
     Bs, o = [], 0

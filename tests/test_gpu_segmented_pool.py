@@ -271,3 +271,58 @@ def test_plan_shared_between_a_pool_over_two_projections_and_a_plain_pool():
                 assert_close(sc.split_dB(t, dBs[t])[pi], rdB[t], f"pool over two projections, shared plan: dB[{t}] of {pi}")
     B.marlaas_check_status(sc.pool)
     B.marlaas_check_status(dc.pool)
+
+
+def _draw_seg(rng):
+    kind = rng.choice(["decode", "mid", "train"])
+    P = int(rng.integers(1, 5))
+    Ns = tuple(256 * int(rng.integers(1, 4)) for _ in range(P))
+    if kind == "decode":
+        T, K = int(rng.integers(1, 257)), 64 * int(rng.integers(1, 7))
+    elif kind == "mid":
+        T, K = int(rng.integers(257, 1025)), 8 * int(rng.integers(4, 40))
+    else:
+        T, K = int(rng.integers(1024, 2300)), 8 * int(rng.integers(8, 40))
+    n = int(rng.integers(1, 7))
+    ranks = [int(rng.choice([0, 1, 4, 8, 16, 17, 32, 48, 64])) for _ in range(n)]
+    if max(ranks) == 0:
+        ranks[0] = 8
+    return kind, T, K, Ns, ranks, int(rng.integers(1, 1 << 30)), bool(rng.integers(0, 2)), int(rng.integers(1, 10)), \
+        int(rng.integers(0, 3)), bool(rng.integers(0, 2))
+
+
+@pytest.mark.parametrize("batch", range(2))
+def test_random_pools_over_several_projections_match_the_oracle(batch):
+    # seeded random draws of the number and widths of the projections, token count, depth, rank mix (rank 0 and odd
+    # ranks included), table form, spare capacity, backward with and without the saved h; every output against the
+    # per-projection oracle runs
+    rng = np.random.default_rng(77100 + batch)
+    for ci in range(12):
+        kind, T, K, Ns, ranks, seed, per_token, nseg, extra, use_saved = _draw_seg(rng)
+        w = _case(seed % 100000, T, K, Ns, ranks, per_token, n_segments=nseg)
+        tag = f"batch {batch} case {ci} ({kind}) T={T} K={K} Ns={Ns} ranks={ranks} per_token={per_token} seed={seed}"
+        ts = w.tok_slot()
+        sc = SegCase(w, capacity=len(ranks) + extra)
+        P, n = len(Ns), len(ranks)
+        hs = torch.full((P, T, sc.pool.rank_stride), 9.0, dtype=torch.float32, device="cuda:0")
+        y = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs)
+        ry, rh = _oracle_forward(w, ts)
+        assert_close(to_np(y), ry, tag + ": y")
+        for p in range(P):
+            hr = np.zeros((T, sc.pool.rank_stride), np.float32)
+            hr[:, :rh[p].shape[1]] = rh[p]
+            assert_close(to_np(hs[p]), hr, tag + f": h_save of projection {p}", atol=1e-3, rtol=1e-3)
+        dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda:0")
+        dA, dB = sc.grads(fill=2.0)
+        B.marlaas_lora_backward(sc.pool, sc.x, sc.W, sc.dy, sc.seg, dx=dx, dA=dA, dB=dB, h_saved=hs if use_saved else None)
+        rdx = 0.0
+        for pi, p in enumerate(w.projections):
+            r, s, A, Bm = oracle.adapters_of(p)
+            rdx = rdx + oracle.backward_dx(p.dy, p.W, r, s, A, Bm, ts)[0]
+            rdA, rdB = oracle.backward_dAdB(p.x, p.dy, r, s, A, Bm, ts)
+            for t in range(n):
+                if ranks[t] > 0:
+                    assert_close(sc.split_dA(t, dA[t])[pi], rdA[t], tag + f": dA[{t}] of projection {pi}")
+                    assert_close(sc.split_dB(t, dB[t])[pi], rdB[t], tag + f": dB[{t}] of projection {pi}")
+        assert_close(to_np(dx), rdx, tag + ": dx")
+        B.marlaas_check_status(sc.pool)
