@@ -92,3 +92,64 @@ def test_cfg5_decoder_layer_full_size():
     for p in w.projections:
         _check_full(w, p, n_rows=24)
         torch.cuda.empty_cache()
+
+
+def _check_fused_full(w, names, n_rows=24):
+    """Projections `names` of the layer through ONE pool over them, at the full size: sampled rows of y and dx over all
+    columns, the adapter gradients of every projection in full."""
+    import copy
+    from test_gpu_segmented_pool import SegCase
+    w2 = copy.copy(w)
+    w2.projections = [p for p in w.projections if p.name in names]
+    assert all(np.array_equal(p.x_bits, w2.projections[0].x_bits) for p in w2.projections)
+    sc = SegCase(w2)
+    ts = w.tok_slot()
+    T, Tb, P = w.T, w.T_bwd, len(w2.projections)
+    tag = f"{w.name}/{'+'.join(names)} through one pool"
+    hs = torch.empty((P, T, sc.pool.rank_stride), dtype=torch.float32, device="cuda:0")
+    y = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg, h_save=hs)
+    rows = _sample_rows(T, n_rows, 11 + P)
+    ridx = torch.from_numpy(rows).cuda()
+    ry = []
+    for pi, p in enumerate(w2.projections):
+        r, s, A, Bm = oracle.adapters_of(p)
+        yy, rh = oracle.forward(p.x[rows], p.W, r, s, A, Bm, ts[rows])
+        ry.append(yy)
+        hr = np.zeros((len(rows), sc.pool.rank_stride), np.float32)
+        hr[:, :rh.shape[1]] = rh
+        assert_close(to_np(hs[pi][ridx]), hr, f"{tag}: h_save of {p.name} (sampled rows)", atol=1e-3, rtol=1e-3)
+    assert_close(to_np(y[ridx]), np.concatenate(ry, axis=1), f"{tag}: y (sampled rows)")
+    if Tb:
+        so, ss = w.seg_offsets, w.seg_slot
+        keep = [s_ for s_ in range(len(ss)) if so[s_] < Tb]
+        seg = B.Segments(torch.from_numpy(np.array([min(int(so[s_]), Tb) for s_ in keep] + [Tb], dtype=np.int32)).cuda(),
+                         torch.from_numpy(np.array([ss[s_] for s_ in keep], dtype=np.int32)).cuda())
+        dx = torch.empty((Tb, sc.K), dtype=torch.bfloat16, device="cuda:0")
+        dA, dB = sc.grads()
+        B.marlaas_lora_backward(sc.pool, sc.x[:Tb], sc.W, sc.dy[:Tb], seg, dx=dx, dA=dA, dB=dB, h_saved=hs[:, :Tb].contiguous())
+        rb = rows[rows < Tb]
+        rdx = 0.0
+        for pi, p in enumerate(w2.projections):
+            r, s, A, Bm = oracle.adapters_of(p)
+            rdx = rdx + oracle.backward_dx(p.dy[rb], p.W, r, s, A, Bm, ts[rb])[0]
+            rdA, rdB = oracle.backward_dAdB(p.x[:Tb], p.dy[:Tb], r, s, A, Bm, ts[:Tb])
+            for t, a in enumerate(p.adapters):
+                if a.rank > 0:
+                    assert_close(sc.split_dA(t, dA[t])[pi], rdA[t], f"{tag}: dA[{t}] of {p.name}")
+                    assert_close(sc.split_dB(t, dB[t])[pi], rdB[t], f"{tag}: dB[{t}] of {p.name}")
+        assert_close(to_np(dx[torch.from_numpy(rb).cuda()]), rdx, f"{tag}: dx (sampled rows)")
+    B.marlaas_check_status(sc.pool)
+
+
+def test_cfg5_layer_through_pools_over_projections_full_size():
+    # the configurations bench.py reports as cfg5-fused and cfg5-decode-fused: q, k, v and gate, up through one pool each,
+    # on the mixed training + decode batch (forward over 4352 rows, backward over 4096) and on the 256 decode rows alone
+    # (48 and 86 column strips: the one-tile-per-pair and the balanced decode kernels)
+    w = wl.make_workload(5)
+    for names in (("q", "k", "v"), ("gate", "up")):
+        _check_fused_full(w, names)
+        torch.cuda.empty_cache()
+    wd = wl.make_variant("cfg5-decode", w)
+    for names in (("q", "k", "v"), ("gate", "up")):
+        _check_fused_full(wd, names, n_rows=64)
+        torch.cuda.empty_cache()
