@@ -14,14 +14,15 @@ constexpr int SS_SUB_UNITS = 8;                              // units per work i
 constexpr int SS_KP = 2;                                     // 64-deep panels per pipeline step
 constexpr uint32_t SS_STEP_BYTES = SS_KP * (A_STAGE_BYTES + SS_SUB_UNITS * UNIT_BYTES);   // 64 KB
 constexpr int SS_MAX_C = 8;
-constexpr int SS_MAX_STAGES = 4;
+constexpr int SS_MAX_STAGES = 8;
 constexpr int SS_MAX_TILES = 160;
 
 struct ShrinkSplitArgs {
     int T, D;
     int num_kb, num_m_tiles;
     int RP, cap;
-    int C, stages;
+    int C;
+    uint32_t stage_area;   // bytes of shared memory for the pipeline stages (and, between items, the gather buffer)
     const int32_t* tok_slot;
     const int32_t* tok_uoff;
     const int32_t* tile_nunits;
@@ -96,8 +97,13 @@ __device__ __forceinline__ int ss_plan_runs(const int32_t* units, int nug, UnitR
 // 64 k), so a tile that mixes many tenants is spread over several clusters instead of holding everyone up.  The
 // clusters walk the item list with a fixed stride; every CTA derives the same list from the per-tile unit counts.
 //
-// Shared memory: [stages x kp x (A panel 16 KB + unit slab 16 KB)] [gather buffer C x 128 rows x 128 floats]
-// [barriers] (the gather buffer is used in the cluster's first CTA only; every CTA reserves it).
+// Shared memory: [pipeline stages] [barriers].  What an SM takes in from HBM is its bytes in flight over the memory
+// latency (about 2 us beside 135 other streaming CTAs), so shared memory is spent on stages and on nothing else:
+//  - a stage is kp x (A panel 16 KB + the item's OWN unit slab, 2 KB per unit), so an item with one or two units (the
+//    common case) runs 5-6 stages deep where a slab sized for 8 units allowed 2-3; the stage count is per item (the
+//    pipeline is drained between items anyway), and each role keeps the phase of every stage barrier in a bit mask;
+//  - the gather buffer (C x 128 rows x RP floats, in the cluster's first CTA) lies over the stages: once every CTA of the
+//    cluster has seen its last MMA complete (one more cluster barrier per item) nothing touches them until the next item.
 __global__ void __launch_bounds__(SS_THREADS, 1)
 k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ StoreMaps tmStore,
                      const ShrinkSplitArgs g) {
@@ -112,13 +118,9 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
     const uint32_t crank = ss_cluster_ctarank();
     const int cid = (int)ss_cluster_id_x(), ncl = (int)(gridDim.x / g.C);
 
-    const int STAGES = g.stages;
-    const uint32_t sA = smem_u32(smem);
-    const uint32_t sB = sA + STAGES * A_STEP;
-    const uint32_t stage_area = (uint32_t)STAGES * (A_STEP + B_STEP);
-    const uint32_t sG = sA + stage_area;
-    const uint32_t gather_bytes = (uint32_t)g.C * 128u * (uint32_t)g.RP * 4u;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + stage_area + gather_bytes);
+    const uint32_t sS = smem_u32(smem);
+    const uint32_t sG = sS;       // the gather buffer lies over the stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + g.stage_area);
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * SS_MAX_STAGES;
     const uint32_t bar_tfull = bar_empty + 8 * SS_MAX_STAGES;
@@ -127,7 +129,7 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
     volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < SS_MAX_STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
@@ -177,8 +179,8 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
     const int ks0 = (int)((int64_t)crank * num_steps / g.C), ks1 = (int)((int64_t)(crank + 1) * num_steps / g.C);
 
     // role-local pipeline state lives across items
-    uint32_t p_s = 0, p_ph = 0, p_it = 0;     // producer
-    uint32_t m_s = 0, m_ph = 0;               // MMA issuer
+    uint32_t p_mask = 0, p_issued = 0, p_stages = 1;     // producer: phase bit of every stage's next use; loads of this item
+    uint32_t m_mask = 0;                                 // MMA issuer: likewise
     uint32_t done = 0;                        // items finished by this cluster (parity of bar_tfull)
     bool ok = true;
 
@@ -193,6 +195,9 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         const int nun = g.tile_nunits[m >> 1];
         const int nug = min(SS_SUB_UNITS, nun - u0);
         const int32_t* units = g.tile_units + (size_t)(m >> 1) * g.umax + u0;
+        // this item's stage geometry
+        const uint32_t b_panel = (uint32_t)nug * UNIT_BYTES, stage_bytes = KP * (A_STAGE_BYTES + b_panel);
+        const uint32_t nst = min((uint32_t)SS_MAX_STAGES, g.stage_area / stage_bytes);
 
         // per-row routing (epilogue threads): the row's units within the tile's list
         const int q = warp & 3;
@@ -213,30 +218,36 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         if (warp == 0) {
             if (lane == 0 && ok) {   // ---- TMA producer: this CTA's slice of the contraction
                 const int nruns = ss_plan_runs(units, nug, s_runs);
-                for (int ks = ks0; ks < ks1 && ok; ++ks, ++p_it) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * p_s, p_ph ^ 1, abort_word, 51))) break;
+                uint32_t p_s = 0;
+                p_issued = 0;
+                p_stages = nst;
+                for (int ks = ks0; ks < ks1 && ok; ++ks) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * p_s, ((p_mask >> p_s) & 1u) ^ 1u, abort_word, 51))) break;
                     const uint32_t full = bar_full + 8 * p_s;
-                    mbar_expect_tx(full, A_STEP + KP * nug * UNIT_BYTES);
-                    tma_load_3d(sA + p_s * A_STEP, &tmSrc, full, 0, m * BM, ks * KP);
+                    const uint32_t a0 = sS + p_s * stage_bytes, b0 = a0 + A_STEP;
+                    mbar_expect_tx(full, A_STEP + KP * b_panel);
+                    tma_load_3d(a0, &tmSrc, full, 0, m * BM, ks * KP);
                     for (int p = 0; p < KP; ++p)
                         for (int i = 0; i < nruns; ++i)
-                            tma_load_2d(sB + p_s * B_STEP + p * B_PANEL + s_runs[i].pos * UNIT_BYTES, &tmStore.m[s_runs[i].lg],
+                            tma_load_2d(b0 + p * b_panel + s_runs[i].pos * UNIT_BYTES, &tmStore.m[s_runs[i].lg],
                                         full, (ks * KP + p) * BK, s_runs[i].row);
-                    if (++p_s == (uint32_t)STAGES) { p_s = 0; p_ph ^= 1; }
+                    p_mask ^= 1u << p_s;
+                    ++p_issued;
+                    if (++p_s == nst) p_s = 0;
                 }
             }
             __syncwarp();
         } else if (warp == 1) {
             if (lane == 0 && ok) {   // ---- MMA issuer
                 const uint32_t idesc = make_idesc(nug * 16, 0);
-                uint32_t acc = 0;
+                uint32_t acc = 0, m_s = 0;
                 for (int ks = ks0; ks < ks1 && ok; ++ks) {
-                    if (!(ok = mbar_wait(bar_full + 8 * m_s, m_ph, abort_word, 54))) break;
+                    if (!(ok = mbar_wait(bar_full + 8 * m_s, (m_mask >> m_s) & 1u, abort_word, 54))) break;
                     tc_fence_after();
-                    const uint32_t a0 = sA + m_s * A_STEP, b0 = sB + m_s * B_STEP;
+                    const uint32_t a0 = sS + m_s * stage_bytes, b0 = a0 + A_STEP;
 #pragma unroll
                     for (int p = 0; p < KP; ++p) {
-                        const uint64_t da0 = desc_k_major(a0 + p * A_STAGE_BYTES), db0 = desc_k_major(b0 + p * B_PANEL);
+                        const uint64_t da0 = desc_k_major(a0 + p * A_STAGE_BYTES), db0 = desc_k_major(b0 + p * b_panel);
 #pragma unroll
                         for (int j = 0; j < BK / 16; ++j) {
                             tc_mma_bf16(tmem_base, da0 + (uint64_t)(2 * j), db0 + (uint64_t)(2 * j), idesc, acc);
@@ -244,18 +255,26 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
                         }
                     }
                     tc_commit(bar_empty + 8 * m_s);
-                    if (++m_s == (uint32_t)STAGES) { m_s = 0; m_ph ^= 1; }
+                    m_mask ^= 1u << m_s;
+                    if (++m_s == nst) m_s = 0;
                 }
                 if (ok) tc_commit(bar_tfull);
             }
             __syncwarp();
         } else {
-            // ---- epilogue: this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
+            // ---- epilogue warps: wait for this CTA's accumulator
             bool eok = mbar_wait(bar_tfull, done & 1, abort_word, 56);
             eok = __all_sync(0xffffffffu, eok);
             ok = eok;
-            if (eok) {
-                tc_fence_after();
+        }
+        // every CTA's MMAs have completed: the stages of the first CTA may now take the partial vectors
+        tc_fence_before();
+        __syncthreads();
+        ss_cluster_sync();
+        tc_fence_after();
+        if (warp >= 2) {
+            // ---- this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
+            if (ok) {
                 const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)g.RP) * 4u;
                 const bool empty_slice = ks0 >= ks1;      // no step: the accumulator was never written
 #pragma unroll 1
@@ -282,7 +301,7 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         ss_cluster_sync();
         tc_fence_after();
         if (crank == 0 && warp >= 2 && row < g.T && ok) {
-            const float* gbuf = reinterpret_cast<const float*>(smem + stage_area);
+            const float* gbuf = reinterpret_cast<const float*>(smem);
             bf16* hrow = g.hd + (size_t)row * g.hd_cols;
             for (int u = 0; u < nug; ++u) {
                 const int gu = u0 + u;
@@ -315,7 +334,9 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
                 hdst[1] = o1;
             }
         }
-        // the gather buffer and the accumulator are free for the cluster's next item
+        // the gather buffer and the accumulator are free for the cluster's next item, whose copies (async proxy) will
+        // overwrite shared memory that generic loads and stores have just used
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         tc_fence_before();
         ss_cluster_sync();
         tc_fence_after();
@@ -324,12 +345,11 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
     // ---- teardown ---------------------------------------------------------------------------------------------
     if (threadIdx.x == 0 && *abort_word != 0) {
         // let the copies already issued land (bounded) before shared memory is released
-        const uint32_t back = p_it < (uint32_t)STAGES ? p_it : (uint32_t)STAGES;
+        const uint32_t back = p_issued < p_stages ? p_issued : p_stages;
         for (uint32_t j = 0; j < back; ++j) {
-            const uint32_t jt = p_it - 1 - j;
+            const uint32_t st = (p_issued - 1 - j) % p_stages;      // its phase bit was flipped when the load went out
             const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(bar_full + 8 * (jt % (uint32_t)STAGES), (jt / (uint32_t)STAGES) & 1) &&
-                   global_ns() - t0 < WAIT_LIMIT_NS) {
+            while (!mbar_try_wait(bar_full + 8 * st, ((p_mask >> st) & 1u) ^ 1u) && global_ns() - t0 < WAIT_LIMIT_NS) {
             }
         }
     }
@@ -361,11 +381,10 @@ static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, 
     for (int C = SS_MAX_C; C >= 1; --C) {
         if ((int64_t)C * tiles > pool->sm_count || (C > 1 && num_kb < 16 * C)) continue;
         const size_t gather = (size_t)C * 128 * pool->RP * 4;
-        const size_t avail = 222 * 1024 - 1024 - 256;
-        if (gather + 2 * SS_STEP_BYTES > avail) continue;
-        int stages = (int)((avail - gather) / SS_STEP_BYTES);
-        if (stages > SS_MAX_STAGES) stages = SS_MAX_STAGES;
-        const size_t smem = 1024 + (size_t)stages * SS_STEP_BYTES + gather + 256;
+        const size_t area = (222 * 1024 - 1024 - 256) / 1024 * 1024;      // stages; the gather buffer lies over them
+        if (gather > area) continue;
+        const int stages = (int)area;
+        const size_t smem = 1024 + area + 256;
         int mc = pool->device < 64 ? max_active[pool->device][C] : 0;
         if (mc == 0) {
             if (cudaFuncSetAttribute(k_shrink_split_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, 222 * 1024) != cudaSuccess) return 0;
@@ -410,7 +429,7 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     g.num_kb = (int)cdiv(D, BK);
     g.num_m_tiles = (int)tiles;
     g.RP = pool->RP; g.cap = pool->cap;
-    g.C = C; g.stages = stages;
+    g.C = C; g.stage_area = (uint32_t)stages;
     g.tok_slot = ws.tok_slot; g.tok_uoff = ws.tok_uoff;
     g.tile_nunits = ws.tile_nunits; g.tile_units = ws.tile_units; g.umax = ws.umax;
     g.d_rank = pool->d_rank; g.d_scale = pool->d_scale;
