@@ -70,6 +70,12 @@ SWEEPS = {
     "prefill": [f"prefill-{T}-{n}" for T in (8192, 16384, 32768) for n in (1, 8, 32)],
     # projections that share their input, fused into one call against one call each, on a decode batch
     "fused": [f"{k}-{T}-32" for T in (64, 256) for k in ("qkvseg", "qkv", "qkvsep", "gateupseg", "gateup", "gateupsep")],
+    # decode batches over the projections of decoder layers of several sizes (hidden x intermediate of 7-8B, 14B and 32B
+    # class models; q / o, gate / up and down shapes), 256 tokens and, for one wide shape, smaller batches
+    "shapes": [f"decode{K}x{N}-{T}-32" for K, N, T in (
+        (4096, 4096, 256), (4096, 12288, 256), (12288, 4096, 256), (4096, 14336, 256), (3584, 18944, 256),
+        (5120, 5120, 256), (5120, 17408, 256), (17408, 5120, 256), (5120, 25600, 256), (25600, 5120, 256),
+        (5120, 17408, 128), (5120, 17408, 64))],
 }
 
 
@@ -85,9 +91,10 @@ def workload_desc(name):
             "one pool over the projections (B side by side), one call" if kind.endswith("seg") else \
             "fused into one projection (block-diagonal B), one call"
         return f"{shape}, {how}; {n} tenants r=16 per projection, {T} decode tokens, fwd only"
-    what = "decode tokens (one per sequence, tenants uniform and unsorted)" if kind == "decode" else \
+    what = "decode tokens (one per sequence, tenants uniform and unsorted)" if kind.startswith("decode") else \
         "prompt tokens in whole-prompt lognormal segments"
-    return f"{kind} sweep point: W 4096x4096, {n} tenants r=16, {T} {what}, fwd only"
+    shape = kind[6:] if kind.startswith("decode") and kind != "decode" else "4096x4096"
+    return f"{kind} sweep point: W {shape}, {n} tenants r=16, {T} {what}, fwd only"
 
 
 def run_sweep(args):

@@ -358,7 +358,7 @@ def fuse_projections(w: Workload, names: Optional[List[str]] = None, segmented: 
     return Workload(w.name + "-fused", w.T, w.T_bwd, w.seg_offsets, w.seg_slot, [fused], w.n_tenants, P * w.max_rank)
 
 
-SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|qkvseg|gateup|gateupsep|gateupseg)-(\d+)-(\d+)$"
+SWEEP_NAME = r"^(decode|prefill|qkv|qkvsep|qkvseg|gateup|gateupsep|gateupseg|decode\d+x\d+)-(\d+)-(\d+)$"
 
 # Variants of the configured workloads (same tensors, another pass or another table):
 VARIANTS = {
@@ -435,6 +435,7 @@ def make_named_workload(name: str) -> Workload:
     4096 x 4096 base weight with rank-16 adapters of scale 2:
 
     ``decode-T-n``   T decode tokens (one per sequence), tenant of each token uniform over n tenants, unsorted;
+    ``decodeKxN-T-n``  the same over a K x N base weight (the projections of decoder layers of other sizes);
     ``prefill-T-n``  T prompt tokens in whole-prompt segments (lognormal lengths, median 1024, clipped to
                      [128, 4096]) dealt to n tenants in shuffled order;
     ``qkv-T-n`` / ``gateup-T-n``  a decode batch through the fused q+k+v (4096 x 12288) or gate+up (4096 x 22016)
@@ -468,9 +469,13 @@ def make_named_workload(name: str) -> Workload:
         f = fuse_projections(w, segmented=kind.endswith("seg"))
         f.name = name
         return f
-    seed = BASE_SEED + 100 + (0 if kind == "decode" else 1)
+    seed = BASE_SEED + 100 + (0 if kind.startswith("decode") else 1)
     K = N = 4096
-    if kind == "decode":
+    if kind.startswith("decode") and kind != "decode":
+        K, N = (int(v) for v in kind[6:].split("x"))
+        if K % 8 or N % 8 or K < 8 or N < 8:
+            raise ValueError(f"workload {name!r}: K and N must be multiples of 8")
+    if kind.startswith("decode"):
         offsets, slots = per_token_table(uniform_token_slots(seed, T, n))
     else:
         offsets, slots = lognormal_segments(seed, T, n)
