@@ -49,6 +49,25 @@ def test_storage_bytes_and_argument_checks(lib):
     assert lib.marlaas_lora_backward(None, 1, None, 0, None, 0, None, 0, None, 0, None, None, None, None, None, 0, 0,
                                      None) == B.MARLAAS_ERR_INVALID_ARG
     assert lib.marlaas_lora_workspace_bytes(None, 5) == 0
+    # pools over several projections: 1 to 4 parts, each a positive multiple of 256 columns
+    def widths(*w):
+        return (ctypes.c_int64 * len(w))(*w)
+    one = lib.marlaas_adapter_pool_storage_bytes(4096, 4096 + 1024 + 1024, 16, 32)
+    seg = lib.marlaas_adapter_pool_storage_bytes_segmented(4096, 3, widths(4096, 1024, 1024), 16, 32)
+    # three blocks of A rows, ONE set of B rows over the side-by-side columns: more than a plain pool of that width by
+    # two blocks of A, far less than the block-diagonal form of rank 48
+    assert seg == one + 2 * 32 * 16 * 4096 * 2
+    assert seg < lib.marlaas_adapter_pool_storage_bytes(4096, 4096 + 1024 + 1024, 48, 32)
+    assert lib.marlaas_adapter_pool_storage_bytes_segmented(4096, 2, widths(4096, 1000), 16, 32) == 0
+    assert lib.marlaas_adapter_pool_storage_bytes_segmented(4096, 5, widths(256, 256, 256, 256, 256), 16, 32) == 0
+    assert lib.marlaas_adapter_pool_storage_bytes_segmented(4096, 0, widths(256), 16, 32) == 0
+    assert lib.marlaas_adapter_pool_storage_bytes_segmented(4096, 2, None, 16, 32) == 0
+    rc = lib.marlaas_adapter_pool_create_segmented(ctypes.byref(h), 0, 512, 2, widths(256, 384), 8, 4, None, 0, None)
+    assert rc == B.MARLAAS_ERR_INVALID_ARG and "multiple of 256" in B.marlaas_last_error()
+    rc = lib.marlaas_adapter_pool_create_segmented(ctypes.byref(h), 0, 512, 2, widths(256, 512), 8, 4, None, 0, None)
+    assert rc in (B.MARLAAS_ERR_UNSUPPORTED_DEVICE, B.MARLAAS_ERR_INVALID_ARG)
+    assert lib.marlaas_adapter_pool_parts(None) == 0
+    assert lib.marlaas_lora_forward_workspace_min_bytes(None, 5) == 0
 
 
 def test_product_path_has_no_oracle_or_cpu_fallback():
