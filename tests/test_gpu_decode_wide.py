@@ -34,6 +34,7 @@ def _case(seed, T, K, N, ranks, per_token):
     (805, 90, 2048, 19200, (16, 8, 16, 32), True),         # 75 tiles on 74 pairs: every pair but the first cuts a tile
     (806, 257, 4096, 11008, (16, 16, 8, 16), False),       # 2 x 43 tiles; the second token tile has one row
     (807, 40, 1664, 24584, (16, 16), True),                # 97 tiles, N not a multiple of 64, K / 64 = 26 steps: pairs span 2-3 tiles
+    (808, 40, 16384, 4864, (16, 8, 16), True),             # 19 tiles, 256 steps each, spread over 74 pairs: 3-5 pieces per tile
 ])
 def test_decode_over_large_weights_matches_the_oracle(seed, T, K, N, ranks, per_token):
     w = _case(seed, T, K, N, ranks, per_token)
