@@ -41,3 +41,37 @@ def test_named_workload_covers_the_configs_and_rejects_other_names():
     for bad in ("cfg", "decode-0-4", "decode-16", "prefill-64-0", "train-64-4"):
         with pytest.raises(ValueError):
             wl.make_named_workload(bad)
+
+
+def test_decode_sweep_point_over_another_weight_shape():
+    w = wl.make_named_workload("decode512x768-48-4")
+    _well_formed(w)
+    p = w.projections[0]
+    assert (p.d_in, p.d_out) == (512, 768) and w.T == 48 and w.T_bwd == 0 and p.x_bits.shape == (48, 512)
+    for bad in ("decode512x-48-4", "decode513x768-48-4", "decodex768-48-4"):
+        with pytest.raises(ValueError):
+            wl.make_named_workload(bad)
+
+
+def test_layer_through_pools_over_projections_keeps_the_tensors_of_the_separate_projections():
+    # a scaled-down 7-projection layer: q, k, v and gate, up as one projection each, o and down as they are
+    w = wl.make_workload(5, scale_down=8)
+    f = wl._fuse_layer(w, "fused")
+    _well_formed(f)
+    by = {p.name: p for p in w.projections}
+    assert [p.name for p in f.projections] == ["q+k+v", "o", "gate+up", "down"]
+    qkv, gu = f.projections[0], f.projections[2]
+    assert qkv.parts == [by[n].d_out for n in "qkv"] and qkv.d_out == sum(qkv.parts)
+    assert gu.parts == [by["gate"].d_out, by["up"].d_out]
+    assert np.array_equal(qkv.W_bits, np.concatenate([by[n].W_bits for n in "qkv"], axis=1))
+    assert np.array_equal(qkv.dy_bits, np.concatenate([by[n].dy_bits for n in "qkv"], axis=1))
+    r = by["q"].adapters[0].rank
+    a = qkv.adapters[0]
+    assert a.rank == r and a.alpha == by["q"].adapters[0].alpha            # rank and scale of ONE projection
+    assert a.A_bits.shape == (qkv.d_in, 3 * r) and a.B_bits.shape == (r, qkv.d_out)
+    assert np.array_equal(a.A_bits[:, r:2 * r], by["k"].adapters[0].A_bits)
+    assert np.array_equal(a.B_bits[:, qkv.parts[0]:qkv.parts[0] + qkv.parts[1]], by["k"].adapters[0].B_bits)
+    # the block-diagonal form of the same projections, for comparison: rank 3 r, zeros off the diagonal
+    d = wl.fuse_projections(w, ["q", "k", "v"]).projections[0]
+    assert d.parts is None and d.adapters[0].rank == 3 * r and d.adapters[0].B_bits.shape == (3 * r, qkv.d_out)
+    assert not d.adapters[0].B_bits[:r, qkv.parts[0]:].any()
