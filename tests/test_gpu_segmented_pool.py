@@ -326,3 +326,25 @@ def test_random_pools_over_several_projections_match_the_oracle(batch):
                     assert_close(sc.split_dB(t, dB[t])[pi], rdB[t], tag + f": dB[{t}] of projection {pi}")
         assert_close(to_np(dx), rdx, tag + ": dx")
         B.marlaas_check_status(sc.pool)
+
+
+def test_unregister_and_reregister_on_a_pool_over_two_projections():
+    # a freed slot serves the base weight only on every projection; registering again (another rank) brings it back
+    T, K, Ns, ranks = 180, 128, (256, 512), (16, 8, 32)
+    w = _case(4100, T, K, Ns, ranks, True)
+    ts = w.tok_slot()
+    sc = SegCase(w, capacity=4)
+    t0 = w.projections[0].adapters[0]
+    B.marlaas_adapter_pool_unregister(sc.pool, t0.tenant_id)
+    y = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg)
+    ts_freed = np.where(ts == 0, -1, ts).astype(np.int32)
+    assert_close(to_np(y), _oracle_forward(w, ts_freed)[0], "after unregister: slot 0 serves the base weight only")
+    with pytest.raises(B.MarlaasError):
+        B.marlaas_adapter_pool_lookup(sc.pool, t0.tenant_id)
+    As = [dev_bf16(p.adapters[0].A_bits) for p in w.projections]
+    Bs = [dev_bf16(p.adapters[0].B_bits) for p in w.projections]
+    assert B.marlaas_adapter_pool_register(sc.pool, t0.tenant_id, 7, t0.rank, t0.alpha, As, Bs) == 0      # lowest free slot
+    y2 = B.marlaas_lora_forward(sc.pool, sc.x, sc.W, sc.seg)
+    assert_close(to_np(y2), _oracle_forward(w, ts)[0], "after registering again")
+    assert B.marlaas_adapter_pool_lookup(sc.pool, t0.tenant_id)[3] == 7
+    B.marlaas_check_status(sc.pool)
