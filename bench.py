@@ -466,6 +466,11 @@ def main():
         extra("cfg5-fused", wl.make_variant("cfg5-fused", w5))
         extra("cfg5-decode", wl.make_variant("cfg5-decode", w5), steps=20, repeats=5)
         extra("cfg5-decode-fused", wl.make_variant("cfg5-decode-fused", w5), steps=20, repeats=5)
+        del w5
+        # decode over a wider weight (gate / up of a 14B-class layer: 68 column strips for the 74 CTA pairs): the shape on
+        # which the one-pass-over-W kernels come closest to the copy peak
+        for nm in ("decode5120x17408-256-32", "decode5120x17408-64-32"):
+            extra(nm, wl.make_named_workload(nm), steps=20, repeats=5)
         out["configs"] = configs
     if rank == 0:
         print(json.dumps(out))
