@@ -77,6 +77,8 @@ struct DecodeArgs {
     int num_ks;          // 64-deep pipeline steps over K
     int num_xs;          // 64-deep pipeline steps over the expand rows (up to the last slot in use)
     int S;               // contraction slices per tile: 1, 2 or 4 CTA pairs
+    int tn;              // tokens per tile = N of the MMA: 256, or 128 / 64 for smaller batches whose contraction is not cut
+                         // (less of every stage is token rows, less tensor work on rows that hold no token)
     int stages;
     int w3d;             // the W-side operand moves with one 3-D copy per step (N a multiple of 64), else one per chunk
     int parts;           // projections held by the pool: hd is [parts][T][..] and a strip takes the plane of its projection
@@ -100,7 +102,9 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int STAGES = g.stages;
-    constexpr uint32_t W_BYTES = 2 * CHUNK_BYTES, X_BYTES = A_STAGE_BYTES, STAGE_BYTES = W_BYTES + X_BYTES;
+    constexpr uint32_t W_BYTES = 2 * CHUNK_BYTES;
+    const int XH = g.tn / 2;                         // token rows a CTA stages: its half of the tile's tokens
+    const uint32_t X_BYTES = (uint32_t)XH * 128u, STAGE_BYTES = W_BYTES + X_BYTES;
     const uint32_t sStage = smem_u32(smem);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
     const uint32_t bar_full = smem_u32(bars);
@@ -141,8 +145,8 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const int gp = (int)dk_cluster_id_x();           // CTA pair
     const int tile = gp / g.S, sl = gp % g.S;        // contraction slice of this pair
     const int n0 = (tile % g.nstrips) * DG_TM;
-    const int m0 = (tile / g.nstrips) * DG_TN;
-    const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
+    const int m0 = (tile / g.nstrips) * g.tn;
+    const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * XH;
     // the projection whose columns the strip lies in (constant indices: a variable one would move the arguments to local memory)
     const int part = (g.parts > 1 ? (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]) : 0);
     const int hd_tok = my_tok + part * g.T;          // this half's rows of the projection's plane of hd
@@ -162,7 +166,7 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
     // bytes the two CTAs of the pair stage per step (boxes wholly outside the tensors are skipped; partly outside boxes
     // are filled with zeros and count in full)
-    auto x_tx = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? X_BYTES : 0u; };
+    auto x_tx = [&](int r) -> uint32_t { return (m0 + r * XH < g.T) ? X_BYTES : 0u; };
     auto w_chunks = [&](int r) -> int { return max(0, min(2, (g.Nout - (n0 + r * 128) + 63) / 64)); };
     auto w_tx = [&](int r) -> uint32_t { const int c = w_chunks(r); return (g.w3d ? (c > 0 ? 2u : 0u) : (uint32_t)c) * CHUNK_BYTES; };
     const uint32_t stage_tx = x_tx(0) + x_tx(1) + w_tx(0) + w_tx(1);
@@ -214,8 +218,8 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         // ================= MMA issuer (the pair's first CTA) =================
         if (lane == 0 && half == 0) {
             // fp32 accumulate, bf16 x bf16, A MN-major (W columns), B K-major (tokens), M = 256, N = 256
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(DG_TN >> 3) << 17) |
-                                       ((uint32_t)(DG_TM >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(g.tn >> 3) << 17) |
+                                   ((uint32_t)(DG_TM >> 4) << 24);
             const uint16_t mask = 3;
             uint32_t acc = 0, s = 0, ph = 0;
             bool ok = true;
@@ -256,7 +260,7 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const uint32_t tl = tmem_base + ((uint32_t)(q * 32) << 16);
         uint8_t* stg = smem + ew * 2048;            // the pipeline stages are free: every MMA of the pair has completed
         const int ncol = my_n + q * 32;             // first W column of this warp
-        const int Wd = DG_TN / g.S, nch = Wd / 64;  // nch: 4, 2, 1 for S = 1, 2, 4
+        const int Wd = g.tn / g.S, nch = Wd / 64;   // nch: 4, 2, 1 for 256 tokens and S = 1, 2, 4; 2, 1 for 128, 64 tokens
         // 32 tokens x this warp's 32 columns, fp32 in registers (one column per thread) -> bf16 rows of y
         auto store_chunk = [&](const float (&v)[32], int tok0) {
 #pragma unroll
@@ -767,17 +771,18 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
     g.T = (int)T; g.Nout = (int)N;
     g.C = y; g.ldc = ldy; g.status = pool->d_status; g.sync = pool->d_sync; g.xbuf = ws.xbuf;
     g.S = shape.S;
+    g.tn = shape.S == 1 && T <= 64 ? 64 : shape.S == 1 && T <= 128 ? 128 : DG_TN;
     g.nstrips = (int)cdiv(N, DG_TM);
     g.num_ks = (int)(K / BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
     g.w3d = (N % 64) == 0;
     g.parts = pool->P;
     for (int p = 0; p < 4; ++p) g.part_end[p] = p < pool->P ? (int)pool->part_begin[p + 1] : 0;
-    constexpr size_t stage_bytes = 2 * CHUNK_BYTES + A_STAGE_BYTES;
+    const size_t stage_bytes = 2 * CHUNK_BYTES + (size_t)(g.tn / 2) * 128;
     // The shrink kernel's CTAs are spread over all SMs (two apiece) when this kernel's CTAs arrive: the pipeline takes
     // what two of them leave of an SM's 227 KB, so that neither kernel waits for the other's shared memory.
     const size_t room = (size_t)227 * 1024 - 2 * decode_shrink_smem_bytes(T, S) - 1024;
-    g.stages = (int)std::max<size_t>(2, std::min<size_t>(7, (room - 1024 - 512) / stage_bytes));
+    g.stages = (int)std::max<size_t>(2, std::min<size_t>(9, (room - 1024 - 512) / stage_bytes));
     const size_t smem_bytes = 1024 + 512 + (size_t)g.stages * stage_bytes;
     if ((size_t)SY_FLAGS + (size_t)(shape.pairs / shape.S) * shape.S * (shape.S - 1) * 16 > DECODE_SYNC_BYTES / 4)
         return fail(MARLAAS_ERR_INVALID_ARG, "lora_forward: the decode path needs more exchange flags than the pool holds");
@@ -786,12 +791,12 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
     if ((rc = launch_decode_shrink(pool, T, x, ldx, S, seg_offsets, seg_slot, ws, h_out, st)) != MARLAAS_OK) return rc;
 
     alignas(64) CUtensorMap tmW, tmX, tmXW, tmXX;
-    if ((rc = make_panel_map(&tmX, x, T, K, ldx, 1, 128)) != MARLAAS_OK) return rc;
+    if ((rc = make_panel_map(&tmX, x, T, K, ldx, 1, (uint32_t)(g.tn / 2))) != MARLAAS_OK) return rc;
     if (g.w3d) rc = make_panel_map(&tmW, W, K, N, ldw, 2, BK);
     else rc = make_map(&tmW, W, K, N, ldw, 64, BK);
     if (rc != MARLAAS_OK) return rc;
     if (g.num_xs > 0) {
-        if ((rc = make_panel_map(&tmXX, ws.hd, T * pool->P, hd_cols, hd_cols, 1, 128)) != MARLAAS_OK) return rc;
+        if ((rc = make_panel_map(&tmXX, ws.hd, T * pool->P, hd_cols, hd_cols, 1, (uint32_t)(g.tn / 2))) != MARLAAS_OK) return rc;
         if (g.w3d) rc = make_panel_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 2, BK);
         else rc = make_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 64, BK);
         if (rc != MARLAAS_OK) return rc;
