@@ -400,6 +400,7 @@ struct StreamArgs {
     int nstep;           // steps per tile = num_ks + num_xs
     int total;           // steps of all tiles
     int npairs;
+    int tn;              // tokens per tile = N of the MMA: 256, or 128 / 64 when the whole batch fits
     int stages;
     int w3d;
     int parts;
@@ -435,7 +436,9 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int STAGES = g.stages;
-    constexpr uint32_t W_BYTES = 2 * CHUNK_BYTES, X_BYTES = A_STAGE_BYTES, STAGE_BYTES = W_BYTES + X_BYTES;
+    constexpr uint32_t W_BYTES = 2 * CHUNK_BYTES;
+    const int XH = g.tn / 2;                         // token rows a CTA stages: its half of the tile's tokens
+    const uint32_t X_BYTES = (uint32_t)XH * 128u, STAGE_BYTES = W_BYTES + X_BYTES;
     constexpr uint32_t STG_BYTES = 8 * 2048;        // epilogue staging, one 2 KB block per warp (the stages stay busy)
     const uint32_t sStage = smem_u32(smem);
     uint8_t* stg_base = smem + (size_t)STAGES * STAGE_BYTES;
@@ -497,11 +500,11 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
             PieceIter pi = {g1, g0, g.nstep};
             int tile, s0, s1;
             while (ok && pi.next(tile, s0, s1)) {
-                const int n0 = (tile % g.nstrips) * DG_TM, m0 = (tile / g.nstrips) * DG_TN;
-                const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * 128;
+                const int n0 = (tile % g.nstrips) * DG_TM, m0 = (tile / g.nstrips) * g.tn;
+                const int my_n = n0 + (int)half * 128, my_tok = m0 + (int)half * XH;
                 const int part = (g.parts > 1 ? (int)(n0 >= g.part_end[0]) + (int)(g.parts > 2 && n0 >= g.part_end[1]) + (int)(g.parts > 3 && n0 >= g.part_end[2]) : 0);
                 const int hd_tok = my_tok + part * g.T;
-                auto x_tx = [&](int r) -> uint32_t { return (m0 + r * 128 < g.T) ? X_BYTES : 0u; };
+                auto x_tx = [&](int r) -> uint32_t { return (m0 + r * XH < g.T) ? X_BYTES : 0u; };
                 auto w_chunks = [&](int r) -> int { return max(0, min(2, (g.Nout - (n0 + r * 128) + 63) / 64)); };
                 auto w_tx = [&](int r) -> uint32_t { const int c = w_chunks(r); return (g.w3d ? (c > 0 ? 2u : 0u) : (uint32_t)c) * CHUNK_BYTES; };
                 const uint32_t stage_tx = x_tx(0) + x_tx(1) + w_tx(0) + w_tx(1);
@@ -546,8 +549,8 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
     } else if (warp == 1) {
         // ================= MMA issuer (the pair's first CTA) =================
         if (lane == 0 && half == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(DG_TN >> 3) << 17) |
-                                       ((uint32_t)(DG_TM >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(g.tn >> 3) << 17) |
+                                   ((uint32_t)(DG_TM >> 4) << 24);
             const uint16_t mask = 3;
             uint32_t s = 0, ph = 0, k = 0;
             bool ok = true;
@@ -587,8 +590,10 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
     } else {
         // ================= epilogue warps =================
         // Thread (q, lane) owns W column n = my_n + 32 q + lane (tensor-memory lane 32 q + lane); the accumulator's columns
-        // are the tile's tokens, and warp (q, ch) takes token columns [128 ch, 128 ch + 128) in four chunks of 32.
+        // are the tile's tokens, and warp (q, ch) takes its half of them, token columns [ch tn / 2, (ch + 1) tn / 2), in
+        // chunks of 32 (four at 256 tokens a tile).
         const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
+        const int nchk = g.tn / 64;
         uint8_t* stg = stg_base + ew * 2048;
         const uint32_t tempty0 = dk_map_to_cta(bar_tempty, 0);
         auto slot_of = [&](int pair) -> size_t { return ((size_t)pair * 2 + half) * 8 + ew; };      // 16 KB each
@@ -602,13 +607,13 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int n0 = (tile % g.nstrips) * DG_TM, m0 = (tile / g.nstrips) * DG_TN;
+            const int n0 = (tile % g.nstrips) * DG_TM, m0 = (tile / g.nstrips) * g.tn;
             const int ncol = n0 + (int)half * 128 + q * 32;
-            const uint32_t tl = tmem_base + ((uint32_t)(q * 32) << 16) + b * DG_TN + ch * 128;
+            const uint32_t tl = tmem_base + ((uint32_t)(q * 32) << 16) + b * DG_TN + ch * XH;
             if (s1 < g.nstep) {
                 // ---- not the tile's last steps: the partial sums go to this pair's slot
                 float* o = g.xbuf + slot_of(gp) * 4096 + lane * 4;
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < nchk; ++c) {
                     uint32_t v[32];
                     tc_ld_32x32(tl + c * 32, v);
                     tc_wait_ld();
@@ -633,7 +638,7 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     __syncwarp();
                     if (!ok) break;
                 }
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < nchk; ++c) {
                     uint32_t v[32];
                     tc_ld_32x32(tl + c * 32, v);
                     tc_wait_ld();
@@ -654,7 +659,7 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
                         }
                     }
                     // 32 tokens x this warp's 32 columns, fp32 in registers (one column per thread) -> bf16 rows of y
-                    const int tok0 = m0 + ch * 128 + c * 32;
+                    const int tok0 = m0 + ch * XH + c * 32;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) reinterpret_cast<bf16*>(stg)[j * 32 + lane] = __float2bfloat16_rn(f[j]);
                     __syncwarp();
@@ -845,15 +850,16 @@ marlaas_status_t launch_decode_stream_sm100(const marlaas_pool* pool, int64_t T,
     g.num_ks = (int)(K / BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
     g.nstep = g.num_ks + g.num_xs;
+    g.tn = T <= 64 ? 64 : T <= 128 ? 128 : DG_TN;      // one token tile in all three cases
     const int64_t tiles = cdiv(T, DG_TN) * g.nstrips;
     g.total = (int)(tiles * g.nstep);
     g.w3d = (N % 64) == 0;
     g.parts = pool->P;
     for (int p = 0; p < 4; ++p) g.part_end[p] = p < pool->P ? (int)pool->part_begin[p + 1] : 0;
-    constexpr size_t stage_bytes = 2 * CHUNK_BYTES + A_STAGE_BYTES;
+    const size_t stage_bytes = 2 * CHUNK_BYTES + (size_t)(g.tn / 2) * 128;
     // as in the one-tile-per-pair kernel, two shrink CTAs share each SM with a CTA of this kernel
     const size_t room = (size_t)227 * 1024 - 2 * decode_shrink_smem_bytes(T, S) - 1024;
-    g.stages = (int)std::max<size_t>(2, std::min<size_t>(6, (room - 1024 - 512 - 8 * 2048) / stage_bytes));
+    g.stages = (int)std::max<size_t>(2, std::min<size_t>(9, (room - 1024 - 512 - 8 * 2048) / stage_bytes));
     const size_t smem_bytes = 1024 + 512 + 8 * 2048 + (size_t)g.stages * stage_bytes;
 
     // every pair must be resident at once only in so far as a pair waits for pairs of lower index, which are placed first;
@@ -882,12 +888,12 @@ marlaas_status_t launch_decode_stream_sm100(const marlaas_pool* pool, int64_t T,
     if ((rc = launch_decode_shrink(pool, T, x, ldx, S, seg_offsets, seg_slot, ws, h_out, st)) != MARLAAS_OK) return rc;
 
     alignas(64) CUtensorMap tmW, tmX, tmXW, tmXX;
-    if ((rc = make_panel_map(&tmX, x, T, K, ldx, 1, 128)) != MARLAAS_OK) return rc;
+    if ((rc = make_panel_map(&tmX, x, T, K, ldx, 1, (uint32_t)(g.tn / 2))) != MARLAAS_OK) return rc;
     if (g.w3d) rc = make_panel_map(&tmW, W, K, N, ldw, 2, BK);
     else rc = make_map(&tmW, W, K, N, ldw, 64, BK);
     if (rc != MARLAAS_OK) return rc;
     if (g.num_xs > 0) {
-        if ((rc = make_panel_map(&tmXX, ws.hd, T * pool->P, hd_cols, hd_cols, 1, 128)) != MARLAAS_OK) return rc;
+        if ((rc = make_panel_map(&tmXX, ws.hd, T * pool->P, hd_cols, hd_cols, 1, (uint32_t)(g.tn / 2))) != MARLAAS_OK) return rc;
         if (g.w3d) rc = make_panel_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 2, BK);
         else rc = make_map(&tmXW, pool->d_Bs, (int64_t)pool->cap * pool->RP, N, pool->ldB, 64, BK);
         if (rc != MARLAAS_OK) return rc;
