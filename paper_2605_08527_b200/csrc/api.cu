@@ -253,7 +253,7 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
             rc = stream_k
                      ? launch_decode_stream_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
                                                   seg->seg_offsets, seg->seg_slot, ws, h, st)
-                 : (decode_wide_sm100_eligible(pool, T) && (has_xbuf || decode_wide_sm100_xbuf_bytes(pool, T) == 0))
+                 : (decode_wide_sm100_eligible(pool, T) && (has_xbuf || !decode_wide_sm100_splits(pool, T)))
                      ? launch_decode_wide_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,
                                                 seg->seg_offsets, seg->seg_slot, ws, h, st)
                      : launch_decode_sm100(pool, T, (const bf16*)x, ldx, (const bf16*)W, ldw, (bf16*)y, ldy, S,

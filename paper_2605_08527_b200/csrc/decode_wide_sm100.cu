@@ -749,8 +749,15 @@ bool decode_stream_sm100_eligible(const marlaas_pool* pool, int64_t T) {
     // or more of the SMs would idle) and the contraction is deep enough to carry the exchange of three or four pieces
     // per tile: 17408 x 5120, 256 tokens: 68.4 against 71.1 us; 25600 x 5120: 87.2 against 95.7 us
     const bool deep_few = tiles * 4 > room && tiles * 3 <= room && pool->K / sm100::BK >= 256;
-    return (tiles > room || deep_few) && tiles * ((pool->K + pool->cap * pool->RP) / sm100::BK + 1) < (1ll << 30);
+    // and for batches of up to 64 tokens over 16 to 44 tiles: partial sums of 64 tokens are cheap to pass on, and an even
+    // share of the steps on every pair beats one tile per pair, cut in 1, 2 or 4 (11008 x 4096: 34.6 against 36.5 us;
+    // 4096 x 8192: 27.8 against 29.9; 4096 x 11008: 31.6 against 33.3; from 48 tiles on it is no faster, then slower)
+    const bool small_batch = T <= 64 && tiles >= 16 && tiles * 5 <= room * 3;
+    return (tiles > room || deep_few || small_batch) && tiles * ((pool->K + pool->cap * pool->RP) / sm100::BK + 1) < (1ll << 30);
 }
+
+// Whether the one-tile-per-pair kernel would cut the contraction (and so need the exchange scratch) for this batch.
+bool decode_wide_sm100_splits(const marlaas_pool* pool, int64_t T) { return decode_shape(pool, T).S > 1; }
 
 size_t decode_wide_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T) {
     if (decode_stream_sm100_eligible(pool, T)) return (size_t)(pool->sm_count / 2) * 2 * 8 * 16384;     // a slot per pair, CTA, warp

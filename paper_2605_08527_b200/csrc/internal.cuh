@@ -189,6 +189,7 @@ size_t decode_shrink_smem_bytes(int64_t T, int32_t S);
 // decode_wide_sm100.cu: the same forward for large weights (W columns on the MMA's M side; see the file)
 bool decode_wide_sm100_eligible(const marlaas_pool* pool, int64_t T);
 size_t decode_wide_sm100_xbuf_bytes(const marlaas_pool* pool, int64_t T);    // its exchange scratch (0 if unused)
+bool decode_wide_sm100_splits(const marlaas_pool* pool, int64_t T);        // true if that kernel would cut the contraction in slices
 marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, const bf16* x, int64_t ldx, const bf16* W,
                                           int64_t ldw, bf16* y, int64_t ldy, int32_t S, const int32_t* seg_offsets,
                                           const int32_t* seg_slot, const Workspace& ws, float* h_out, cudaStream_t st);

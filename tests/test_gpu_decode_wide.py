@@ -35,10 +35,12 @@ def _case(seed, T, K, N, ranks, per_token):
     (806, 257, 4096, 11008, (16, 16, 8, 16), False),       # 2 x 43 tiles; the second token tile has one row
     (807, 40, 1664, 24584, (16, 16), True),                # 97 tiles, N not a multiple of 64, K / 64 = 26 steps: pairs span 2-3 tiles
     (808, 40, 16384, 4864, (16, 8, 16), True),             # 19 tiles, 256 steps each, spread over 74 pairs: 3-5 pieces per tile
-    (809, 40, 4096, 11008, (16, 8, 16, 4), True),          # 43 tiles, no split, 64-token tiles: the second CTA's rows 32..39 only
-    (810, 64, 4096, 10248, (16, 16, 32), True),            # 41 tiles of 64 tokens, all rows; N not a multiple of 64
-    (811, 17, 4096, 11008, (16, 16), True),                # 64-token tiles whose second half holds no token at all
+    (809, 40, 4096, 13312, (16, 8, 16, 4), True),          # 52 tiles, no split, 64-token tiles: the second CTA's rows 32..39 only
+    (810, 64, 4096, 12808, (16, 16, 32), True),            # 51 tiles of 64 tokens, all rows; N not a multiple of 64
+    (811, 17, 4096, 14336, (16, 16), True),                # 56 tiles of 64 tokens whose second half holds no token at all
     (812, 128, 4096, 11008, (16, 8, 16, 16), False),       # 128-token tiles, every row a token
+    (813, 17, 4096, 11008, (16, 16), True),                # 43 tiles, up to 64 tokens: steps spread over all pairs, 1-2 pieces per tile
+    (814, 64, 11008, 4096, (16, 8, 32), False),            # 16 tiles, 64 tokens: 4-5 pieces per tile
 ])
 def test_decode_over_large_weights_matches_the_oracle(seed, T, K, N, ranks, per_token):
     w = _case(seed, T, K, N, ranks, per_token)
