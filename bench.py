@@ -71,11 +71,13 @@ SWEEPS = {
     # projections that share their input, fused into one call against one call each, on a decode batch
     "fused": [f"{k}-{T}-32" for T in (64, 256) for k in ("qkvseg", "qkv", "qkvsep", "gateupseg", "gateup", "gateupsep")],
     # decode batches over the projections of decoder layers of several sizes (hidden x intermediate of 7-8B, 14B and 32B
-    # class models; q / o, gate / up and down shapes), 256 tokens and, for one wide shape, smaller batches
+    # class models; q / o, gate / up and down shapes), 256 tokens and smaller batches
     "shapes": [f"decode{K}x{N}-{T}-32" for K, N, T in (
         (4096, 4096, 256), (4096, 12288, 256), (12288, 4096, 256), (4096, 14336, 256), (3584, 18944, 256),
         (5120, 5120, 256), (5120, 17408, 256), (17408, 5120, 256), (5120, 25600, 256), (25600, 5120, 256),
-        (5120, 17408, 128), (5120, 17408, 64))],
+        (5120, 17408, 128), (5120, 17408, 64),
+        # batches of 64 tokens: the kernels run with 64-token tiles
+        (4096, 12288, 64), (12288, 4096, 64), (3584, 18944, 64), (17408, 5120, 64), (5120, 25600, 64), (5120, 34816, 32))],
 }
 
 
