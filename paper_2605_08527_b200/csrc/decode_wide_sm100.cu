@@ -77,7 +77,7 @@ struct DecodeArgs {
     int num_ks;          // 64-deep pipeline steps over K
     int num_xs;          // 64-deep pipeline steps over the expand rows (up to the last slot in use)
     int S;               // contraction slices per tile: 1, 2 or 4 CTA pairs
-    int tn;              // tokens per tile = N of the MMA: 256, or 128 / 64 for smaller batches whose contraction is not cut
+    int tn;              // tokens per tile = N of the MMA: 256, or 64 / 128 / 192 for smaller batches whose contraction is not cut
                          // (less of every stage is token rows, less tensor work on rows that hold no token)
     int stages;
     int w3d;             // the W-side operand moves with one 3-D copy per step (N a multiple of 64), else one per chunk
@@ -260,7 +260,7 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const uint32_t tl = tmem_base + ((uint32_t)(q * 32) << 16);
         uint8_t* stg = smem + ew * 2048;            // the pipeline stages are free: every MMA of the pair has completed
         const int ncol = my_n + q * 32;             // first W column of this warp
-        const int Wd = g.tn / g.S, nch = Wd / 64;   // nch: 4, 2, 1 for 256 tokens and S = 1, 2, 4; 2, 1 for 128, 64 tokens
+        const int Wd = g.tn / g.S, nch = Wd / 64;   // nch: 4, 2, 1 for 256 tokens and S = 1, 2, 4; 3, 2, 1 for 192, 128, 64 tokens
         // 32 tokens x this warp's 32 columns, fp32 in registers (one column per thread) -> bf16 rows of y
         auto store_chunk = [&](const float (&v)[32], int tok0) {
 #pragma unroll
@@ -400,7 +400,7 @@ struct StreamArgs {
     int nstep;           // steps per tile = num_ks + num_xs
     int total;           // steps of all tiles
     int npairs;
-    int tn;              // tokens per tile = N of the MMA: 256, or 128 / 64 when the whole batch fits
+    int tn;              // tokens per tile = N of the MMA: 256, or 64 / 128 / 192 when the whole batch fits
     int stages;
     int w3d;
     int parts;
@@ -783,7 +783,7 @@ marlaas_status_t launch_decode_wide_sm100(const marlaas_pool* pool, int64_t T, c
     g.T = (int)T; g.Nout = (int)N;
     g.C = y; g.ldc = ldy; g.status = pool->d_status; g.sync = pool->d_sync; g.xbuf = ws.xbuf;
     g.S = shape.S;
-    g.tn = shape.S == 1 && T <= 64 ? 64 : shape.S == 1 && T <= 128 ? 128 : DG_TN;
+    g.tn = shape.S == 1 && T < DG_TN ? (int)cdiv(T, 64) * 64 : DG_TN;
     g.nstrips = (int)cdiv(N, DG_TM);
     g.num_ks = (int)(K / BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
@@ -857,7 +857,7 @@ marlaas_status_t launch_decode_stream_sm100(const marlaas_pool* pool, int64_t T,
     g.num_ks = (int)(K / BK);
     g.num_xs = (int)cdiv((int64_t)(last_used + 1) * pool->RP, (int64_t)BK);
     g.nstep = g.num_ks + g.num_xs;
-    g.tn = T <= 64 ? 64 : T <= 128 ? 128 : DG_TN;      // one token tile in all three cases
+    g.tn = T < DG_TN ? (int)cdiv(T, 64) * 64 : DG_TN;  // one token tile whenever it is narrower than 256
     const int64_t tiles = cdiv(T, DG_TN) * g.nstrips;
     g.total = (int)(tiles * g.nstep);
     g.w3d = (N % 64) == 0;

@@ -41,6 +41,8 @@ def _case(seed, T, K, N, ranks, per_token):
     (812, 128, 4096, 11008, (16, 8, 16, 16), False),       # 128-token tiles, every row a token
     (813, 17, 4096, 11008, (16, 16), True),                # 43 tiles, up to 64 tokens: steps spread over all pairs, 1-2 pieces per tile
     (814, 64, 11008, 4096, (16, 8, 32), False),            # 16 tiles, 64 tokens: 4-5 pieces per tile
+    (815, 150, 4096, 11008, (16, 8, 16), True),            # 43 tiles of 192 tokens (96 per CTA; the second CTA's last 42 rows empty)
+    (816, 190, 2048, 19200, (16, 16, 8), True),            # 75 tiles of 192 tokens on 74 pairs
 ])
 def test_decode_over_large_weights_matches_the_oracle(seed, T, K, N, ranks, per_token):
     w = _case(seed, T, K, N, ranks, per_token)

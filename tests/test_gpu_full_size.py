@@ -153,3 +153,23 @@ def test_cfg5_layer_through_pools_over_projections_full_size():
     for names in (("q", "k", "v"), ("gate", "up")):
         _check_fused_full(wd, names, n_rows=64)
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", [
+    "decode5120x17408-256-32",     # 68 strips, one tile per CTA pair, 256-token tiles
+    "decode5120x17408-64-32",      # the same weight with 64-token tiles
+    "decode12288x4096-64-32",      # 16 strips, 64 tokens: the steps spread over all pairs, 4-5 pieces per tile
+    "decode5120x25600-64-32",      # 100 strips on 74 pairs, 64-token tiles
+])
+def test_decode_over_wide_weights_every_row(name):
+    # the decode configurations bench.py reports beside the configured workloads: every row of y against the oracle
+    w = wl.make_named_workload(name)
+    p = w.projections[0]
+    ts = w.tok_slot()
+    r, s, A, Bm = oracle.adapters_of(p)
+    dc = DeviceCase(w, p)
+    y = dc.forward()
+    ry, _ = oracle.forward(p.x, p.W, r, s, A, Bm, ts)
+    assert_close(to_np(y), ry, f"{name}: y (every row)")
+    assert torch.equal(y, dc.forward())
+    B.marlaas_check_status(dc.pool)
