@@ -76,6 +76,20 @@ def test_small_ragged_cases(flags, seed, T, K, N, ranks):
     _check_case(w, w.projections[0], flags=flags, capacity=len(ranks) + 2)
 
 
+@pytest.mark.parametrize("seed,T,K,N,ranks", [
+    # 5 x 16 = 80 tiles on 74 CTA pairs in forward and in dx: a second, nearly empty round.  Depths not multiples of 64
+    # (one panel per step); last tile of y: 160 columns, of dx: 200
+    (61, 1280, 4040, 4000, (16, 8, 32)),
+    # depths in whole panels (two per step); last tile of y has 64 columns, of dx 192
+    (62, 1280, 4032, 3904, (16, 16, 64, 4)),
+    # 9 x 9 = 81 tiles forward (7 in the last round), dx in a single round; 10 rows in the last row tile
+    (63, 2058, 1024, 2304, (32, 8)),
+])
+def test_more_tiles_than_cta_pairs_with_ragged_edges(seed, T, K, N, ranks):
+    w = wl.small_random_case(seed, T, K, N, list(ranks), n_segments=9)
+    _check_case(w, w.projections[0], capacity=len(ranks) + 1)
+
+
 def test_finely_interleaved_tenants_with_backward():
     # every token its own segment, tenants drawn uniformly: the per-block tenant copies of the tensor-core gradient
     # reduction do not fit, so the device-side switch to the CUDA-core reduction is exercised
