@@ -173,7 +173,10 @@ int32_t marlaas_adapter_pool_rank_stride(const marlaas_pool_t* pool);
 /* ---- the layer ---- */
 
 /* Bytes of workspace forward/backward need for a batch of T tokens on this pool (device memory, 256-byte
- * aligned, contents need not be preserved between calls; two calls in flight need two workspaces). */
+ * aligned, contents need not be preserved between calls; two calls in flight need two workspaces).  The size does not
+ * grow monotonically with T: the decode-shaped kernels chosen for small batches over large weights may use more exchange
+ * scratch than those chosen for larger batches, so a workspace shared by calls of several batch sizes takes the largest
+ * of their sizes (a call given less than its own full size still runs, see marlaas_lora_forward_workspace_min_bytes). */
 size_t marlaas_lora_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
 /* The part of that workspace a forward call uses (its leading bytes): enough for marlaas_lora_forward alone. */
 size_t marlaas_lora_forward_workspace_bytes(const marlaas_pool_t* pool, int64_t T);
