@@ -526,8 +526,10 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
                                                           gs, ws.hm2, GRAD_PHASE_COPIES)) != MARLAAS_OK) return r;
                     if (want_dB && (r = launch_grad_sm100(pool, T, Np, dyp, lddy, hp, nullptr, dBp, false, acc, ws,
                                                           gs, ws.hm, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
+                    // the dA reduction reads x and its own copies (made above), nothing of the dB reduction: started behind it
+                    // as a programmatic dependent, its CTAs take the SMs that the dB reduction's CTAs leave one by one
                     if (want_dA && (r = launch_grad_sm100(pool, T, pool->K, (const bf16*)x, ldx, gp, nullptr, dAp, true, acc, ws,
-                                                          gs, ws.hm2, GRAD_PHASE_REDUCE)) != MARLAAS_OK) return r;
+                                                          gs, ws.hm2, GRAD_PHASE_REDUCE | (want_dB ? GRAD_PHASE_EARLY : 0))) != MARLAAS_OK) return r;
                 }
                 return MARLAAS_OK;
             };

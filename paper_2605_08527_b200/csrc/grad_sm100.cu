@@ -192,6 +192,9 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
     constexpr int MAX_STAGES = GRAD_STAGES;
     const int STAGES = g.stages;
     constexpr uint32_t TMEM_COLS = 512;
+    // A second reduction launched behind this one as a programmatic dependent (it reads nothing this one writes) may
+    // take over every SM a CTA of this grid leaves.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (g.gflag[0] != 0) return;   // copies did not fit: the CUDA-core reduction handles this call
 
     extern __shared__ uint8_t smem_raw[];
@@ -448,6 +451,8 @@ k_grad_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_constant__ 
     if (threadIdx.x == 0 && *abort_word != 0) {
         if (atomicCAS(g.status, 0, DEV_TIMEOUT) == 0) g.status[1] = *abort_word * 1000000 + (int)blockIdx.x;
     }
+    // launched early behind another reduction: never complete before it (what follows in the stream relies on both)
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace sm100
@@ -514,7 +519,22 @@ marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t 
     }
     const int items = g.num_c_tiles * g.cap;
     const int grid = items < pool->sm_count ? items : pool->sm_count;
-    k_grad_sm100<<<grid, GRAD_THREADS, smem_bytes, st>>>(tmSrc, tmHm, g);
+    if (phases & GRAD_PHASE_EARLY) {
+        // the caller states that this launch reads nothing the kernel before it in the stream writes: its CTAs may start
+        // on SMs that kernel's CTAs have left
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(GRAD_THREADS);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_grad_sm100, tmSrc, tmHm, g));
+    } else {
+        k_grad_sm100<<<grid, GRAD_THREADS, smem_bytes, st>>>(tmSrc, tmHm, g);
+    }
     MARLAAS_LAUNCH_CHECK("k_grad_sm100");
     return MARLAAS_OK;
 }

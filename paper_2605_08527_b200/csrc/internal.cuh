@@ -239,7 +239,8 @@ marlaas_status_t launch_grad_reduce(const marlaas_pool* pool, int64_t C, const b
 bool grad_sm100_eligible(const marlaas_pool* pool, int64_t T);
 marlaas_status_t launch_grad_plan(const marlaas_pool* pool, int64_t T, const Workspace& ws, cudaStream_t st);
 // phases: build the masked hi/lo copies of the r-vectors into hm, reduce from hm, or both
-enum { GRAD_PHASE_COPIES = 1, GRAD_PHASE_REDUCE = 2 };
+// GRAD_PHASE_EARLY: the reduction reads nothing the kernel before it in the stream writes and may start while that one ends
+enum { GRAD_PHASE_COPIES = 1, GRAD_PHASE_REDUCE = 2, GRAD_PHASE_EARLY = 4 };
 marlaas_status_t launch_grad_sm100(const marlaas_pool* pool, int64_t T, int64_t C, const bf16* src, int64_t ld,
                                    const float* hg, float* const* out_ptrs, float* const* host_ptrs, bool transpose_out,
                                    bool accumulate, const Workspace& ws, cudaStream_t st, bf16* hm, int phases = GRAD_PHASE_COPIES | GRAD_PHASE_REDUCE);
