@@ -269,11 +269,17 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
         const bool pre_zero = T >= 512 && shrink_split_sm100_eligible(pool, T, pool->K);
         if (pre_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(h, 0, sizeof(float) * (size_t)NP * T * pool->RP, st));
         if (!(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = make_plan(pool, T, seg, flags, host_ts, ws, st)) != MARLAAS_OK) return rc;
-        // one shrink per projection (its block of A rows, its plane of h and hd), then ONE product over the side-by-side W
-        for (int p = 0; p < NP; ++p) {
-            const Workspace wp = part_workspace(pool, ws, p, T);
-            if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K, pool->K, wp,
-                             h + (size_t)p * T * pool->RP, st, pre_zero)) != MARLAAS_OK) return rc;
+        // ONE shrink over all projections' blocks of A rows where the cluster kernel applies (x is read once; planes of h
+        // and hd per projection), else one shrink per projection; then ONE product over the side-by-side W
+        if (NP > 1 && T >= 512 && shrink_split_sm100_parts_eligible(pool, T, pool->K, NP)) {
+            if ((rc = launch_shrink_split_sm100(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, pool->K, ws, h, st, pre_zero,
+                                                NP)) != MARLAAS_OK) return rc;
+        } else {
+            for (int p = 0; p < NP; ++p) {
+                const Workspace wp = part_workspace(pool, ws, p, T);
+                if ((rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K, pool->K, wp,
+                                 h + (size_t)p * T * pool->RP, st, pre_zero)) != MARLAAS_OK) return rc;
+            }
         }
         GemmOperands o;
         o.M = T; o.Nout = pool->N; o.Kc = pool->K;

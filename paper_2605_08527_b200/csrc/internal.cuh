@@ -214,7 +214,9 @@ marlaas_status_t launch_shrink_sm100(const marlaas_pool* pool, int64_t T, const 
 bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D);
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
                                            const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st,
-                                           bool out_is_zero = false);
+                                           bool out_is_zero = false, int P = 1);
+// whether ONE launch can serve all P blocks of adapter rows of a pool over several projections (planes of out and hd)
+bool shrink_split_sm100_parts_eligible(const marlaas_pool* pool, int64_t T, int64_t D, int P);
 
 // cuda_core_kernels.cu
 // h/g (fp32, [T][RP]) as launch_rowdot, plus the bf16 block-diagonal operand rows hd for the tensor-core path

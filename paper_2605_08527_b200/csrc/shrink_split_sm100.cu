@@ -4,6 +4,11 @@
 // the contraction dimension through the same TMA / tcgen05 pipeline, and every CTA's epilogue sends, for each token,
 // only the columns of the token's own tenant (at most RP floats) to the cluster's first CTA, which adds the C
 // partial vectors in rank order and writes the results.  No atomics: the sum order is fixed.
+//
+// A pool over several projections that read the same activations (P blocks of adapter rows, one per projection) is served
+// by ONE pass over the activations: an item's slab holds its units' rows of every block (virtual unit p * n + u = unit u
+// of block p, so items take 8 / P units), the accumulator one group of 16 columns per virtual unit, and the results go
+// to plane p of the outputs.
 #include "sm100_ptx.cuh"
 
 namespace marlaas {
@@ -30,9 +35,13 @@ struct ShrinkSplitArgs {
     int umax;
     const int32_t* d_rank;
     const float* d_scale;
-    float* out;       // [T][RP], zero-filled before the launch
-    bf16* hd;         // [T][hd_cols]
+    float* out;       // [P][T][RP], zero-filled before the launch
+    bf16* hd;         // [P][T][hd_cols]
     int hd_cols;
+    int P;            // blocks of adapter rows (projections of the pool) served by this pass
+    int sub;          // units per work item: SS_SUB_UNITS / P
+    int part_rows;    // store rows from one block to the next
+    long long out_plane, hd_plane;   // elements from one plane of out / hd to the next
     int32_t* status;
 };
 
@@ -147,7 +156,7 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // items per tile, then their exclusive scan (one warp, five tiles per lane)
     for (int m = threadIdx.x; m < SS_MAX_TILES; m += SS_THREADS)
-        s_first[m] = m < g.num_m_tiles ? (g.tile_nunits[m >> 1] + SS_SUB_UNITS - 1) / SS_SUB_UNITS : 0;
+        s_first[m] = m < g.num_m_tiles ? (g.tile_nunits[m >> 1] + g.sub - 1) / g.sub : 0;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(TMEM_COLS)
@@ -191,12 +200,13 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
             const int mid = (lo + hi + 1) >> 1;
             if (s_first[mid] <= item) lo = mid; else hi = mid - 1;
         }
-        const int m = lo, u0 = (item - s_first[lo]) * SS_SUB_UNITS;
+        const int m = lo, u0 = (item - s_first[lo]) * g.sub;
         const int nun = g.tile_nunits[m >> 1];
-        const int nug = min(SS_SUB_UNITS, nun - u0);
+        const int nug = min(g.sub, nun - u0);
+        const int nvu = nug * g.P;                // virtual units: the item's units in every block of adapter rows
         const int32_t* units = g.tile_units + (size_t)(m >> 1) * g.umax + u0;
         // this item's stage geometry
-        const uint32_t b_panel = (uint32_t)nug * UNIT_BYTES, stage_bytes = KP * (A_STAGE_BYTES + b_panel);
+        const uint32_t b_panel = (uint32_t)nvu * UNIT_BYTES, stage_bytes = KP * (A_STAGE_BYTES + b_panel);
         const uint32_t nst = min((uint32_t)SS_MAX_STAGES, g.stage_area / stage_bytes);
 
         // per-row routing (epilogue threads): the row's units within the tile's list
@@ -217,7 +227,10 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
 
         if (warp == 0) {
             if (lane == 0 && ok) {   // ---- TMA producer: this CTA's slice of the contraction
-                const int nruns = ss_plan_runs(units, nug, s_runs);
+                int32_t vunits[SS_SUB_UNITS];
+                for (int p = 0; p < g.P; ++p)
+                    for (int u = 0; u < nug; ++u) vunits[p * nug + u] = units[u] + p * g.part_rows;
+                const int nruns = ss_plan_runs(vunits, nvu, s_runs);
                 uint32_t p_s = 0;
                 p_issued = 0;
                 p_stages = nst;
@@ -239,7 +252,7 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
             __syncwarp();
         } else if (warp == 1) {
             if (lane == 0 && ok) {   // ---- MMA issuer
-                const uint32_t idesc = make_idesc(nug * 16, 0);
+                const uint32_t idesc = make_idesc(nvu * 16, 0);
                 uint32_t acc = 0, m_s = 0;
                 for (int ks = ks0; ks < ks1 && ok; ++ks) {
                     if (!(ok = mbar_wait(bar_full + 8 * m_s, (m_mask >> m_s) & 1u, abort_word, 54))) break;
@@ -275,16 +288,16 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         if (warp >= 2) {
             // ---- this CTA's partial values of the row's own tenant columns -> gather buffer of CTA 0
             if (ok) {
-                const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)g.RP) * 4u;
+                const uint32_t gdst = ss_map_to_cta(sG, 0) + ((crank * 128u + (uint32_t)rl) * (uint32_t)(g.P * g.RP)) * 4u;
                 const bool empty_slice = ks0 >= ks1;      // no step: the accumulator was never written
 #pragma unroll 1
-                for (int u = 0; u < nug; ++u) {
+                for (int vu = 0; vu < nvu; ++vu) {
                     uint32_t v[16];
-                    ss_tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + u * 16, v);
+                    ss_tc_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + vu * 16, v);
                     tc_wait_ld();
-                    const int gu = u0 + u;
+                    const int p = vu / nug, gu = u0 + (vu - p * nug);
                     if (uo >= 0 && gu >= uo && gu < uo + nu) {
-                        const uint32_t a = gdst + (uint32_t)(gu - uo) * 64u;
+                        const uint32_t a = gdst + (uint32_t)(p * g.RP) * 4u + (uint32_t)(gu - uo) * 64u;
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             if (empty_slice) ss_st_cluster_v4(a + e * 16, 0u, 0u, 0u, 0u);
@@ -302,19 +315,20 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
         tc_fence_after();
         if (crank == 0 && warp >= 2 && row < g.T && ok) {
             const float* gbuf = reinterpret_cast<const float*>(smem);
-            bf16* hrow = g.hd + (size_t)row * g.hd_cols;
-            for (int u = 0; u < nug; ++u) {
-                const int gu = u0 + u;
+            const int prp = g.P * g.RP;
+            for (int vu = 0; vu < nvu; ++vu) {
+                const int p = vu / nug, gu = u0 + (vu - p * nug);
+                bf16* hrow = g.hd + (size_t)p * g.hd_plane + (size_t)row * g.hd_cols;
                 uint4 o0 = make_uint4(0u, 0u, 0u, 0u), o1 = o0;
                 if (uo >= 0 && gu >= uo && gu < uo + nu) {
                     float v[16];
 #pragma unroll
                     for (int e = 0; e < 16; ++e) v[e] = 0.f;
                     for (int c = 0; c < g.C; ++c) {      // fixed order
-                        const float4* p = reinterpret_cast<const float4*>(gbuf + ((size_t)c * 128 + rl) * g.RP + (gu - uo) * 16);
+                        const float4* src4 = reinterpret_cast<const float4*>(gbuf + ((size_t)c * 128 + rl) * prp + p * g.RP + (gu - uo) * 16);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float4 t4 = p[e];
+                            const float4 t4 = src4[e];
                             v[4 * e] += t4.x; v[4 * e + 1] += t4.y; v[4 * e + 2] += t4.z; v[4 * e + 3] += t4.w;
                         }
                     }
@@ -325,7 +339,7 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
                                     *reinterpret_cast<uint32_t*>(&pk[2]), *reinterpret_cast<uint32_t*>(&pk[3]));
                     o1 = make_uint4(*reinterpret_cast<uint32_t*>(&pk[4]), *reinterpret_cast<uint32_t*>(&pk[5]),
                                     *reinterpret_cast<uint32_t*>(&pk[6]), *reinterpret_cast<uint32_t*>(&pk[7]));
-                    float4* dst = reinterpret_cast<float4*>(g.out + (size_t)row * g.RP + (gu - uo) * 16);
+                    float4* dst = reinterpret_cast<float4*>(g.out + (size_t)p * g.out_plane + (size_t)row * g.RP + (gu - uo) * 16);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                 }
@@ -374,13 +388,13 @@ k_shrink_split_sm100(const __grid_constant__ CUtensorMap tmSrc, const __grid_con
 // Cluster width for T tokens: as many CTAs per tile as keep one cluster per tile resident in a single wave (0 = this
 // kernel does not apply: more tiles than SMs, where the persistent one-CTA-per-tile kernel is the better fit).
 static int split_width(const marlaas_pool* pool, int64_t tiles, int64_t num_kb, size_t* smem_out, int* stages_out,
-                       int* clusters_out) {
+                       int* clusters_out, int P = 1) {
     using namespace sm100;
     if (tiles > pool->sm_count || tiles > SS_MAX_TILES) return 0;
     static int max_active[64][SS_MAX_C + 1] = {};
     for (int C = SS_MAX_C; C >= 1; --C) {
         if ((int64_t)C * tiles > pool->sm_count || (C > 1 && num_kb < 16 * C)) continue;
-        const size_t gather = (size_t)C * 128 * pool->RP * 4;
+        const size_t gather = (size_t)C * 128 * pool->RP * 4 * (size_t)P;
         const size_t area = (222 * 1024 - 1024 - 256) / 1024 * 1024;      // stages; the gather buffer lies over them
         if (gather > area) continue;
         const int stages = (int)area;
@@ -414,15 +428,23 @@ bool shrink_split_sm100_eligible(const marlaas_pool* pool, int64_t T, int64_t D)
     return T > 0 && (D % 64) == 0 && split_width(pool, cdiv(T, sm100::BM), cdiv(D, sm100::BK), &smem, &stages, &clusters) > 0;
 }
 
+// All P blocks of adapter rows of a pool over several projections in one pass over the activations (the blocks lie one
+// after the other in the store, cap * RP rows each; out and hd are P planes of T rows).
+bool shrink_split_sm100_parts_eligible(const marlaas_pool* pool, int64_t T, int64_t D, int P) {
+    size_t smem; int stages, clusters;
+    return T > 0 && P >= 1 && P <= 4 && (D % 64) == 0 &&
+           split_width(pool, cdiv(T, sm100::BM), cdiv(D, sm100::BK), &smem, &stages, &clusters, P) > 0;
+}
+
 marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, const bf16* src, int64_t ld, int64_t D,
                                            const bf16* store, int64_t sld, const Workspace& ws, float* out, cudaStream_t st,
-                                           bool out_is_zero) {
+                                           bool out_is_zero, int P) {
     using namespace sm100;
     if (T <= 0) return MARLAAS_OK;
     const int64_t tiles = cdiv(T, BM);
     size_t smem_bytes = 0;
     int stages = 0, clusters = 0;
-    const int C = split_width(pool, tiles, cdiv(D, BK), &smem_bytes, &stages, &clusters);
+    const int C = split_width(pool, tiles, cdiv(D, BK), &smem_bytes, &stages, &clusters, P);
     if (C <= 0) return fail(MARLAAS_ERR_INVALID_ARG, "shrink_split: %lld tiles do not fit one wave", (long long)tiles);
     ShrinkSplitArgs g;
     g.T = (int)T; g.D = (int)D;
@@ -434,14 +456,16 @@ marlaas_status_t launch_shrink_split_sm100(const marlaas_pool* pool, int64_t T, 
     g.tile_nunits = ws.tile_nunits; g.tile_units = ws.tile_units; g.umax = ws.umax;
     g.d_rank = pool->d_rank; g.d_scale = pool->d_scale;
     g.out = out; g.hd = ws.hd; g.hd_cols = ws.umax * 16;
+    g.P = P; g.sub = SS_SUB_UNITS / P; g.part_rows = pool->cap * pool->RP;
+    g.out_plane = (long long)T * pool->RP; g.hd_plane = (long long)T * g.hd_cols;
     g.status = pool->d_status;
     alignas(64) CUtensorMap tmSrc;
     alignas(64) StoreMaps maps;
     marlaas_status_t rc;
     if ((rc = make_panel_map(&tmSrc, src, T, D, ld, SS_KP)) != MARLAAS_OK) return rc;
     for (int i = 0; i < 4; ++i)
-        if ((rc = make_map(&maps.m[i], store, (int64_t)pool->cap * pool->RP, D, sld, BK, 16u << i)) != MARLAAS_OK) return rc;
-    if (!out_is_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)T * pool->RP, st));
+        if ((rc = make_map(&maps.m[i], store, (int64_t)P * pool->cap * pool->RP, D, sld, BK, 16u << i)) != MARLAAS_OK) return rc;
+    if (!out_is_zero) MARLAAS_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(float) * (size_t)P * T * pool->RP, st));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(clusters * C));
     cfg.blockDim = dim3(SS_THREADS);

@@ -111,6 +111,14 @@ def test_store_roundtrip_of_a_pool_over_three_projections():
     (700, 128, (256, 512), (16, 8, 24, 16), False, 0),                    # training shape below 1024 rows
     (1500, 192, (256, 256, 512), (16, 32, 8, 64, 16), False, 0),          # training shape, several row tiles
     (300, 136, (256, 256), (16, 8, 24), False, B.MARLAAS_FLAG_CUDA_CORE_PATH),
+    # one shrink over all projections' adapter rows, the contraction cut over a cluster: three planes of rank stride 64
+    (1500, 4096, (256, 512, 256), (16, 32, 8, 64, 16), False, 0),
+    # every token its own tenant: eight and more units per 128-token tile, four per work item with two projections; a tenant
+    # of three units lies across two items
+    (900, 2048, (512, 256), (16, 8, 16, 40, 16, 16, 24, 16, 16), True, 0),
+    (640, 1024, (256, 256, 256, 256), (16, 24, 8), True, 0),              # four projections: two units per work item
+    (600, 512, (256, 256, 256, 256), (128, 16), False, 0),                # rank stride 128 x 4 planes: one shrink per projection
+    (777, 1024, (256, 512), (16, 16), False, 0),                          # last tile with 9 rows
 ])
 def test_forward_of_a_pool_over_several_projections(T, K, Ns, ranks, per_token, flags):
     w = _case(900 + T, T, K, Ns, ranks, per_token)
@@ -138,6 +146,7 @@ def test_forward_of_a_pool_over_several_projections(T, K, Ns, ranks, per_token, 
     (150, 64, (256, 256), (16, 8), 0, True),
     (1100, 128, (512, 256), (16, 0, 24, 8), 0, True),             # a tenant of rank 0: no gradient arrays, base-only rows
     (300, 136, (256, 256), (16, 8, 24), B.MARLAAS_FLAG_CUDA_CORE_PATH, True),
+    (1300, 2048, (256, 256, 512), (16, 32, 8, 64), 0, True),      # forward through one shrink over the three projections
 ])
 def test_backward_of_a_pool_over_several_projections(T, K, Ns, ranks, flags, saved):
     w = _case(1700 + T, T, K, Ns, ranks, False)
