@@ -547,6 +547,13 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
         }
         if (tc_grad && !(flags & MARLAAS_FLAG_REUSE_PLAN) && (rc = launch_grad_plan(pool, T, ws, st)) != MARLAAS_OK) return rc;
         if (!fits && (rc = launch_slot_sort(pool, T, ws.tok_slot, ws.slot_count, ws.slot_offset, ws.perm, st, run_flag)) != MARLAAS_OK) return rc;
+        // h was not kept: recomputed here, for all projections of the pool in one pass over x where the cluster kernel applies
+        bool h_all = false;
+        if (want_dB && !h_saved && tc_path && NP > 1 && T >= 512 && shrink_split_sm100_parts_eligible(pool, T, pool->K, NP)) {
+            if ((rc = launch_shrink_split_sm100(pool, T, (const bf16*)x, ldx, pool->K, pool->d_At, pool->K, ws, ws.h, st, false,
+                                                NP)) != MARLAAS_OK) return rc;
+            h_all = true;
+        }
         for (int p = 0; p < NP; ++p) {
             if (tc_grad && (p > 0 || (flags & MARLAAS_FLAG_REUSE_PLAN)))
                 MARLAAS_CUDA_TRY(cudaMemsetAsync(ws.gflag + 2, 0, 2 * sizeof(int32_t), st));
@@ -558,6 +565,7 @@ marlaas_status_t marlaas_lora_backward(marlaas_pool_t* pool, int64_t T, const vo
             const Workspace wp = part_workspace(pool, ws, p, T);
             if (want_dB) {
                 const float* h = h_saved ? h_saved + p * plane : nullptr;
+                if (!h && h_all) h = wp.h;
                 if (!h && T > 0) {
                     const bf16* Ap = pool->d_At + (size_t)p * pool->cap * pool->RP * pool->K;
                     if (tc_path) rc = shrink(pool, T, (const bf16*)x, ldx, pool->K, Ap, pool->K, wp, wp.h, st);
