@@ -9,7 +9,9 @@
 //                        row-major weight), the 256 tokens its N side (128 per CTA).  A 64-deep step brings as many bytes
 //                        of W as of x into a CTA (16 KB each), and one MMA covers 256 x 256 outputs, so the single
 //                        MMA-issuing thread is not the limit.  Launched as a programmatic dependent of the shrink: it
-//                        streams W at once and waits for the shrink grid only before its first read of hd.
+//                        streams W at once and waits for the shrink grid only before its first read of hd.  A batch of
+//                        fewer than 256 tokens whose contraction is not cut runs with token tiles of 64, 128 or 192 (the
+//                        N of the MMA): fewer token rows per step, more steps in flight, no tensor work on empty rows.
 //
 // With at least 33 tiles (token tile x 256-column strip) every tile's contraction stays in one CTA pair and nothing is
 // exchanged.  With fewer tiles the contraction is cut into S = 2 or 4 slices and the partial accumulators meet through an
