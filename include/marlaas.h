@@ -64,13 +64,28 @@ enum {
                                          refused with MARLAAS_ERR_INVALID_ARG) */
     MARLAAS_FLAG_VALIDATE_SYNC = 4u,  /* synchronise the stream after the call and return the device status word */
     MARLAAS_FLAG_CUDA_CORE_PATH = 8u, /* diagnostics: run the plain CUDA-core kernels instead of the tcgen05 path */
-    MARLAAS_FLAG_REUSE_PLAN = 16u     /* the workspace still holds the plan of the previous call of the same kind
+    MARLAAS_FLAG_REUSE_PLAN = 16u,    /* the workspace still holds the plan of the previous call of the same kind
                                          (forward after forward, backward after backward) and that call had the same T,
                                          the same segment table contents and a pool of the same capacity and max_rank:
                                          the per-token slots and per-tile unit lists are not rebuilt.  For the
                                          projections of one decoder layer, which all see the same mixed batch.  The
                                          caller vouches for the condition; batches of at most 1024 tokens ignore the
                                          flag (their plan is built inside the first kernel anyway). */
+    MARLAAS_FLAG_OVERLAP_PREVIOUS = 32u /* forward, decode-shaped batches (at most 1024 tokens): the caller states that the
+                                         work submitted to the stream immediately before this call -- typically the same
+                                         layer's call for another micro-batch of a serving loop that interleaves two --
+                                         is independent of it: it does not produce this call's x, W or segment table,
+                                         and it touches neither this call's workspace, y, h_save nor its pool.  The
+                                         call's first kernel (the shrink) is then launched behind that work as a
+                                         programmatic dependent that does not wait for it, and runs beside the end of
+                                         it; a preceding marlaas_lora_forward lets it start once its own shrink has
+                                         completed, so at most two consecutive calls are in flight together (two
+                                         workspaces and two pools, used in turn, satisfy the condition).  Stream order
+                                         holds for everything submitted after the call: it never completes before its
+                                         predecessor.  Results are bit-identical with and without the flag.  Ignored
+                                         for larger batches and with MARLAAS_FLAG_HOST_TABLE; refused by
+                                         marlaas_lora_forward_multi and marlaas_lora_forward_static_ws.  If the
+                                         condition does not hold the call races with its predecessor. */
 };
 
 /* Token-to-adapter segment table of one mixed batch: segment s covers tokens

@@ -32,6 +32,7 @@ MARLAAS_FLAG_HOST_TABLE = 2
 MARLAAS_FLAG_VALIDATE_SYNC = 4
 MARLAAS_FLAG_CUDA_CORE_PATH = 8
 MARLAAS_FLAG_REUSE_PLAN = 16
+MARLAAS_FLAG_OVERLAP_PREVIOUS = 32
 
 EXPORTED_SYMBOLS = [
     "marlaas_adapter_pool_storage_bytes", "marlaas_adapter_pool_create", "marlaas_adapter_pool_destroy",

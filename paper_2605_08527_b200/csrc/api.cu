@@ -228,7 +228,8 @@ static marlaas_status_t forward_impl(marlaas_pool_t* pool, int64_t T, const void
     std::vector<int32_t> host_ts;
     if ((rc = check_segments(fn, pool, T, seg, flags, &host_ts)) != MARLAAS_OK) return rc;
     if (!workspace || ((uintptr_t)workspace & 255)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: workspace NULL or misaligned", fn);
-    const Workspace ws = carve_workspace(pool, T, workspace);
+    Workspace ws = carve_workspace(pool, T, workspace);
+    ws.early_shrink = (flags & MARLAAS_FLAG_OVERLAP_PREVIOUS) && !(flags & MARLAAS_FLAG_HOST_TABLE);
     if (workspace_bytes < ws.fwd_min)
         return fail(MARLAAS_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < required %zu", fn, workspace_bytes, ws.fwd_min);
     // between the minimum and the full forward size the scratch for exchanged partial sums is missing: the decode kernels
@@ -322,8 +323,8 @@ marlaas_status_t marlaas_lora_forward_multi(int32_t n, const marlaas_forward_cal
     const char* fn = "lora_forward_multi";
     if (n < 0 || (n > 0 && !calls)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: bad call list", fn);
     if (n == 0) return MARLAAS_OK;
-    if (flags & (MARLAAS_FLAG_VALIDATE_SYNC | MARLAAS_FLAG_REUSE_PLAN))
-        return fail(MARLAAS_ERR_INVALID_ARG, "%s: VALIDATE_SYNC and REUSE_PLAN do not apply to a set of concurrent calls", fn);
+    if (flags & (MARLAAS_FLAG_VALIDATE_SYNC | MARLAAS_FLAG_REUSE_PLAN | MARLAAS_FLAG_OVERLAP_PREVIOUS))
+        return fail(MARLAAS_ERR_INVALID_ARG, "%s: VALIDATE_SYNC, REUSE_PLAN and OVERLAP_PREVIOUS do not apply to a set of concurrent calls", fn);
     marlaas_status_t rc;
     // every call is validated before anything is launched
     for (int i = 0; i < n; ++i) {

@@ -199,7 +199,10 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
         }
     }
     __syncthreads();
-    if (gi * DS_PASS >= n_t) return;     // nothing for this cluster (uniform over it)
+    if (gi * DS_PASS >= n_t) {           // nothing for this cluster (uniform over it)
+        if (threadIdx.x == 0) dk_wait_prerequisites();
+        return;
+    }
 
     const int own0 = r_t > 0 ? t * g.RP : 0, own1 = r_t > 0 ? own0 + g.RP : 0;   // hd columns written by the MMA part
     const int ngroups = (r_t + 15) >> 4;
@@ -217,7 +220,10 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
         if (r_t == 0)
             for (int j = lane; j < g.RP; j += 32) h_out[(size_t)tok * g.RP + j] = 0.f;
     }
-    if (r_t == 0) return;        // uniform over the cluster
+    if (r_t == 0) {              // uniform over the cluster
+        if (threadIdx.x == 0) dk_wait_prerequisites();
+        return;
+    }
 
     for (int p0 = gi * DS_PASS; p0 < n_t; p0 += DS_PASS * g.G) {
         const int np = min(DS_PASS, n_t - p0);
@@ -299,6 +305,9 @@ __global__ void __launch_bounds__(DS_THREADS, 4) k_decode_shrink(const DecodeShr
             }
         }
     }
+    // With MARLAAS_FLAG_OVERLAP_PREVIOUS this grid was launched behind the previous call's GEMM without waiting for it:
+    // it must not complete first (what follows in the stream relies on stream order).  A no-op otherwise.
+    if (threadIdx.x == 0) dk_wait_prerequisites();
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -505,6 +514,14 @@ k_decode_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         __syncwarp();
     } else {
         // ================= epilogue warps: wait for the pair's accumulator =================
+        // Idle until then, one of them hands over to the next call: once the shrink grid has completed (and with it
+        // whatever that grid was launched behind), a next call launched with MARLAAS_FLAG_OVERLAP_PREVIOUS may start its
+        // shrink beside the rest of this kernel.  Every CTA does this, so the hand-over happens as early as it may.
+        if (warp == 2 && lane == 0) {
+            dk_wait_prerequisites();
+            dk_launch_dependents();
+        }
+        __syncwarp();
         epi_ok = mbar_wait(bar_tfull, 0, abort_word, 46);
         epi_ok = __all_sync(0xffffffffu, epi_ok);
         tc_fence_after();
@@ -676,10 +693,14 @@ marlaas_status_t launch_decode_shrink(const marlaas_pool* pool, int64_t T, const
     cfg.blockDim = dim3(DS_THREADS);
     cfg.dynamicSmemBytes = decode_shrink_dyn_smem(T, S);
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
+    // the caller has stated that the previous call on the stream is independent of this one: the shrink starts once that
+    // call's GEMM has let its dependents go (after its own shrink has completed) and runs beside it
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = ws.early_shrink ? 2 : 1;
     MARLAAS_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_decode_shrink, a));
     count_launch();
     return MARLAAS_OK;

@@ -256,6 +256,14 @@ k_decode_gemm_wide(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         // columns are the tile's tokens.  Slice j finishes token columns [j Wd, (j + 1) Wd), Wd = 256 / S; the two warps
         // of a lane quarter split each such range in halves of nch chunks of 32 columns.
         const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
+        // Idle until the accumulator is complete, one epilogue thread hands over to the next call: once the shrink grid
+        // has completed (and with it whatever that grid was launched behind), a next call launched with
+        // MARLAAS_FLAG_OVERLAP_PREVIOUS may start its shrink beside the rest of this kernel.  Every CTA does this.
+        if (ew == 0 && lane == 0) {
+            dk_wait_prerequisites();
+            dk_launch_dependents();
+        }
+        __syncwarp();
         bool epi_ok = mbar_wait(bar_tfull, 0, abort_word, 46);
         epi_ok = __all_sync(0xffffffffu, epi_ok);
         tc_fence_after();
@@ -530,10 +538,18 @@ k_decode_gemm_stream(const __grid_constant__ CUtensorMap tmW, const __grid_const
                         dk_wait_prerequisites();
                         fence_proxy_async_all();
                         hd_ready = true;
+                        // the shrink grid has completed (and with it whatever it was launched behind): a next call launched
+                        // with MARLAAS_FLAG_OVERLAP_PREVIOUS may start its shrink beside the rest of this kernel (here the
+                        // epilogue warps are busy with early pieces, so the producer hands over)
+                        dk_launch_dependents();
                     }
                     if (have_rows) dg_tma_pair_3d(dx, mx, full0 + 8 * s, 0, ex ? hd_tok : my_tok, step);
                     if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1; }
                 }
+            }
+            if (ok && !hd_ready) {
+                dk_wait_prerequisites();
+                dk_launch_dependents();
             }
             if (!ok && half == 0) {
                 // let the copies already issued land (bounded) before shared memory is released

@@ -138,6 +138,8 @@ struct Workspace {
     bf16* hm2;             // a second set of copies, so that the dB and dA reductions need not share one
     int32_t max_copies, HW;
     size_t total;
+    bool early_shrink = false;   // this call: the decode shrink is launched behind the stream's previous kernel without
+                                 // waiting for it (MARLAAS_FLAG_OVERLAP_PREVIOUS)
 };
 Workspace carve_workspace(const marlaas_pool* pool, int64_t T, void* base);
 

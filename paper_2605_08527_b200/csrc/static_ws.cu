@@ -53,6 +53,9 @@ marlaas_status_t marlaas_lora_forward_static_ws(marlaas_pool_t* pool, int64_t T,
     const char* fn = "lora_forward_static_ws";
     if (!pool) return fail(MARLAAS_ERR_INVALID_ARG, "%s: pool is NULL", fn);
     if (T < 0 || T >= (1ll << 31)) return fail(MARLAAS_ERR_INVALID_ARG, "%s: T out of range", fn);
+    if (flags & MARLAAS_FLAG_OVERLAP_PREVIOUS)
+        return fail(MARLAAS_ERR_INVALID_ARG, "%s: MARLAAS_FLAG_OVERLAP_PREVIOUS needs a workspace of the call's own; every call "
+                    "through this entry uses the one built-in array", fn);
     if (T == 0) return MARLAAS_OK;
     // forward's share of the workspace, without the scratch only the kernels that exchange partial sums use
     const size_t need = marlaas_lora_forward_workspace_min_bytes(pool, T);
