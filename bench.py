@@ -403,6 +403,9 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra MARLAAS_FLAG_* bits for every call (diagnostics)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches even for forward-only workloads")
     ap.add_argument("--repeats", type=int, default=5, help="replays of the captured K-step graph (median reported)")
+    ap.add_argument("--overlap", action="store_true",
+                    help="forward-only workloads: every call carries MARLAAS_FLAG_OVERLAP_PREVIOUS and has a workspace of its own, "
+                         "as between two micro-batches that a serving loop interleaves (consecutive calls are independent)")
     ap.add_argument("--multi", action="store_true",
                     help="forward-only multi-projection workloads: q,k,v and gate,up through marlaas_lora_forward_multi (measured: no faster)")
     ap.add_argument("--headline-only", action="store_true", help="default workload without the `configs` entries of the other workloads")
@@ -473,6 +476,22 @@ def main():
         # which the one-pass-over-W kernels come closest to the copy peak
         for nm in ("decode5120x17408-256-32", "decode5120x17408-64-32"):
             extra(nm, wl.make_named_workload(nm), steps=20, repeats=5)
+        # the decode workloads once more with consecutive calls overlapped (independent calls, a workspace each: what a
+        # serving loop that interleaves two micro-batches submits); reported beside, never instead of, the figures above
+        import argparse as _ap
+        args_ov = _ap.Namespace(**{**vars(args), "overlap": True})
+
+        def extra_overlap(name, wk, steps=20, repeats=5):
+            time.sleep(1.0)
+            t0 = time.time()
+            d = measure(ctx, args_ov, wk, name, steps, 3, repeats, 0, False)
+            configs[name + "+overlap"] = summarize(d, time.time() - t0)
+
+        extra_overlap("cfg2", wl.make_named_workload("cfg2"), steps=50)
+        w5 = wl.make_named_workload("cfg5")
+        extra_overlap("cfg5-decode-fused", wl.make_variant("cfg5-decode-fused", w5))
+        del w5
+        extra_overlap("decode5120x17408-256-32", wl.make_named_workload("decode5120x17408-256-32"))
         out["configs"] = configs
     if rank == 0:
         print(json.dumps(out))
@@ -484,7 +503,7 @@ def summarize(d, seconds):
     """The figures of one extra workload that the one-line report carries."""
     r = d["roofline"]
     keep = {"metric": d["metric"], "tokens_per_s": d["value"], "ms_per_step": d["ms_per_step"], "ms_per_step_min": d["ms_per_step_min"],
-            "steps": d["steps"], "timed_as": d["config"]["timed_as"], "segments": d["config"]["segments"],
+            "steps": d["steps"], "timed_as": d["config"]["timed_as"], "calls": d["config"]["calls"], "segments": d["config"]["segments"],
             "tenants_present": d["config"]["tenants_present"], "gpu_launches": d["gpu_launches"], "clocks": d["clocks"],
             "work_per_step": d["work_per_step"], "wall_s": round(seconds, 1),
             "roofline": {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "traffic_source", "peak_source", "kernel",
@@ -523,6 +542,9 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
         + sum(x.nbytes for x in {id(p.x_bits): p.x_bits for p in w.projections}.values()) \
         + sum(2 * a.rank * (p.d_in + p.d_out) for p in w.projections for a in p.adapters)
     R = int(min(16, max(1, -(-3 * l2_bytes // input_bytes))))
+    overlap = bool(getattr(args, "overlap", False)) and not Tb
+    if overlap:
+        R = max(R, 2)      # consecutive calls must not share a pool: a single projection alternates between two copies
     l2_note = f"inputs of a step ({input_bytes / 1e6:.0f} MB) rotate over {R} independent copies (> 3x the {l2_bytes / 1e6:.0f} MB L2)" \
         if R > 1 else f"inputs of a step ({input_bytes / 1e6:.0f} MB) are larger than 3x the {l2_bytes / 1e6:.0f} MB L2"
     pinned = {}
@@ -583,8 +605,8 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
     # call each, which may run them side by side; o and down stay calls of their own (in a model they wait for attention
     # and for the activation function).  Concurrent calls need a workspace each.
     GROUPS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
-    use_multi = (not Tb) and len(w.projections) > 1 and args.multi
-    if use_multi:
+    use_multi = (not Tb) and len(w.projections) > 1 and args.multi and not overlap
+    if use_multi or overlap:
         for c in copies:
             for st_ in c:
                 st_["ws"] = torch.empty(max(B.marlaas_lora_forward_workspace_bytes(st_["pool"], w.T), 256), dtype=torch.uint8, device=dev)
@@ -606,6 +628,10 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
             return
         for j, s in enumerate(cs):
             fl = args.flags | (B.MARLAAS_FLAG_REUSE_PLAN if j > 0 else 0)
+            if overlap:
+                # the call before this one used another pool, another workspace and other outputs (the previous projection
+                # of this copy, or the last one of the previous copy), and its x, W and table are constants here
+                fl = args.flags | B.MARLAAS_FLAG_OVERLAP_PREVIOUS
             B.marlaas_lora_forward(s["pool"], x_of(s), s["W"], seg, y=s["y"], h_save=s["h"], workspace=s["ws"], flags=fl)
         if Tb:
             for j, s in enumerate(cs):
@@ -881,7 +907,9 @@ def measure(ctx, args, w, wname, steps, warmup, repeats, e2e_steps, want_cpu, su
                        "backward_tokens": Tb, "segments": int(len(w.seg_slot)),
                        "tenants_present": int(len(set(int(v) for v in ts_np.tolist() if v >= 0))), "l2": l2_note,
                        "timed_as": "one CUDA graph of K steps, median of %d replays" % reps if graph is not None else "K direct steps",
-                       "calls": "q,k,v and gate,up through marlaas_lora_forward_multi (independent projections side by side)" if use_multi else "one call per projection and pass",
+                       "calls": "q,k,v and gate,up through marlaas_lora_forward_multi (independent projections side by side)" if use_multi else ("one call per projection, each started beside the end of the one before (MARLAAS_FLAG_OVERLAP_PREVIOUS: consecutive calls "
+                                 "are independent, as between two interleaved micro-batches; a workspace per call)" if overlap else
+                                 "one call per projection and pass"),
                        "multi_gpu": "replicas only (independent copies of the batch per GPU, no collective)"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "sustained": sustained, "gpu_launches": int(launches),
             "clocks": clocks,
