@@ -104,7 +104,7 @@ def run_sweep(args):
     import subprocess
     for name in SWEEPS[args.sweep]:
         cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, "--steps", str(args.steps), "--warmup",
-               str(args.warmup), "--no-cpu-baseline", "--e2e-steps", "0", "--flags", str(args.flags)]
+               str(args.warmup), "--no-cpu-baseline", "--e2e-steps", "0", "--flags", str(args.flags)] + (["--overlap"] if args.overlap else [])
         r = subprocess.run(cmd, capture_output=True, text=True)
         lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
         if r.returncode != 0 or not lines:
