@@ -357,3 +357,25 @@ def test_unregister_and_reregister_on_a_pool_over_two_projections():
     assert_close(to_np(y2), _oracle_forward(w, ts)[0], "after registering again")
     assert B.marlaas_adapter_pool_lookup(sc.pool, t0.tenant_id)[3] == 7
     B.marlaas_check_status(sc.pool)
+
+
+@pytest.mark.parametrize("T,K,Ns", [
+    (96, 4096, (8192, 8192)),        # one tile per CTA pair, both projections' planes of hd
+    (64, 2048, (9728, 9728)),        # more tiles than CTA pairs
+    (200, 256, (512, 256, 256)),     # the token-major decode kernel
+])
+def test_overlapped_decode_calls_on_pools_over_several_projections(T, K, Ns):
+    # MARLAAS_FLAG_OVERLAP_PREVIOUS on pools over several projections: two pools used in turn, bit-identical to serial calls
+    w = _case(2300 + T, T, K, Ns, (16, 8, 32), True)
+    cases = [SegCase(w, capacity=4) for _ in range(2)]
+    ref = B.marlaas_lora_forward(cases[0].pool, cases[0].x, cases[0].W, cases[0].seg).clone()
+    torch.cuda.synchronize()
+    ys = [torch.empty_like(ref) for _ in range(6)]
+    for j in range(6):
+        c = cases[j % 2]
+        B.marlaas_lora_forward(c.pool, c.x, c.W, c.seg, y=ys[j], flags=B.MARLAAS_FLAG_OVERLAP_PREVIOUS)
+    torch.cuda.synchronize()
+    for y in ys:
+        assert torch.equal(y, ref)
+    for c in cases:
+        B.marlaas_check_status(c.pool)
