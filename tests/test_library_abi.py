@@ -78,3 +78,21 @@ def test_product_path_has_no_oracle_or_cpu_fallback():
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src, f
                 assert "marlaas_oracle" not in src, f
+
+
+def test_header_is_valid_c99(tmp_path):
+    # the boundary is a C ABI: the header must compile as plain C, with every flag a distinct power of two
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    flags = re.findall(r"\b(MARLAAS_FLAG_[A-Z_]+)\s*=\s*(\d+)u", open(os.path.join(ROOT, "include", "marlaas.h")).read())
+    values = [int(v) for _, v in flags]
+    assert len(flags) >= 6 and len(set(values)) == len(values) and all(v & (v - 1) == 0 for v in values)
+    src = tmp_path / "h.c"
+    src.write_text('#include "marlaas.h"\nint main(void) { return (int)sizeof(marlaas_segments_t) > 0 ? 0 : 1; }\n')
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                        "-c", str(src), "-o", str(tmp_path / "h.o")], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    for name, v in flags:
+        assert getattr(B, name) == int(v), name
